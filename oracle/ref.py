@@ -1,0 +1,162 @@
+"""ctypes front end of the CPU oracle (``sg_ref.c``).
+
+TEST INFRASTRUCTURE ONLY: the product (the CUDA library and its Python binding)
+never imports this module.  It marshals NumPy arrays into the plain-C loop
+nests, which evaluate the op definitions of the paper (Section 3 index
+notation for conv_1d_nwc_wcf; Section 4.6.1 for matmul; Section 4.6.2 for the
+strided/dilated 1-D and 2-D convolutions) with f64 accumulation.
+
+All functions take f32 NumPy arrays (any strides) and return
+``(out_f64, sum_abs_f64)`` where ``sum_abs`` is sum |a*b| per output element.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sg_ref.c")
+_LIB = os.path.join(_HERE, "libsgref.so")
+_lock = threading.Lock()
+_lib = None
+
+_i64 = ctypes.c_int64
+_p = ctypes.c_void_p
+
+
+def build(force: bool = False) -> str:
+    """Compile sg_ref.c into libsgref.so with gcc (no CUDA involved)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib():
+    global _lib
+    with _lock:
+        if _lib is None:
+            build()
+            _lib = ctypes.CDLL(_LIB)
+            _lib.sg_ref_max_threads.restype = ctypes.c_int
+    return _lib
+
+
+def max_threads() -> int:
+    return int(lib().sg_ref_max_threads())
+
+
+def _f32(a):
+    a = np.asarray(a)
+    if a.dtype != np.float32:
+        raise TypeError("oracle inputs must be float32 arrays")
+    return a
+
+
+def _estrides(a):
+    return [s // a.itemsize for s in a.strides]
+
+
+def _i64arr(v):
+    return (ctypes.c_int64 * len(v))(*[int(x) for x in v])
+
+
+def _ptr(a):
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def matmul(A, B, C_in=None, threads=0):
+    """C[m,n] = (C_in[m,n]) + sum_k A[m,k]*B[k,n]."""
+    A, B = _f32(A), _f32(B)
+    M, K = A.shape
+    K2, N = B.shape
+    assert K == K2
+    mode = 0 if C_in is None else 1
+    C = np.zeros((M, N), np.float64) if C_in is None else np.array(C_in, dtype=np.float64, order="C")
+    S = np.zeros((M, N), np.float64)
+    sa, sb = _estrides(A), _estrides(B)
+    rc = lib().sg_ref_matmul(_i64(M), _i64(N), _i64(K), _ptr(A), _i64(sa[0]), _i64(sa[1]),
+                             _ptr(B), _i64(sb[0]), _i64(sb[1]), _ptr(C), _i64(N), _i64(1),
+                             _ptr(S), ctypes.c_int(mode), ctypes.c_int(threads))
+    if rc:
+        raise ValueError("sg_ref_matmul rejected its arguments")
+    return C, S
+
+
+def matmul_points(A, B, pm, pn, threads=0):
+    A, B = _f32(A), _f32(B)
+    K = A.shape[1]
+    pm = np.ascontiguousarray(pm, np.int64)
+    pn = np.ascontiguousarray(pn, np.int64)
+    out = np.zeros(pm.shape[0], np.float64)
+    sab = np.zeros(pm.shape[0], np.float64)
+    sa, sb = _estrides(A), _estrides(B)
+    lib().sg_ref_matmul_points(_i64(K), _ptr(A), _i64(sa[0]), _i64(sa[1]), _ptr(B), _i64(sb[0]),
+                               _i64(sb[1]), _i64(pm.shape[0]), _ptr(pm), _ptr(pn), _ptr(out),
+                               _ptr(sab), ctypes.c_int(threads))
+    return out, sab
+
+
+def conv1d_nwc_wcf(I, Kf, stride=1, dilation=1, O_in=None, W_out=None, threads=0):
+    """O[n,w,f] = (O_in) + sum_{kw,c} I[n, w*stride + kw*dilation, c] * Kf[kw,c,f]."""
+    I, Kf = _f32(I), _f32(Kf)
+    N, W_in, C = I.shape
+    KW, C2, F = Kf.shape
+    assert C == C2
+    if W_out is None:
+        W_out = (W_in - (KW - 1) * dilation - 1) // stride + 1
+    mode = 0 if O_in is None else 1
+    O = np.zeros((N, W_out, F), np.float64) if O_in is None else np.array(O_in, dtype=np.float64, order="C")
+    S = np.zeros((N, W_out, F), np.float64)
+    rc = lib().sg_ref_conv1d_nwc_wcf(_i64(N), _i64(W_out), _i64(F), _i64(KW), _i64(C), _i64(W_in),
+                                     _i64(stride), _i64(dilation), _ptr(I), _i64arr(_estrides(I)),
+                                     _ptr(Kf), _i64arr(_estrides(Kf)), _ptr(O),
+                                     _i64arr([W_out * F, F, 1]), _ptr(S), ctypes.c_int(mode),
+                                     ctypes.c_int(threads))
+    if rc:
+        raise ValueError("sg_ref_conv1d_nwc_wcf rejected its arguments")
+    return O, S
+
+
+def conv2d_nhwc_hwcf(I, Kf, stride=(1, 1), dilation=(1, 1), O_in=None, out_hw=None, threads=0):
+    """O[n,h,w,f] = (O_in) + sum_{kh,kw,c} I[n,h*sh+kh*dh,w*sw+kw*dw,c] * Kf[kh,kw,c,f]."""
+    I, Kf = _f32(I), _f32(Kf)
+    N, H_in, W_in, C = I.shape
+    KH, KW, C2, F = Kf.shape
+    assert C == C2
+    sh, sw = stride
+    dh, dw = dilation
+    if out_hw is None:
+        out_hw = ((H_in - (KH - 1) * dh - 1) // sh + 1, (W_in - (KW - 1) * dw - 1) // sw + 1)
+    Ho, Wo = out_hw
+    mode = 0 if O_in is None else 1
+    O = np.zeros((N, Ho, Wo, F), np.float64) if O_in is None else np.array(O_in, dtype=np.float64, order="C")
+    S = np.zeros((N, Ho, Wo, F), np.float64)
+    rc = lib().sg_ref_conv2d_nhwc_hwcf(_i64(N), _i64(Ho), _i64(Wo), _i64(F), _i64(KH), _i64(KW),
+                                       _i64(C), _i64(H_in), _i64(W_in), _i64(sh), _i64(sw),
+                                       _i64(dh), _i64(dw), _ptr(I), _i64arr(_estrides(I)),
+                                       _ptr(Kf), _i64arr(_estrides(Kf)), _ptr(O),
+                                       _i64arr([Ho * Wo * F, Wo * F, F, 1]), _ptr(S),
+                                       ctypes.c_int(mode), ctypes.c_int(threads))
+    if rc:
+        raise ValueError("sg_ref_conv2d_nhwc_hwcf rejected its arguments")
+    return O, S
+
+
+def conv2d_points(I, Kf, pn, ph, pw, pf, stride=(1, 1), dilation=(1, 1), threads=0):
+    I, Kf = _f32(I), _f32(Kf)
+    KH, KW, C, _ = Kf.shape
+    pts = [np.ascontiguousarray(p, np.int64) for p in (pn, ph, pw, pf)]
+    n = pts[0].shape[0]
+    out = np.zeros(n, np.float64)
+    sab = np.zeros(n, np.float64)
+    lib().sg_ref_conv2d_points(_i64(KH), _i64(KW), _i64(C), _i64(stride[0]), _i64(stride[1]),
+                               _i64(dilation[0]), _i64(dilation[1]), _ptr(I),
+                               _i64arr(_estrides(I)), _ptr(Kf), _i64arr(_estrides(Kf)), _i64(n),
+                               _ptr(pts[0]), _ptr(pts[1]), _ptr(pts[2]), _ptr(pts[3]), _ptr(out),
+                               _ptr(sab), ctypes.c_int(threads))
+    return out, sab
