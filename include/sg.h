@@ -1,0 +1,156 @@
+/*
+ * sg.h: C ABI of the structured contraction library for NVIDIA B200 (sm_100a).
+ *
+ * Three ops, each defined by a rectangular iteration domain and one indexing
+ * map per operand, evaluated on the GPU by hand-written CUDA kernels:
+ *
+ *   sg_matmul             C[m,n]     (+)= sum_k         A[m,k] * B[k,n]
+ *   sg_conv1d_nwc_wcf     O[n,w,f]   (+)= sum_{kw,c}    I[n, w*sw + kw*dw, c] * K[kw,c,f]
+ *   sg_conv2d_nhwc_hwcf   O[n,h,w,f] (+)= sum_{kh,kw,c} I[n, h*sh + kh*dh, w*sw + kw*dw, c] * K[kh,kw,c,f]
+ *
+ * Conventions common to all entry points
+ *   - Every data pointer is a DEVICE pointer owned by the caller.  Inputs are
+ *     read only; the output is written (SG_OVERWRITE) or read and written
+ *     (SG_ACCUMULATE).  The output must not overlap an input.
+ *   - Strides are in ELEMENTS of the operand's type (the strided-buffer
+ *     convention of the paper's memref type, Section 2.2), may be any
+ *     positive value and need not be dense.
+ *   - `in_dtype` is the element type of BOTH inputs.  The output is always
+ *     f32 and products are accumulated in f32 (bf16 inputs are widened
+ *     exactly; f32 inputs keep f32 accuracy).
+ *   - Calls only enqueue work on `stream` and return; they never synchronise
+ *     and never allocate device memory.  The first call on a device creates
+ *     small host-side state (driver entry points, a tensor-map cache).
+ *   - The return value reports argument and launch errors.  Device-side
+ *     pipeline time-outs (which indicate a library bug, not a user error) are
+ *     recorded in a per-device status word that sg_check() reads.
+ *   - Zero-sized parallel dimensions are a successful no-op.  A zero-sized
+ *     reduction zero-fills the output in SG_OVERWRITE mode and leaves it
+ *     untouched in SG_ACCUMULATE mode.
+ *   - Shapes whose layout allows it (unit stride on the contiguous dimension,
+ *     16-byte aligned bases and row pitches) run on the tensor-core path
+ *     (TMA + tcgen05, bf16 inputs); everything else runs on a strided
+ *     CUDA-core FFMA kernel.  There is no CPU fallback.
+ */
+#ifndef SG_H_
+#define SG_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Opaque stand-in for cudaStream_t so that this header needs no CUDA include. */
+typedef void *sg_stream_t;
+
+typedef enum {
+    SG_OK = 0,
+    SG_ERR_INVALID_ARG = 1,    /* null pointer, negative size, stride/dilation < 1, input too small */
+    SG_ERR_UNSUPPORTED = 2,    /* unknown dtype or mode, sizes beyond 2^31-1 per dimension         */
+    SG_ERR_ALIGNMENT = 3,      /* pointer not aligned to its element size                          */
+    SG_ERR_CUDA = 4,           /* a CUDA runtime or driver call failed                             */
+    SG_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait expired (reported by sg_check)        */
+    SG_ERR_INTERNAL = 6
+} sg_status;
+
+typedef enum { SG_F32 = 0, SG_BF16 = 1 } sg_dtype;
+
+enum { SG_OVERWRITE = 0, SG_ACCUMULATE = 1 };
+
+/* Kernel families, for sg_set_kernel_override(). */
+enum { SG_KERNEL_AUTO = 0, SG_KERNEL_FFMA = 1, SG_KERNEL_TENSOR = 2 };
+
+/*
+ * Matrix multiplication (paper Section 4.6.1, variant "AB"; iterators
+ * (m,n,k) = (parallel, parallel, reduction), maps A:(m,k) B:(k,n) C:(m,n)).
+ * The transposed variants of the same section are obtained through the
+ * stride arguments alone.
+ *   A  : M x K elements of in_dtype, element (m,k) at A[m*a_stride_m + k*a_stride_k]
+ *   B  : K x N elements of in_dtype, element (k,n) at B[k*b_stride_k + n*b_stride_n]
+ *   C  : M x N f32,                  element (m,n) at C[m*c_stride_m + n*c_stride_n]
+ *   mode: SG_OVERWRITE  C = A.B ;  SG_ACCUMULATE  C = C_in + A.B  (C is the tied
+ *         in/out operand of the destination-passing form, Section 3.4)
+ */
+sg_status sg_matmul(int64_t M, int64_t N, int64_t K,
+                    const void *A, int64_t a_stride_m, int64_t a_stride_k,
+                    const void *B, int64_t b_stride_k, int64_t b_stride_n,
+                    float *C, int64_t c_stride_m, int64_t c_stride_n,
+                    sg_dtype in_dtype, int mode, sg_stream_t stream);
+
+/*
+ * 1-D convolution, input layout NWC, filter layout WCF, output NWF
+ * (index notation of Section 3; strided/dilated form of Section 4.6.2, "(1-D)").
+ * Iteration domain 0<=n<N, 0<=w<W_out, 0<=f<F, 0<=kw<KW, 0<=c<C; the filter
+ * is not flipped and nothing is padded: the call is rejected unless
+ * W_in >= (W_out-1)*stride_w + (KW-1)*dilation_w + 1.  Input columns beyond
+ * that are not read.
+ *   I : N x W_in x C,   strides i_strides[3] = {n, w, c}
+ *   Kf: KW x C x F,     strides k_strides[3] = {kw, c, f}
+ *   O : N x W_out x F,  strides o_strides[3] = {n, w, f}   (f32)
+ */
+sg_status sg_conv1d_nwc_wcf(int64_t N, int64_t W_out, int64_t F, int64_t KW, int64_t C,
+                            int64_t W_in, int64_t stride_w, int64_t dilation_w,
+                            const void *I, const int64_t i_strides[3],
+                            const void *Kf, const int64_t k_strides[3],
+                            float *O, const int64_t o_strides[3],
+                            sg_dtype in_dtype, int mode, sg_stream_t stream);
+
+/*
+ * 2-D convolution, input NHWC, filter HWCF, output NHWF (Section 4.6.2, "(2-D)").
+ * Iteration domain (n,h,w,f,kh,kw,c); same rules as the 1-D op in both
+ * spatial dimensions.
+ *   I : N x H_in x W_in x C,    strides {n, h, w, c}
+ *   Kf: KH x KW x C x F,        strides {kh, kw, c, f}
+ *   O : N x H_out x W_out x F,  strides {n, h, w, f}   (f32)
+ */
+sg_status sg_conv2d_nhwc_hwcf(int64_t N, int64_t H_out, int64_t W_out, int64_t F,
+                              int64_t KH, int64_t KW, int64_t C, int64_t H_in, int64_t W_in,
+                              int64_t stride_h, int64_t stride_w,
+                              int64_t dilation_h, int64_t dilation_w,
+                              const void *I, const int64_t i_strides[4],
+                              const void *Kf, const int64_t k_strides[4],
+                              float *O, const int64_t o_strides[4],
+                              sg_dtype in_dtype, int mode, sg_stream_t stream);
+
+/*
+ * Synchronises `stream` and returns the current device's status word:
+ * SG_OK, SG_ERR_DEVICE_TIMEOUT if any kernel since the last sg_check gave up
+ * on a bounded wait (its output is then undefined), or SG_ERR_CUDA if the
+ * synchronisation itself failed.  Reading clears the word.
+ */
+sg_status sg_check(sg_stream_t stream);
+
+/* Static, NUL-terminated description of a status code. */
+const char *sg_status_string(sg_status status);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int sg_version(void);
+
+/*
+ * Which kernel family the most recent successful call on this host thread
+ * selected: SG_KERNEL_FFMA or SG_KERNEL_TENSOR (0 before any call).
+ */
+int sg_last_kernel(void);
+
+/*
+ * Number of kernels this library has launched in this process so far
+ * (monotonic, all threads).  Used by benchmarks to report launch counts.
+ */
+int64_t sg_launch_count(void);
+
+/*
+ * Force a kernel family for later calls on this process (testing and
+ * benchmarking): SG_KERNEL_AUTO restores the default selection.  Forcing
+ * SG_KERNEL_TENSOR makes calls whose layout the tensor-core path cannot take
+ * return SG_ERR_UNSUPPORTED instead of falling back.
+ */
+sg_status sg_set_kernel_override(int kernel_family);
+
+/* Drops cached tensor maps and other host-side state.  Safe to call twice. */
+void sg_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SG_H_ */

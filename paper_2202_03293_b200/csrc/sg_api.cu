@@ -1,0 +1,181 @@
+// C ABI entry points: argument validation, the implicit-GEMM view of each op, kernel selection.
+#include <atomic>
+#include <limits>
+
+#include "sg_internal.cuh"
+
+namespace sg {
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+std::atomic<int> g_override{SG_KERNEL_AUTO};
+thread_local int t_last_kernel = 0;
+
+constexpr int64_t kMaxDim = std::numeric_limits<int32_t>::max();
+
+inline bool fits(int64_t v) { return v >= 0 && v <= kMaxDim; }
+
+sg_status run(const Problem &p, const void *In, const void *Flt, float *O, cudaStream_t stream) {
+    if (p.M == 0 || p.N == 0) return SG_OK;                       // nothing to write
+    if (p.K == 0) {                                               // empty reduction: the sum is 0
+        if (p.accumulate) return SG_OK;
+        return launch_zero_fill(p, O, stream) == cudaSuccess ? SG_OK : SG_ERR_CUDA;
+    }
+    const int force = g_override.load();
+    if (force != SG_KERNEL_FFMA) {
+        sg_status st = launch_tensor(p, In, Flt, O, stream);
+        if (st == SG_OK) { t_last_kernel = SG_KERNEL_TENSOR; return SG_OK; }
+        if (st != SG_ERR_UNSUPPORTED || force == SG_KERNEL_TENSOR) return st;
+    }
+    if (launch_ffma(p, In, Flt, O, stream) != cudaSuccess) return SG_ERR_CUDA;
+    t_last_kernel = SG_KERNEL_FFMA;
+    return SG_OK;
+}
+
+sg_status check_common(const void *a, const void *b, const void *o, sg_dtype dt, int mode) {
+    if (dt != SG_F32 && dt != SG_BF16) return SG_ERR_UNSUPPORTED;
+    if (mode != SG_OVERWRITE && mode != SG_ACCUMULATE) return SG_ERR_UNSUPPORTED;
+    const uintptr_t es = dt == SG_BF16 ? 2 : 4;
+    if (a && reinterpret_cast<uintptr_t>(a) % es) return SG_ERR_ALIGNMENT;
+    if (b && reinterpret_cast<uintptr_t>(b) % es) return SG_ERR_ALIGNMENT;
+    if (o && reinterpret_cast<uintptr_t>(o) % 4) return SG_ERR_ALIGNMENT;
+    return SG_OK;
+}
+
+}  // namespace
+
+void count_launch(int n) { g_launches.fetch_add(n); }
+
+}  // namespace sg
+
+using namespace sg;
+
+extern "C" {
+
+sg_status sg_matmul(int64_t M, int64_t N, int64_t K, const void *A, int64_t a_stride_m, int64_t a_stride_k,
+                    const void *B, int64_t b_stride_k, int64_t b_stride_n, float *C, int64_t c_stride_m,
+                    int64_t c_stride_n, sg_dtype in_dtype, int mode, sg_stream_t stream) {
+    if (M < 0 || N < 0 || K < 0) return SG_ERR_INVALID_ARG;
+    sg_status st = check_common(A, B, C, in_dtype, mode);
+    if (st != SG_OK) return st;
+    if (!fits(M) || !fits(N) || !fits(K)) return SG_ERR_UNSUPPORTED;
+    const bool has_out = M > 0 && N > 0;
+    if (has_out && !C) return SG_ERR_INVALID_ARG;
+    if (has_out && K > 0 && (!A || !B)) return SG_ERR_INVALID_ARG;
+    if (a_stride_m < 0 || a_stride_k < 0 || b_stride_k < 0 || b_stride_n < 0 || c_stride_m < 0 || c_stride_n < 0)
+        return SG_ERR_INVALID_ARG;
+    Problem p{};
+    p.M = (int)M; p.N = (int)N; p.K = (int)K;
+    p.batch = 1; p.Ho = 1; p.Wo = (int)M;
+    p.KH = 1; p.KW = 1; p.C = (int)K;
+    p.Hin = 1; p.Win = (int)M;
+    p.sh = p.sw = p.dh = p.dw = 1;
+    p.i_n = 0; p.i_h = 0; p.i_w = a_stride_m; p.i_c = a_stride_k;
+    p.k_kh = 0; p.k_kw = 0; p.k_c = b_stride_k; p.k_f = b_stride_n;
+    p.o_n = 0; p.o_h = 0; p.o_w = c_stride_m; p.o_f = c_stride_n;
+    p.in_bf16 = in_dtype == SG_BF16; p.accumulate = mode == SG_ACCUMULATE; p.spatial_rank = 0;
+    return run(p, A, B, C, static_cast<cudaStream_t>(stream));
+}
+
+sg_status sg_conv1d_nwc_wcf(int64_t N, int64_t W_out, int64_t F, int64_t KW, int64_t C, int64_t W_in,
+                            int64_t stride_w, int64_t dilation_w, const void *I, const int64_t i_strides[3],
+                            const void *Kf, const int64_t k_strides[3], float *O, const int64_t o_strides[3],
+                            sg_dtype in_dtype, int mode, sg_stream_t stream) {
+    if (N < 0 || W_out < 0 || F < 0 || KW < 0 || C < 0 || W_in < 0) return SG_ERR_INVALID_ARG;
+    if (stride_w < 1 || dilation_w < 1) return SG_ERR_INVALID_ARG;
+    if (!i_strides || !k_strides || !o_strides) return SG_ERR_INVALID_ARG;
+    sg_status st = check_common(I, Kf, O, in_dtype, mode);
+    if (st != SG_OK) return st;
+    for (int i = 0; i < 3; ++i)
+        if (i_strides[i] < 0 || k_strides[i] < 0 || o_strides[i] < 0) return SG_ERR_INVALID_ARG;
+    if (!fits(N) || !fits(W_out) || !fits(F) || !fits(KW) || !fits(C) || !fits(W_in) || !fits(stride_w) ||
+        !fits(dilation_w)) return SG_ERR_UNSUPPORTED;
+    if (W_out > 0 && KW > 0 && W_in < (W_out - 1) * stride_w + (KW - 1) * dilation_w + 1) return SG_ERR_INVALID_ARG;
+    if (!fits(N * W_out) || !fits(KW * C)) return SG_ERR_UNSUPPORTED;
+    const bool has_out = N > 0 && W_out > 0 && F > 0;
+    if (has_out && !O) return SG_ERR_INVALID_ARG;
+    if (has_out && KW * C > 0 && (!I || !Kf)) return SG_ERR_INVALID_ARG;
+    Problem p{};
+    p.M = (int)(N * W_out); p.N = (int)F; p.K = (int)(KW * C);
+    p.batch = (int)N; p.Ho = 1; p.Wo = (int)W_out;
+    p.KH = 1; p.KW = (int)KW; p.C = (int)C;
+    p.Hin = 1; p.Win = (int)W_in;
+    p.sh = 1; p.sw = (int)stride_w; p.dh = 1; p.dw = (int)dilation_w;
+    p.i_n = i_strides[0]; p.i_h = 0; p.i_w = i_strides[1]; p.i_c = i_strides[2];
+    p.k_kh = 0; p.k_kw = k_strides[0]; p.k_c = k_strides[1]; p.k_f = k_strides[2];
+    p.o_n = o_strides[0]; p.o_h = 0; p.o_w = o_strides[1]; p.o_f = o_strides[2];
+    p.in_bf16 = in_dtype == SG_BF16; p.accumulate = mode == SG_ACCUMULATE; p.spatial_rank = 1;
+    return run(p, I, Kf, O, static_cast<cudaStream_t>(stream));
+}
+
+sg_status sg_conv2d_nhwc_hwcf(int64_t N, int64_t H_out, int64_t W_out, int64_t F, int64_t KH, int64_t KW, int64_t C,
+                              int64_t H_in, int64_t W_in, int64_t stride_h, int64_t stride_w, int64_t dilation_h,
+                              int64_t dilation_w, const void *I, const int64_t i_strides[4], const void *Kf,
+                              const int64_t k_strides[4], float *O, const int64_t o_strides[4], sg_dtype in_dtype,
+                              int mode, sg_stream_t stream) {
+    if (N < 0 || H_out < 0 || W_out < 0 || F < 0 || KH < 0 || KW < 0 || C < 0 || H_in < 0 || W_in < 0)
+        return SG_ERR_INVALID_ARG;
+    if (stride_h < 1 || stride_w < 1 || dilation_h < 1 || dilation_w < 1) return SG_ERR_INVALID_ARG;
+    if (!i_strides || !k_strides || !o_strides) return SG_ERR_INVALID_ARG;
+    sg_status st = check_common(I, Kf, O, in_dtype, mode);
+    if (st != SG_OK) return st;
+    for (int i = 0; i < 4; ++i)
+        if (i_strides[i] < 0 || k_strides[i] < 0 || o_strides[i] < 0) return SG_ERR_INVALID_ARG;
+    if (!fits(N) || !fits(H_out) || !fits(W_out) || !fits(F) || !fits(KH) || !fits(KW) || !fits(C) || !fits(H_in) ||
+        !fits(W_in) || !fits(stride_h) || !fits(stride_w) || !fits(dilation_h) || !fits(dilation_w))
+        return SG_ERR_UNSUPPORTED;
+    if (H_out > 0 && KH > 0 && H_in < (H_out - 1) * stride_h + (KH - 1) * dilation_h + 1) return SG_ERR_INVALID_ARG;
+    if (W_out > 0 && KW > 0 && W_in < (W_out - 1) * stride_w + (KW - 1) * dilation_w + 1) return SG_ERR_INVALID_ARG;
+    if (!fits(H_out * W_out) || !fits(N * H_out * W_out) || !fits(KH * KW) || !fits(KH * KW * C))
+        return SG_ERR_UNSUPPORTED;
+    const bool has_out = N > 0 && H_out > 0 && W_out > 0 && F > 0;
+    if (has_out && !O) return SG_ERR_INVALID_ARG;
+    if (has_out && KH * KW * C > 0 && (!I || !Kf)) return SG_ERR_INVALID_ARG;
+    Problem p{};
+    p.M = (int)(N * H_out * W_out); p.N = (int)F; p.K = (int)(KH * KW * C);
+    p.batch = (int)N; p.Ho = (int)H_out; p.Wo = (int)W_out;
+    p.KH = (int)KH; p.KW = (int)KW; p.C = (int)C;
+    p.Hin = (int)H_in; p.Win = (int)W_in;
+    p.sh = (int)stride_h; p.sw = (int)stride_w; p.dh = (int)dilation_h; p.dw = (int)dilation_w;
+    p.i_n = i_strides[0]; p.i_h = i_strides[1]; p.i_w = i_strides[2]; p.i_c = i_strides[3];
+    p.k_kh = k_strides[0]; p.k_kw = k_strides[1]; p.k_c = k_strides[2]; p.k_f = k_strides[3];
+    p.o_n = o_strides[0]; p.o_h = o_strides[1]; p.o_w = o_strides[2]; p.o_f = o_strides[3];
+    p.in_bf16 = in_dtype == SG_BF16; p.accumulate = mode == SG_ACCUMULATE; p.spatial_rank = 2;
+    return run(p, I, Kf, O, static_cast<cudaStream_t>(stream));
+}
+
+sg_status sg_check(sg_stream_t stream) {
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(s) != cudaSuccess) return SG_ERR_CUDA;
+    return tensor_read_status(s);
+}
+
+const char *sg_status_string(sg_status status) {
+    switch (status) {
+        case SG_OK: return "ok";
+        case SG_ERR_INVALID_ARG: return "invalid argument";
+        case SG_ERR_UNSUPPORTED: return "unsupported dtype, mode, size or layout";
+        case SG_ERR_ALIGNMENT: return "pointer not aligned to its element size";
+        case SG_ERR_CUDA: return "CUDA runtime or driver call failed";
+        case SG_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+        case SG_ERR_INTERNAL: return "internal error";
+    }
+    return "unknown status";
+}
+
+int sg_version(void) { return 100; }
+
+int sg_last_kernel(void) { return t_last_kernel; }
+
+int64_t sg_launch_count(void) { return g_launches.load(); }
+
+sg_status sg_set_kernel_override(int kernel_family) {
+    if (kernel_family != SG_KERNEL_AUTO && kernel_family != SG_KERNEL_FFMA && kernel_family != SG_KERNEL_TENSOR)
+        return SG_ERR_INVALID_ARG;
+    g_override.store(kernel_family);
+    return SG_OK;
+}
+
+void sg_shutdown(void) { tensor_shutdown(); }
+
+}  // extern "C"

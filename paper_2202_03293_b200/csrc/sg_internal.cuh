@@ -1,0 +1,49 @@
+// Shared declarations of the CUDA side of the library (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "sg.h"
+
+namespace sg {
+
+// Every op is run as one implicit GEMM  O[m, f] (+)= sum_k  In(m, k) * Flt(k, f)  with
+//   m = (n, h, w)  flattened over the output's batch and spatial iterators,
+//   k = (kh, kw, c) flattened over the reduction iterators,
+// and operand addresses that separate into a row part and a reduction part:
+//   In (m,k) at  n*i_n + (h*sh + kh*dh)*i_h + (w*sw + kw*dw)*i_w + c*i_c
+//   Flt(k,f) at  kh*k_kh + kw*k_kw + c*k_c + f*k_f
+//   O  (m,f) at  n*o_n + h*o_h + w*o_w + f*o_f
+// A matmul is the case Ho = KH = KW = 1, batch 1, Wo = M, C = K (a 1x1 filter).
+struct Problem {
+    int M, N, K;             // GEMM extents: M = batch*Ho*Wo, N = F, K = KH*KW*C
+    int batch, Ho, Wo;       // decomposition of m
+    int KH, KW, C;           // decomposition of k
+    int Hin, Win;            // input spatial extents (bounds of the im2col box)
+    int sh, sw, dh, dw;      // strides and dilations of the window
+    int64_t i_n, i_h, i_w, i_c;
+    int64_t k_kh, k_kw, k_c, k_f;
+    int64_t o_n, o_h, o_w, o_f;
+    int in_bf16;             // 1: inputs are bf16, 0: f32
+    int accumulate;          // 1: O = O_in + result
+    int spatial_rank;        // 0 matmul, 1 conv1d, 2 conv2d
+};
+
+// Launchers (each returns the cudaError_t of its launch).
+cudaError_t launch_ffma(const Problem &p, const void *In, const void *Flt, float *O,
+                        cudaStream_t stream);
+cudaError_t launch_zero_fill(const Problem &p, float *O, cudaStream_t stream);
+
+// Tensor-core path: returns SG_ERR_UNSUPPORTED (and launches nothing) when the layout
+// does not satisfy the TMA rules.
+sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float *O,
+                        cudaStream_t stream);
+void tensor_shutdown();
+// Reads and clears the current device's status word (written by kernels whose bounded
+// waits expire); the caller has already synchronised the stream.
+sg_status tensor_read_status(cudaStream_t stream);
+
+void count_launch(int n = 1);
+
+}  // namespace sg

@@ -1,0 +1,594 @@
+// Tensor-core path for sm_100a: TMA -> swizzled shared memory -> tcgen05.mma -> TMEM -> TMA store.
+//
+// One persistent CTA per SM walks a static list of 128 x BN output tiles.  Inside a CTA
+// the work is split by warp role:
+//
+//   warp 0  producer : per k-block waits for a free stage, then issues the TMA loads of the
+//                      input tile (tiled mode for matmul, im2col mode for the convolutions:
+//                      the TMA unit itself gathers the sliding window, Section 3.2's
+//                      "padding/packing" done in hardware) and of the filter tile.
+//   warp 1  MMA      : one thread waits for a full stage and issues tcgen05.mma into one of
+//                      two TMEM accumulator buffers; tcgen05.commit releases the stage and,
+//                      after the last k-block, publishes the accumulator.
+//   warps 2-5 epilogue: each owns one 32-lane quarter of TMEM; tcgen05.ld -> registers ->
+//                      swizzled staging buffer -> TMA store (or TMA reduce-add when the op
+//                      accumulates into its output), overlapping the next tile's main loop.
+//
+// Shared-memory operand layouts (both 128-byte swizzled, written by TMA, read by the MMA
+// unit through matrix descriptors):
+//   input tile   K-major : 128 rows (output pixels) x 64 bf16 (128 B per row)
+//   filter tile  N-major : BN/64 sub-tiles, each 64 k-rows x 64 bf16 (128 B per row); the
+//                          filter is stored [k][f] with f contiguous, so it is consumed as
+//                          an MN-major operand instead of being transposed.
+//
+// Every wait in this file is bounded: a wait that expires sets an abort flag in shared
+// memory and a bit in the device status word, every role then leaves its loop, the CTA
+// drains its copies, frees its TMEM and returns.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "sg_internal.cuh"
+
+namespace sg {
+namespace {
+
+constexpr int BM = 128;           // rows of an output tile = lanes of TMEM = M of one MMA
+constexpr int BK = 64;            // bf16 elements per k-block = one 128-byte swizzle row
+constexpr int UMMA_K = 16;        // k extent of one tcgen05.mma for 16-bit inputs
+constexpr int NUM_THREADS = 192;  // 6 warps: producer, MMA, 4 epilogue
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int STAGING_BYTES = 4 * 2 * 4096;   // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
+constexpr long long WAIT_BUDGET_CYCLES = 2000000000LL;   // ~1 s: far beyond any legitimate wait
+
+__device__ unsigned int g_status_word = 0;
+
+struct TcParams {
+    int M, N;
+    int num_m_tiles, num_n_tiles;
+    int num_kb;          // k-blocks per tile = taps * kb_per_tap
+    int kb_per_tap;      // ceil(C / 64)
+    int KW;              // taps are ordered (kh, kw)
+    int a_mode;          // 0: tiled 2-D (matmul), 1: im2col 3-D (conv1d), 2: im2col 4-D (conv2d)
+    int Ho, Wo, sh, sw, dh, dw;
+    int accumulate;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the budget expired or another role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_BUDGET_CYCLES) {
+                *abort_flag = 1;
+                atomicOr(&g_status_word, 1u);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z, int w) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+// im2col mode: coordinates name the first base pixel (c, w, [h,] n); the 16-bit offsets are
+// added to every pixel's spatial coordinates (the filter tap's kw*dw, kh*dh).
+__device__ __forceinline__ void tma_load_im2col_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                                   int c, int w, int n, unsigned short off_w) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2], {%6};"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(n), "h"(off_w) : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                                   int c, int w, int h, int n, unsigned short off_w, unsigned short off_h) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, uint32_t src, int x, int y) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem], 128 x N x 16, bf16 inputs, f32 accumulate.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives on the mbarrier once every tcgen05.mma issued so far by this thread has finished.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// This warp's 32 lanes x 32 consecutive f32 columns of TMEM -> 32 registers per thread.
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (sm_100 format): start address, leading and stride byte
+// offsets (all >> 4), descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;   // version
+    d |= (uint64_t)2 << 61;   // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor: f32 accumulator, bf16 A and B, A K-major, B N-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int n) {
+    return (1u << 4)                       // D format: f32
+         | (1u << 7)                       // A format: bf16
+         | (1u << 10)                      // B format: bf16
+         | (0u << 15)                      // A major: K
+         | (1u << 16)                      // B major: MN (filter stored [k][f], f contiguous)
+         | ((uint32_t)(n >> 3) << 17)      // N / 8
+         | ((uint32_t)(BM >> 4) << 24);    // M / 16
+}
+
+template <int BN>
+struct Cfg {
+    static constexpr int B_STAGE_BYTES = BK * BN * 2;
+    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+    static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
+    static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // two accumulator buffers
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+// Static tile order: groups of 8 tile-rows, row index fastest inside a group, so that the
+// CTAs running at the same time share filter columns and a bounded set of input rows in L2.
+__device__ __forceinline__ void tile_coords(int t, int num_m_tiles, int num_n_tiles, int &mt, int &nt) {
+    constexpr int GM = 8;
+    int per_group = GM * num_n_tiles;
+    int g = t / per_group, r = t - g * per_group;
+    int rows = num_m_tiles - g * GM;
+    if (rows > GM) rows = GM;
+    nt = r / rows;
+    mt = g * GM + (r - nt * rows);
+}
+
+template <int BN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_flt,
+               const __grid_constant__ CUtensorMap map_out, const TcParams p) {
+    using C = Cfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+    const uint32_t stages_addr = smem_base;
+    const uint32_t staging_addr = smem_base + C::STAGES * C::STAGE_BYTES;
+    uint8_t *staging_gen = smem_gen + C::STAGES * C::STAGE_BYTES;
+    const uint32_t bars_addr = staging_addr + STAGING_BYTES;
+    uint8_t *bars_gen = staging_gen + STAGING_BYTES;
+    // barrier block: full[STAGES] | empty[STAGES] | acc_full[2] | acc_empty[2] | tmem_ptr | abort
+    auto full_bar = [&](int s) { return bars_addr + 8u * s; };
+    auto empty_bar = [&](int s) { return bars_addr + 8u * (C::STAGES + s); };
+    auto acc_full_bar = [&](int b) { return bars_addr + 8u * (2 * C::STAGES + b); };
+    auto acc_empty_bar = [&](int b) { return bars_addr + 8u * (2 * C::STAGES + 2 + b); };
+    volatile uint32_t *tmem_ptr_slot = reinterpret_cast<volatile uint32_t *>(bars_gen + 8 * (2 * C::STAGES + 4));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_gen + 8 * (2 * C::STAGES + 4) + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // TMEM allocation is a warp-wide operation
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(const_cast<uint32_t *>(tmem_ptr_slot))), "r"((uint32_t)C::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_ptr_slot;
+
+    const int num_tiles = p.num_m_tiles * p.num_n_tiles;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            int it = 0;   // k-block counter across all of this CTA's tiles
+            bool ok = true;
+            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+                int mt, nt;
+                tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+                const int m0 = mt * BM, n0 = nt * BN;
+                int pix_n = 0, pix_h = 0, pix_w = 0;   // first output pixel of the tile
+                if (p.a_mode != 0) {
+                    int hw = p.Ho * p.Wo;
+                    pix_n = m0 / hw;
+                    int r = m0 - pix_n * hw;
+                    pix_h = r / p.Wo;
+                    pix_w = r - pix_h * p.Wo;
+                }
+                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                    const int s = it % C::STAGES;
+                    const uint32_t ph = (it / C::STAGES) & 1;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t a_dst = stages_addr + s * C::STAGE_BYTES;
+                    const uint32_t b_dst = a_dst + A_STAGE_BYTES;
+                    mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
+                    const int tap = kb / p.kb_per_tap;
+                    const int c0 = (kb - tap * p.kb_per_tap) * BK;
+                    const int kh = tap / p.KW, kw = tap - kh * p.KW;
+                    if (p.a_mode == 0) {
+                        tma_load_2d(a_dst, &map_in, full_bar(s), c0, m0);
+                    } else if (p.a_mode == 1) {
+                        tma_load_im2col_3d(a_dst, &map_in, full_bar(s), c0, pix_w * p.sw, pix_n,
+                                           (unsigned short)(kw * p.dw));
+                    } else {
+                        tma_load_im2col_4d(a_dst, &map_in, full_bar(s), c0, pix_w * p.sw, pix_h * p.sh, pix_n,
+                                           (unsigned short)(kw * p.dw), (unsigned short)(kh * p.dh));
+                    }
+#pragma unroll
+                    for (int j = 0; j < BN / 64; ++j)
+                        tma_load_4d(b_dst + j * (BK * 128), &map_flt, full_bar(s), n0 + j * 64, c0, kw, kh);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(BN);
+            int it = 0, tl = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tl) {
+                const int buf = tl & 1;
+                if (!mbar_wait(acc_empty_bar(buf), ((tl >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                    const int s = it % C::STAGES;
+                    const uint32_t ph = (it / C::STAGES) & 1;
+                    if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = stages_addr + s * C::STAGE_BYTES;
+                    const uint32_t b_addr = a_addr + A_STAGE_BYTES;
+                    // input tile, K-major: 8-row groups are 1024 B apart; a k-step of 16 bf16 is 32 B
+                    // inside the swizzled 128-byte row.
+                    const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024);
+                    // filter tile, N-major: 64-column sub-tiles are BK*128 B apart (leading offset),
+                    // 8-row k groups 1024 B apart (stride offset); a k-step of 16 rows is 2048 B.
+                    const uint64_t b_desc = make_smem_desc(b_addr, BK * 128, 1024);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        umma_bf16(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc,
+                                  (kb > 0 || k > 0) ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar(s));   // the stage is free once these MMAs have read it
+                }
+                if (ok) umma_commit(acc_full_bar(buf));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int q = warp & 3;   // TMEM lane quarter this warp may access
+        const uint32_t stg_addr = staging_addr + (warp - 2) * 8192;
+        uint8_t *stg_gen = staging_gen + (warp - 2) * 8192;
+        int tl = 0, chunk_count = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tl) {
+            int mt, nt;
+            tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+            const int m0 = mt * BM, n0 = nt * BN;
+            const int buf = tl & 1;
+            if (!mbar_wait(acc_full_bar(buf), (tl >> 1) & 1, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll 1
+            for (int j = 0; j < BN / 32; ++j, ++chunk_count) {
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + j * 32), r);
+                tmem_ld_wait();
+                const int sb = chunk_count & 1;
+                // the bulk store issued two chunks ago must have finished reading this buffer
+                if (lane == 0) bulk_wait_read<1>();
+                __syncwarp();
+                uint8_t *row = stg_gen + sb * 4096 + lane * 128;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint4 v = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+                    *reinterpret_cast<uint4 *>(row + ((c ^ (lane & 7)) << 4)) = v;
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    const int x = n0 + j * 32, y = m0 + q * 32;
+                    if (x < p.N && y < p.M) {
+                        if (p.accumulate) tma_reduce_add_2d(&map_out, stg_addr + sb * 4096, x, y);
+                        else tma_store_2d(&map_out, stg_addr + sb * 4096, x, y);
+                    }
+                    bulk_commit();
+                }
+            }
+            // every tcgen05.ld of this buffer has completed: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+        }
+        if (lane == 0) bulk_wait_all();
+    }
+
+    // ---------------------------------------------------------------- teardown
+    __syncthreads();
+    if (*abort_flag) {
+        // give any TMA load still in flight time to land before the shared memory is released
+        for (int i = 0; i < 200; ++i) __nanosleep(5000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const int *, const int *, cuuint32_t, cuuint32_t,
+                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct Driver {
+    EncodeTiledFn tiled = nullptr;
+    EncodeIm2colFn im2col = nullptr;
+    int num_sms = 0;
+    int device = -1;
+    bool attr_set[3] = {false, false, false};
+    bool ok = false;
+};
+std::mutex g_mu;
+Driver g_drv;
+int g_bn_override = -1;   // -1: not read yet; 0: automatic
+
+bool init_driver() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (g_drv.ok && g_drv.device == dev) return true;
+    g_drv = Driver{};   // first use, or the caller switched devices: per-device state starts over
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess || !fn) return false;
+    g_drv.tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn, cudaEnableDefault, &qr) != cudaSuccess || !fn) return false;
+    g_drv.im2col = reinterpret_cast<EncodeIm2colFn>(fn);
+    if (cudaDeviceGetAttribute(&g_drv.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+    int major = 0;
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (major != 10) return false;
+    g_drv.device = dev;
+    g_drv.ok = true;
+    return true;
+}
+
+inline bool mult(int64_t v, int64_t q) { return v % q == 0; }
+
+template <int BN>
+sg_status launch_bn(const CUtensorMap &mi, const CUtensorMap &mf, const CUtensorMap &mo, const TcParams &tp,
+                    int slot, cudaStream_t stream) {
+    using C = Cfg<BN>;
+    if (!g_drv.attr_set[slot]) {
+        if (cudaFuncSetAttribute(tc_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+            return SG_ERR_CUDA;
+        g_drv.attr_set[slot] = true;
+    }
+    int tiles = tp.num_m_tiles * tp.num_n_tiles;
+    int grid = tiles < g_drv.num_sms ? tiles : g_drv.num_sms;
+    tc_gemm_kernel<BN><<<grid, NUM_THREADS, C::SMEM_BYTES, stream>>>(mi, mf, mo, tp);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? SG_OK : SG_ERR_CUDA;
+}
+
+}  // namespace
+
+sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float *O, cudaStream_t stream) {
+    // ---- layout rules of the TMA descriptors (bytes): unit inner stride, 16-byte aligned
+    //      bases and pitches; output rows uniformly strided so that O is one 2-D matrix ----
+    if (!p.in_bf16) return SG_ERR_UNSUPPORTED;
+    const int64_t es = 2;
+    if (p.i_c != 1 || p.k_f != 1 || p.o_f != 1) return SG_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(In) % 16 || reinterpret_cast<uintptr_t>(Flt) % 16 ||
+        reinterpret_cast<uintptr_t>(O) % 16) return SG_ERR_UNSUPPORTED;
+    if (!mult(p.i_w * es, 16) || !mult(p.k_c * es, 16) || !mult(p.o_w * 4, 16)) return SG_ERR_UNSUPPORTED;
+    if (p.Ho > 1 && p.o_h != (int64_t)p.Wo * p.o_w) return SG_ERR_UNSUPPORTED;
+    if (p.batch > 1 && p.o_n != (int64_t)p.Ho * p.Wo * p.o_w) return SG_ERR_UNSUPPORTED;
+    if (p.KW > 1 && !mult(p.k_kw * es, 16)) return SG_ERR_UNSUPPORTED;
+    if (p.KH > 1 && !mult(p.k_kh * es, 16)) return SG_ERR_UNSUPPORTED;
+    if (p.i_w < p.C || p.k_c < p.N || p.o_w < p.N) return SG_ERR_UNSUPPORTED;   // overlapping rows
+    const int64_t pitch_limit = (int64_t)1 << 40;
+    if (p.i_w * es >= pitch_limit || p.k_c * es >= pitch_limit || p.o_w * 4 >= pitch_limit) return SG_ERR_UNSUPPORTED;
+
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!init_driver()) return SG_ERR_CUDA;
+    if (g_bn_override < 0) {
+        const char *e = getenv("SG_TC_BN");
+        g_bn_override = e ? atoi(e) : 0;
+    }
+
+    alignas(64) CUtensorMap map_in, map_flt, map_out;
+    TcParams tp{};
+    tp.M = p.M; tp.N = p.N;
+    tp.KW = p.KW;
+    tp.kb_per_tap = (p.C + BK - 1) / BK;
+    tp.num_kb = p.KH * p.KW * tp.kb_per_tap;
+    tp.Ho = p.Ho; tp.Wo = p.Wo; tp.sh = p.sh; tp.sw = p.sw; tp.dh = p.dh; tp.dw = p.dw;
+    tp.accumulate = p.accumulate;
+
+    const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+    CUresult r;
+    // ---- input operand ----
+    if (p.spatial_rank == 0) {
+        tp.a_mode = 0;
+        cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)p.M};
+        cuuint64_t strides[1] = {(cuuint64_t)(p.i_w * es)};
+        cuuint32_t box[2] = {BK, BM};
+        r = g_drv.tiled(&map_in, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(In), dims, strides, box, ones,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
+    } else {
+        // im2col descriptors: the bounding box of base pixels is [0, used - (K-1)*d) per spatial
+        // dimension, walked with the conv stride, which yields exactly W_out (H_out) base
+        // pixels per row (column); the filter tap is added per load as an offset.
+        const int64_t used_w = (int64_t)(p.Wo - 1) * p.sw + (int64_t)(p.KW - 1) * p.dw + 1;
+        const int64_t used_h = (int64_t)(p.Ho - 1) * p.sh + (int64_t)(p.KH - 1) * p.dh + 1;
+        const int64_t span_w = (int64_t)(p.KW - 1) * p.dw, span_h = (int64_t)(p.KH - 1) * p.dh;
+        if (p.sw > 8 || p.sh > 8) return SG_ERR_UNSUPPORTED;
+        // Tensors below 128 KiB are kept off the im2col path.
+        int64_t in_bytes = (int64_t)p.batch * (p.spatial_rank == 2 ? used_h : 1) * used_w * p.C * es;
+        if (in_bytes < 131072) return SG_ERR_UNSUPPORTED;
+        if (p.spatial_rank == 1) {
+            if (span_w > 32767) return SG_ERR_UNSUPPORTED;
+            if (p.batch > 1 && !mult(p.i_n * es, 16)) return SG_ERR_UNSUPPORTED;
+            tp.a_mode = 1;
+            cuuint64_t dims[3] = {(cuuint64_t)p.C, (cuuint64_t)used_w, (cuuint64_t)p.batch};
+            cuuint64_t strides[2] = {(cuuint64_t)(p.i_w * es), (cuuint64_t)((p.batch > 1 ? p.i_n : used_w * p.i_w) * es)};
+            int lower[1] = {0}, upper[1] = {(int)-span_w};
+            cuuint32_t trav[3] = {1, (cuuint32_t)p.sw, 1};
+            r = g_drv.im2col(&map_in, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(In), dims, strides, lower,
+                             upper, BK, BM, trav, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        } else {
+            if (span_w > 127 || span_h > 127) return SG_ERR_UNSUPPORTED;
+            if (!mult(p.i_h * es, 16) || (p.batch > 1 && !mult(p.i_n * es, 16))) return SG_ERR_UNSUPPORTED;
+            tp.a_mode = 2;
+            cuuint64_t dims[4] = {(cuuint64_t)p.C, (cuuint64_t)used_w, (cuuint64_t)used_h, (cuuint64_t)p.batch};
+            cuuint64_t strides[3] = {(cuuint64_t)(p.i_w * es), (cuuint64_t)(p.i_h * es),
+                                     (cuuint64_t)((p.batch > 1 ? p.i_n : used_h * p.i_h) * es)};
+            int lower[2] = {0, 0}, upper[2] = {(int)-span_w, (int)-span_h};
+            cuuint32_t trav[4] = {1, (cuuint32_t)p.sw, (cuuint32_t)p.sh, 1};
+            r = g_drv.im2col(&map_in, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(In), dims, strides, lower,
+                             upper, BK, BM, trav, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        }
+        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
+    }
+    // ---- filter operand: 4-D {f, c, kw, kh}, one 64 x 64 box per load ----
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)p.N, (cuuint64_t)p.C, (cuuint64_t)p.KW, (cuuint64_t)p.KH};
+        int64_t s_kw = p.KW > 1 ? p.k_kw : (int64_t)p.C * p.k_c;
+        int64_t s_kh = p.KH > 1 ? p.k_kh : (int64_t)p.KW * s_kw;
+        cuuint64_t strides[3] = {(cuuint64_t)(p.k_c * es), (cuuint64_t)(s_kw * es), (cuuint64_t)(s_kh * es)};
+        cuuint32_t box[4] = {64, BK, 1, 1};
+        r = g_drv.tiled(&map_flt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(Flt), dims, strides, box, ones,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
+    }
+    // ---- output: 2-D {f, m} f32, stored in 32 x 32 boxes ----
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)p.N, (cuuint64_t)p.M};
+        cuuint64_t strides[1] = {(cuuint64_t)(p.o_w * 4)};
+        cuuint32_t box[2] = {32, 32};
+        r = g_drv.tiled(&map_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, O, dims, strides, box, ones,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
+    }
+
+    // ---- tile width: fewest (waves x per-tile cost); narrower tiles cost more shared-memory
+    //      traffic per flop, wider ones quantise worse ----
+    int bn = g_bn_override;
+    if (bn != 64 && bn != 128 && bn != 256) {
+        double best = 1e300;
+        const int cand[3] = {64, 128, 256};
+        const double step_cost[3] = {48.0, 64.0, 128.0};
+        for (int i = 0; i < 3; ++i) {
+            if (cand[i] > 64 && cand[i] / 2 >= p.N) continue;   // at most half of the tile would be used
+            int64_t tiles = (int64_t)((p.M + BM - 1) / BM) * ((p.N + cand[i] - 1) / cand[i]);
+            int64_t waves = (tiles + g_drv.num_sms - 1) / g_drv.num_sms;
+            double cost = (double)waves * step_cost[i];
+            if (cost < best) { best = cost; bn = cand[i]; }
+        }
+    }
+    tp.num_m_tiles = (p.M + BM - 1) / BM;
+    tp.num_n_tiles = (p.N + bn - 1) / bn;
+    if (bn == 64) return launch_bn<64>(map_in, map_flt, map_out, tp, 0, stream);
+    if (bn == 128) return launch_bn<128>(map_in, map_flt, map_out, tp, 1, stream);
+    return launch_bn<256>(map_in, map_flt, map_out, tp, 2, stream);
+}
+
+sg_status tensor_read_status(cudaStream_t stream) {
+    unsigned int word = 0, zero = 0;
+    if (cudaMemcpyFromSymbolAsync(&word, g_status_word, sizeof(word), 0, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+        return SG_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return SG_ERR_CUDA;
+    if (word != 0) {
+        if (cudaMemcpyToSymbolAsync(g_status_word, &zero, sizeof(zero), 0, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+            return SG_ERR_CUDA;
+        cudaStreamSynchronize(stream);
+        return SG_ERR_DEVICE_TIMEOUT;
+    }
+    return SG_OK;
+}
+
+void tensor_shutdown() {
+    std::lock_guard<std::mutex> lock(g_mu);
+    g_drv = Driver{};
+}
+
+}  // namespace sg

@@ -1,0 +1,351 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle, element by element,
+within |err| <= 1e-4 * sum_k |a*b|, on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import assert_within_bound, operand
+from oracle import ref
+from paper_2202_03293_b200 import binding as sg
+from paper_2202_03293_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+SEED = inputs.BASE_SEED
+FFMA, TENSOR = sg.SG_KERNEL_FFMA, sg.SG_KERNEL_TENSOR
+
+
+@pytest.fixture(autouse=True)
+def _reset_override():
+    sg.sg_set_kernel_override(sg.SG_KERNEL_AUTO)
+    yield
+    sg.sg_set_kernel_override(sg.SG_KERNEL_AUTO)
+    sg.sg_check()      # no kernel of the test gave up on a bounded wait
+
+
+def run_matmul(M, N, K, dtype, family=None, accumulate=False, dist="uniform", seed=SEED):
+    A, a = operand((M, K), seed, 1, dist, dtype)
+    B, b = operand((K, N), seed, 2, dist, dtype)
+    if accumulate:
+        C, c0 = operand((M, N), seed, 3, "uniform", "f32")
+        C = C.clone()
+    else:
+        C, c0 = torch.full((M, N), float("nan"), device="cuda"), None
+    if family is not None:
+        sg.sg_set_kernel_override(family)
+    sg.sg_matmul(A, B, C, sg.SG_ACCUMULATE if accumulate else sg.SG_OVERWRITE)
+    torch.cuda.synchronize()
+    want, S = ref.matmul(a, b, C_in=c0)
+    if accumulate:
+        S = S + np.abs(c0)          # the added term |C_in * 1| belongs to the sum of magnitudes
+    return C, want, S
+
+
+# ------------------------------------------------------------------ config 1: matmul 128^3 f32
+
+@pytest.mark.parametrize("accumulate", [False, True])
+def test_c1_matmul_128_f32(accumulate):
+    C, want, S = run_matmul(128, 128, 128, "f32", accumulate=accumulate, seed=SEED + 0)
+    assert sg.sg_last_kernel() == FFMA
+    assert_within_bound(C, want, S, "matmul 128^3 f32")
+
+
+# ------------------------------------------------------------------ matmul, both kernel families
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (256, 256, 256), (300, 200, 136), (129, 72, 8), (1, 8, 8),
+                                   (515, 264, 1000), (128, 64, 4096), (384, 520, 72)])
+@pytest.mark.parametrize("family", [FFMA, TENSOR])
+def test_matmul_bf16_shapes(M, N, K, family):
+    C, want, S = run_matmul(M, N, K, "bf16", family=family, seed=SEED + 1)
+    assert sg.sg_last_kernel() == family
+    assert_within_bound(C, want, S, f"matmul bf16 {M}x{N}x{K} family {family}")
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 64, 64), (130, 70, 50), (257, 129, 33), (1, 1, 1), (5, 3, 2), (512, 256, 384)])
+def test_matmul_f32_shapes(M, N, K):
+    C, want, S = run_matmul(M, N, K, "f32", seed=SEED + 1)
+    assert_within_bound(C, want, S, f"matmul f32 {M}x{N}x{K}")
+
+
+@pytest.mark.parametrize("bn", ["64", "128", "256"])
+def test_matmul_bf16_every_tile_width(bn, monkeypatch):
+    # the tile width is normally chosen from the shape; exercise each instantiation on a
+    # shape with ragged edges in m, n and k.  SG_TC_BN is read once per process, so these
+    # run in a child interpreter.
+    import subprocess, sys, os
+    code = (
+        "import sys; sys.path.insert(0, 'tests'); sys.path.insert(0, '.');"
+        "import test_gpu_parity as t;"
+        "from helpers import assert_within_bound;"
+        "C, want, S = t.run_matmul(400, 520, 200, 'bf16', family=t.TENSOR, seed=t.SEED + 7);"
+        "assert_within_bound(C, want, S, 'bn');"
+        "C, want, S = t.run_matmul(400, 520, 200, 'bf16', family=t.TENSOR, accumulate=True, seed=t.SEED + 7);"
+        "assert_within_bound(C, want, S, 'bn acc'); t.sg.sg_check(); print('child-ok')"
+    )
+    env = dict(os.environ, SG_TC_BN=bn)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0 and "child-ok" in out.stdout, out.stdout + out.stderr
+
+
+@pytest.mark.parametrize("family", [FFMA, TENSOR])
+def test_matmul_integer_inputs_are_bit_exact(family):
+    # integers in [-2,2]: every product and partial sum is exact in f32, so every summation
+    # order gives the same bits as the f64 oracle.
+    C, want, S = run_matmul(256, 192, 320, "bf16", family=family, dist="ints", seed=SEED + 2)
+    assert np.array_equal(C.cpu().numpy().astype(np.float64), want)
+
+
+@pytest.mark.parametrize("family", [FFMA, TENSOR])
+def test_matmul_accumulate_into_nonzero_output(family):
+    C, want, S = run_matmul(260, 136, 200, "bf16", family=family, accumulate=True, seed=SEED + 3)
+    assert sg.sg_last_kernel() == family
+    assert_within_bound(C, want, S, "accumulate")
+
+
+def test_matmul_paper_example_ones():
+    # Appendix A.4: ones(M,K) . ones(K,N) accumulated into zeros(M,N) gives K everywhere.
+    for dt, tdt in (("f32", torch.float32), ("bf16", torch.bfloat16)):
+        M, N, K = 200, 136, 328
+        A = torch.ones(M, K, device="cuda", dtype=tdt)
+        B = torch.ones(K, N, device="cuda", dtype=tdt)
+        C = torch.zeros(M, N, device="cuda")
+        sg.sg_matmul(A, B, C, sg.SG_ACCUMULATE)
+        torch.cuda.synchronize()
+        assert torch.all(C == K)
+
+
+def test_matmul_transposed_operands_through_strides():
+    # Section 4.6.1: A^T B and A B^T are the same op under different strides.
+    M, N, K = 150, 90, 70
+    At, a_t = operand((K, M), SEED, 4, "uniform", "f32")      # stored A[k,m]
+    Bt, b_t = operand((N, K), SEED, 5, "uniform", "f32")      # stored B[n,k]
+    B, b = operand((K, N), SEED, 6, "uniform", "f32")
+    A, a = operand((M, K), SEED, 7, "uniform", "f32")
+    C = torch.empty(M, N, device="cuda")
+    sg.sg_matmul(At.t(), B, C)
+    want, S = ref.matmul(np.ascontiguousarray(a_t.T), b)
+    assert_within_bound(C, want, S, "A^T B")
+    sg.sg_matmul(A, Bt.t(), C)
+    want, S = ref.matmul(a, np.ascontiguousarray(b_t.T))
+    assert_within_bound(C, want, S, "A B^T")
+    # column-major output view
+    Ct = torch.empty(N, M, device="cuda")
+    sg.sg_matmul(A, B, Ct.t())
+    want, S = ref.matmul(a, b)
+    assert_within_bound(Ct.t(), want, S, "column-major C")
+
+
+def test_matmul_padded_rows_and_offsets():
+    # non-dense pitches and an element offset that breaks 16-byte alignment: generic path
+    M, N, K = 100, 60, 40
+    Abig, a = operand((M, K + 3), SEED, 8, "uniform", "bf16")
+    Bbig, b = operand((K, N + 5), SEED, 9, "uniform", "bf16")
+    Cbig = torch.zeros(M, N + 7, device="cuda")
+    A, B, C = Abig[:, 1:K + 1], Bbig[:, 3:N + 3], Cbig[:, 2:N + 2]
+    sg.sg_matmul(A, B, C)
+    assert sg.sg_last_kernel() == FFMA
+    want, S = ref.matmul(a[:, 1:K + 1], b[:, 3:N + 3])
+    assert_within_bound(C, want, S, "padded")
+    assert torch.all(Cbig[:, :2] == 0) and torch.all(Cbig[:, N + 2:] == 0)     # nothing outside the view written
+    # aligned pitches larger than the row: still tensor-core eligible
+    M, N, K = 100, 56, 40
+    Abig, a = operand((M, K + 24), SEED, 10, "uniform", "bf16")
+    Cbig = torch.zeros(M, N + 4, device="cuda")
+    Bd, b = operand((K, N), SEED, 11, "uniform", "bf16")
+    sg.sg_matmul(Abig[:, 8:K + 8], Bd, Cbig[:, 4:])
+    assert sg.sg_last_kernel() == TENSOR
+    want, S = ref.matmul(a[:, 8:K + 8], b)
+    assert_within_bound(Cbig[:, 4:], want, S, "pitched")
+    assert torch.all(Cbig[:, :4] == 0)
+
+
+def test_degenerate_sizes():
+    A = torch.ones(8, 0, device="cuda", dtype=torch.bfloat16)
+    B = torch.ones(0, 8, device="cuda", dtype=torch.bfloat16)
+    C = torch.full((8, 8), 5.0, device="cuda")
+    sg.sg_matmul(A, B, C, sg.SG_ACCUMULATE)       # empty reduction adds nothing
+    torch.cuda.synchronize()
+    assert torch.all(C == 5.0)
+    sg.sg_matmul(A, B, C, sg.SG_OVERWRITE)        # empty reduction: the sum is zero
+    torch.cuda.synchronize()
+    assert torch.all(C == 0.0)
+    Cpad = torch.full((8, 12), 5.0, device="cuda")
+    sg.sg_matmul(A, B, Cpad[:, 2:10], sg.SG_OVERWRITE)
+    torch.cuda.synchronize()
+    assert torch.all(Cpad[:, 2:10] == 0.0) and torch.all(Cpad[:, :2] == 5.0) and torch.all(Cpad[:, 10:] == 5.0)
+    E = torch.empty(0, 8, device="cuda")
+    sg.sg_matmul(torch.empty(0, 4, device="cuda"), torch.empty(4, 8, device="cuda"), E)
+
+
+# ------------------------------------------------------------------ convolutions
+
+def run_conv1d(N, Wo, C, KW, F, sw, dw, dtype, family=None, accumulate=False, dist="uniform", seed=SEED, extra_w=0):
+    W_in = (Wo - 1) * sw + (KW - 1) * dw + 1 + extra_w
+    I, i = operand((N, W_in, C), seed, 1, dist, dtype)
+    Kf, k = operand((KW, C, F), seed, 2, dist, dtype)
+    if accumulate:
+        O, o0 = operand((N, Wo, F), seed, 3, "uniform", "f32")
+        O = O.clone()
+    else:
+        O, o0 = torch.full((N, Wo, F), float("nan"), device="cuda"), None
+    if family is not None:
+        sg.sg_set_kernel_override(family)
+    sg.sg_conv1d_nwc_wcf(I, Kf, O, sw, dw, sg.SG_ACCUMULATE if accumulate else sg.SG_OVERWRITE)
+    torch.cuda.synchronize()
+    want, S = ref.conv1d_nwc_wcf(i, k, stride=sw, dilation=dw, O_in=o0, W_out=Wo)
+    if accumulate:
+        S = S + np.abs(o0)
+    return O, want, S
+
+
+def run_conv2d(N, Ho, Wo, C, KH, KW, F, st, dl, dtype, family=None, accumulate=False, dist="normal", seed=SEED,
+               extra=(0, 0)):
+    H_in = (Ho - 1) * st[0] + (KH - 1) * dl[0] + 1 + extra[0]
+    W_in = (Wo - 1) * st[1] + (KW - 1) * dl[1] + 1 + extra[1]
+    I, i = operand((N, H_in, W_in, C), seed, 1, dist, dtype)
+    Kf, k = operand((KH, KW, C, F), seed, 2, dist, dtype)
+    if accumulate:
+        O, o0 = operand((N, Ho, Wo, F), seed, 3, "uniform", "f32")
+        O = O.clone()
+    else:
+        O, o0 = torch.full((N, Ho, Wo, F), float("nan"), device="cuda"), None
+    if family is not None:
+        sg.sg_set_kernel_override(family)
+    sg.sg_conv2d_nhwc_hwcf(I, Kf, O, st, dl, sg.SG_ACCUMULATE if accumulate else sg.SG_OVERWRITE)
+    torch.cuda.synchronize()
+    want, S = ref.conv2d_nhwc_hwcf(i, k, stride=st, dilation=dl, O_in=o0, out_hw=(Ho, Wo))
+    if accumulate:
+        S = S + np.abs(o0)
+    return O, want, S
+
+
+def test_c3_conv1d_f32_full():
+    # config 3: N=32, W=1026, C=64, KW=3, F=128, stride 1, f32, uniform[-1,1)
+    O, want, S = run_conv1d(32, 1024, 64, 3, 128, 1, 1, "f32", seed=SEED + 2)
+    assert_within_bound(O, want, S, "conv1d config 3")
+
+
+def test_c4_conv2d_bf16_full():
+    # config 4: N=16, H=W=58, C=64, 3x3, F=128, stride 1, bf16 in / f32 out, N(0,1)
+    O, want, S = run_conv2d(16, 56, 56, 64, 3, 3, 128, (1, 1), (1, 1), "bf16", seed=SEED + 3)
+    assert sg.sg_last_kernel() == TENSOR
+    assert_within_bound(O, want, S, "conv2d config 4")
+
+
+@pytest.mark.parametrize("family", [FFMA, TENSOR])
+@pytest.mark.parametrize("N,Wo,C,KW,F,sw,dw", [(4, 300, 64, 3, 128, 1, 1), (3, 333, 72, 5, 40, 1, 1),
+                                               (2, 500, 64, 3, 64, 2, 1), (2, 411, 128, 3, 72, 1, 2),
+                                               (5, 97, 200, 2, 136, 3, 2)])
+def test_conv1d_bf16(family, N, Wo, C, KW, F, sw, dw):
+    O, want, S = run_conv1d(N, Wo, C, KW, F, sw, dw, "bf16", family=family, seed=SEED + 4)
+    assert sg.sg_last_kernel() == family
+    assert_within_bound(O, want, S, "conv1d bf16")
+
+
+@pytest.mark.parametrize("family", [FFMA, TENSOR])
+@pytest.mark.parametrize("N,Ho,Wo,C,KH,KW,F,st,dl", [(3, 20, 20, 64, 3, 3, 128, (1, 1), (1, 1)),
+                                                      (4, 13, 17, 72, 2, 3, 40, (1, 1), (1, 1)),
+                                                      (2, 20, 19, 64, 3, 3, 64, (2, 2), (1, 1)),
+                                                      (3, 21, 18, 64, 3, 2, 72, (1, 1), (2, 2)),
+                                                      (1, 40, 40, 32, 3, 3, 64, (2, 1), (1, 3)),
+                                                      (1, 55, 55, 32, 3, 3, 64, (2, 2), (2, 2))])
+def test_conv2d_bf16(family, N, Ho, Wo, C, KH, KW, F, st, dl):
+    O, want, S = run_conv2d(N, Ho, Wo, C, KH, KW, F, st, dl, "bf16", family=family, seed=SEED + 5)
+    assert sg.sg_last_kernel() == family
+    assert_within_bound(O, want, S, "conv2d bf16")
+
+
+@pytest.mark.parametrize("N,Ho,Wo,C,KH,KW,F,st,dl", [(1, 5, 6, 3, 2, 3, 5, (1, 1), (1, 1)), (2, 9, 7, 32, 3, 3, 64, (1, 2), (2, 1)),
+                                                      (1, 20, 20, 32, 3, 3, 64, (1, 1), (1, 1))])
+def test_conv2d_f32(N, Ho, Wo, C, KH, KW, F, st, dl):
+    O, want, S = run_conv2d(N, Ho, Wo, C, KH, KW, F, st, dl, "f32", seed=SEED + 6)
+    assert_within_bound(O, want, S, "conv2d f32")
+
+
+@pytest.mark.parametrize("family", [FFMA, TENSOR])
+def test_conv_integer_inputs_are_bit_exact(family):
+    O, want, S = run_conv2d(2, 24, 24, 64, 3, 3, 64, (1, 1), (1, 1), "bf16", family=family, dist="ints", seed=SEED + 7)
+    assert np.array_equal(O.cpu().numpy().astype(np.float64), want)
+    O, want, S = run_conv1d(3, 400, 64, 3, 64, 1, 1, "bf16", family=family, dist="ints", seed=SEED + 7)
+    assert np.array_equal(O.cpu().numpy().astype(np.float64), want)
+
+
+@pytest.mark.parametrize("family", [FFMA, TENSOR])
+def test_conv_accumulate_and_oversized_input(family):
+    O, want, S = run_conv2d(3, 18, 22, 64, 3, 3, 72, (1, 1), (1, 1), "bf16", family=family, accumulate=True,
+                            seed=SEED + 8, extra=(2, 3))
+    assert_within_bound(O, want, S, "conv2d accumulate, larger input")
+    O, want, S = run_conv1d(3, 350, 64, 3, 64, 1, 1, "bf16", family=family, accumulate=True, seed=SEED + 8, extra_w=5)
+    assert_within_bound(O, want, S, "conv1d accumulate, larger input")
+
+
+def test_conv_delta_filter_is_a_shift_on_gpu():
+    # closed form on the device path: K[kh0,kw0,c,f] = delta(c,f)  =>  O[n,h,w,f] = I[n,h+kh0,w+kw0,f]
+    N, H, W, C = 2, 30, 34, 64
+    I, i = operand((N, H, W, C), SEED, 12, "normal", "bf16")
+    Kf = torch.zeros(3, 3, C, C, device="cuda", dtype=torch.bfloat16)
+    Kf[2, 1] = torch.eye(C, device="cuda", dtype=torch.bfloat16)
+    O = torch.empty(N, H - 2, W - 2, C, device="cuda")
+    for fam in (FFMA, TENSOR):
+        sg.sg_set_kernel_override(fam)
+        O.fill_(float("nan"))
+        sg.sg_conv2d_nhwc_hwcf(I, Kf, O)
+        torch.cuda.synchronize()
+        assert torch.equal(O, I[:, 2:H, 1:W - 1, :].float())
+
+
+def test_conv_noncontiguous_views_use_generic_kernel():
+    N, Ho, Wo, C, F = 2, 10, 12, 16, 24
+    Ibig, i = operand((N, Ho + 2, Wo + 2, C + 2), SEED, 13, "normal", "bf16")
+    Kf, k = operand((3, 3, C, F), SEED, 14, "normal", "bf16")
+    Obig = torch.zeros(N, Ho, Wo, F + 1, device="cuda")
+    sg.sg_conv2d_nhwc_hwcf(Ibig[..., 1:C + 1], Kf, Obig[..., 1:])
+    assert sg.sg_last_kernel() == FFMA
+    want, S = ref.conv2d_nhwc_hwcf(np.ascontiguousarray(i[..., 1:C + 1]), k)
+    assert_within_bound(Obig[..., 1:], want, S, "strided views")
+    assert torch.all(Obig[..., 0] == 0)
+
+
+# ------------------------------------------------------------------ full-size problems, sampled outputs
+
+def sample_points(M, N, count, seed):
+    h = inputs.splitmix64(np.arange(2 * count, dtype=np.uint64) ^ np.uint64(seed))
+    pm = (h[:count] % np.uint64(M)).astype(np.int64)
+    pn = (h[count:] % np.uint64(N)).astype(np.int64)
+    # add the corners and the tile seams, where an indexing mistake would show first
+    edge_m = np.array([0, 0, M - 1, M - 1, 127 % M, 128 % M, M // 2], np.int64)
+    edge_n = np.array([0, N - 1, 0, N - 1, 63 % N, 64 % N, N // 2], np.int64)
+    return np.concatenate([pm, edge_m]), np.concatenate([pn, edge_n])
+
+
+@pytest.mark.parametrize("M,N,K,cfg", [(4096, 4096, 4096, 1), (8192, 8192, 8192, 4), (16384, 64, 4096, 4),
+                                       (4096, 256, 2048, 1), (256, 4096, 512, 1)])
+def test_full_size_bf16_matmul_sampled(M, N, K, cfg):
+    A, a = operand((M, K), SEED + cfg, 1, "uniform", "bf16")
+    B, b = operand((K, N), SEED + cfg, 2, "uniform", "bf16")
+    C = torch.full((M, N), float("nan"), device="cuda")
+    sg.sg_matmul(A, B, C)
+    torch.cuda.synchronize()
+    assert sg.sg_last_kernel() == TENSOR
+    pm, pn = sample_points(M, N, 4096, 99)
+    want, S = ref.matmul_points(a, b, pm, pn)
+    got = C[torch.from_numpy(pm).cuda(), torch.from_numpy(pn).cuda()]
+    assert_within_bound(got, want, S, f"sampled {M}x{N}x{K}")
+    assert not torch.isnan(C).any()            # every element was written
+    # a property that holds at any size: row sums of C equal A . (row sums of B)
+    rs = (A.double() @ B.double().sum(dim=1, keepdim=True)).squeeze(1)
+    assert torch.allclose(C.double().sum(dim=1), rs, rtol=1e-6, atol=1e-2 * K ** 0.5)
+
+
+def test_full_size_f32_matmul_sampled():
+    M = N = K = 1024
+    A, a = operand((M, K), SEED + 1, 1, "uniform", "f32")
+    B, b = operand((K, N), SEED + 1, 2, "uniform", "f32")
+    C = torch.full((M, N), float("nan"), device="cuda")
+    sg.sg_matmul(A, B, C)
+    torch.cuda.synchronize()
+    pm, pn = sample_points(M, N, 4096, 98)
+    want, S = ref.matmul_points(a, b, pm, pn)
+    got = C[torch.from_numpy(pm).cuda(), torch.from_numpy(pn).cuda()]
+    assert_within_bound(got, want, S, "sampled f32 1024^3")
+    assert not torch.isnan(C).any()
