@@ -125,55 +125,101 @@ def time_launches(fn, iters, warmup):
     return e0.elapsed_time(e1) / iters
 
 
-def per_op_table(sg, peaks, seed):
-    """Other configured ops: (name, flops, compulsory bytes, dtype, callable over rotating buffers)."""
+def time_graph(calls, reps, warmup=3):
+    """Average device time per call in ms with the calls captured once into a CUDA graph
+    and replayed, so that host-side call overhead is outside the measurement."""
     import torch
-    rows = []
-    ffma_peak = 148 * 128 * 2 * 1.965e9 / 1e12      # TFLOP/s at the maximum SM clock
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for c in calls[:2]:
+            c()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        for c in calls:
+            c()
+    for _ in range(warmup):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps / len(calls)
 
-    def add(name, flops, bytes_, dtype, make, call, iters):
-        sets = max(2, int(400e6 // max(bytes_, 1)) + 1)
-        sets = min(sets, 16)
-        bufs = [make(s) for s in range(sets)]
-        ms = time_launches(lambda i: call(*bufs[i % sets]), iters, 3)
-        fam = sg.sg_last_kernel()
-        tf = flops / (ms * 1e-3) / 1e12
-        t_compute = flops / ((peaks["bf16_tflops"] if fam == sg.SG_KERNEL_TENSOR else ffma_peak) * 1e12)
-        t_bytes = bytes_ / (peaks["hbm_gbs"] * 1e9)
-        bound = max(t_compute, t_bytes)
-        rows.append({"op": name, "dtype": dtype, "kernel": "tensor" if fam == sg.SG_KERNEL_TENSOR else "ffma",
-                     "us": round(ms * 1e3, 2), "gflops": round(tf * 1e3, 1),
-                     "bound": "hbm" if t_bytes > t_compute else ("tensor" if fam == sg.SG_KERNEL_TENSOR else "ffma"),
-                     "roofline_us": round(bound * 1e6, 2), "frac": round(bound / (ms * 1e-3), 4),
-                     "rotating_sets": sets})
-        del bufs
-        torch.cuda.empty_cache()
 
-    def mm(Mx, Nx, Kx, dtype, iters, label):
+def op_specs(sg, seed):
+    """The other configured ops: name -> (label, flops, compulsory bytes, dtype, make(set) -> buffers, call)."""
+    import torch
+
+    def mm(Mx, Nx, Kx, dtype, label):
         es = 2 if dtype == "bf16" else 4
-        add(label, 2.0 * Mx * Nx * Kx, (Mx * Kx + Kx * Nx) * es + Mx * Nx * 4, dtype,
-            lambda s: (gpu_operand((Mx, Kx), seed, 10 + s, "uniform", dtype), gpu_operand((Kx, Nx), seed, 40 + s, "uniform", dtype),
-                       torch.empty(Mx, Nx, device="cuda")),
-            lambda a, b, c: sg.sg_matmul(a, b, c), iters)
+        return (label, 2.0 * Mx * Nx * Kx, (Mx * Kx + Kx * Nx) * es + Mx * Nx * 4, dtype,
+                lambda s: (gpu_operand((Mx, Kx), seed, 10 + s, "uniform", dtype),
+                           gpu_operand((Kx, Nx), seed, 40 + s, "uniform", dtype), torch.empty(Mx, Nx, device="cuda")),
+                lambda a, b, c: sg.sg_matmul(a, b, c))
 
-    mm(128, 128, 128, "f32", 200, "matmul 128^3 f32 (config 1)")
-    mm(4096, 4096, 4096, "f32", 5, "matmul 4096^3 f32 (sweep corner)")
-    mm(1024, 1024, 1024, "bf16", 50, "matmul 1024^3 bf16 (sweep point)")
-    mm(8192, 8192, 8192, "bf16", 5, "matmul 8192^3 bf16 (config 5)")
-    mm(16384, 64, 4096, "bf16", 50, "matmul 16384x64x4096 bf16 (config 5, skinny)")
-    # conv1d config 3: N=32, W=1026, C=64, KW=3, F=128, f32
-    add("conv_1d_nwc_wcf 32x1026x64 * 3x64x128 f32 (config 3)", 2.0 * 32 * 1024 * 128 * 3 * 64,
-        (32 * 1026 * 64 + 3 * 64 * 128) * 4 + 32 * 1024 * 128 * 4, "f32",
-        lambda s: (gpu_operand((32, 1026, 64), seed, 70 + s, "uniform", "f32"), gpu_operand((3, 64, 128), seed, 90, "uniform", "f32"),
-                   torch.empty(32, 1024, 128, device="cuda")),
-        lambda i, k, o: sg.sg_conv1d_nwc_wcf(i, k, o), 20)
-    # conv2d config 4: N=16, 58x58x64, 3x3, F=128, bf16
-    add("conv_2d_nhwc_hwcf 16x58x58x64 * 3x3x64x128 bf16 (config 4)", 2.0 * 16 * 56 * 56 * 128 * 9 * 64,
-        (16 * 58 * 58 * 64 + 9 * 64 * 128) * 2 + 16 * 56 * 56 * 128 * 4, "bf16",
-        lambda s: (gpu_operand((16, 58, 58, 64), seed, 100 + s, "normal", "bf16"), gpu_operand((3, 3, 64, 128), seed, 120, "normal", "bf16"),
-                   torch.empty(16, 56, 56, 128, device="cuda")),
-        lambda i, k, o: sg.sg_conv2d_nhwc_hwcf(i, k, o), 50)
-    return rows
+    return {
+        "matmul128_f32": mm(128, 128, 128, "f32", "matmul 128^3 f32 (config 1)"),
+        "matmul4096_f32": mm(4096, 4096, 4096, "f32", "matmul 4096^3 f32 (sweep corner)"),
+        "matmul4096_bf16": mm(4096, 4096, 4096, "bf16", "matmul 4096^3 bf16 (sweep corner)"),
+        "matmul1024_bf16": mm(1024, 1024, 1024, "bf16", "matmul 1024^3 bf16 (sweep point)"),
+        "matmul8192_bf16": mm(8192, 8192, 8192, "bf16", "matmul 8192^3 bf16 (config 5)"),
+        "matmul_skinny_bf16": mm(16384, 64, 4096, "bf16", "matmul 16384x64x4096 bf16 (config 5, skinny)"),
+        # conv1d config 3: N=32, W=1026, C=64, KW=3, F=128, f32
+        "conv1d_c3": ("conv_1d_nwc_wcf 32x1026x64 * 3x64x128 f32 (config 3)", 2.0 * 32 * 1024 * 128 * 3 * 64,
+                      (32 * 1026 * 64 + 3 * 64 * 128) * 4 + 32 * 1024 * 128 * 4, "f32",
+                      lambda s: (gpu_operand((32, 1026, 64), seed, 70 + s, "uniform", "f32"),
+                                 gpu_operand((3, 64, 128), seed, 90, "uniform", "f32"),
+                                 torch.empty(32, 1024, 128, device="cuda")),
+                      lambda i, k, o: sg.sg_conv1d_nwc_wcf(i, k, o)),
+        # conv2d config 4: N=16, 58x58x64, 3x3, F=128, bf16
+        "conv2d_c4": ("conv_2d_nhwc_hwcf 16x58x58x64 * 3x3x64x128 bf16 (config 4)", 2.0 * 16 * 56 * 56 * 128 * 9 * 64,
+                      (16 * 58 * 58 * 64 + 9 * 64 * 128) * 2 + 16 * 56 * 56 * 128 * 4, "bf16",
+                      lambda s: (gpu_operand((16, 58, 58, 64), seed, 100 + s, "normal", "bf16"),
+                                 gpu_operand((3, 3, 64, 128), seed, 120, "normal", "bf16"),
+                                 torch.empty(16, 56, 56, 128, device="cuda")),
+                      lambda i, k, o: sg.sg_conv2d_nhwc_hwcf(i, k, o)),
+    }
+
+
+def measure_op(sg, peaks, spec, reps=None):
+    """Times one op: buffers rotate over enough sets to exceed L2 between reuses."""
+    import torch
+    label, flops, bytes_, dtype, make, call = spec
+    ffma_peak = 148 * 128 * 2 * 1.965e9 / 1e12      # TFLOP/s at the maximum SM clock
+    sets = min(16, max(2, int(400e6 // max(bytes_, 1)) + 1))
+    bufs = [make(s) for s in range(sets)]
+    ncalls = sets * 2 if bytes_ < 100e6 else sets
+    calls = [(lambda b=bufs[i % sets]: call(*b)) for i in range(ncalls)]
+    call(*bufs[0])
+    torch.cuda.synchronize()
+    fam = sg.sg_last_kernel()
+    est_ms = max(flops / 3e14, 5e-3)
+    if reps is None:
+        reps = int(max(3, min(50, 0.25 / (est_ms * 1e-3 * ncalls))))
+    ms = time_graph(calls, reps)
+    host_ms = time_launches(lambda i: call(*bufs[i % sets]), max(3, min(100, ncalls * 2)), 2)
+    tf = flops / (ms * 1e-3) / 1e12
+    t_compute = flops / ((peaks["bf16_tflops"] if fam == sg.SG_KERNEL_TENSOR else ffma_peak) * 1e12)
+    t_bytes = bytes_ / (peaks["hbm_gbs"] * 1e9)
+    bound = max(t_compute, t_bytes)
+    row = {"op": label, "dtype": dtype, "kernel": "tensor" if fam == sg.SG_KERNEL_TENSOR else "ffma",
+           "us": round(ms * 1e3, 2), "us_with_host_call": round(host_ms * 1e3, 2), "gflops": round(tf * 1e3, 1),
+           "gbs": round(bytes_ / (ms * 1e-3) / 1e9, 1),
+           "bound": "hbm" if t_bytes > t_compute else ("tensor" if fam == sg.SG_KERNEL_TENSOR else "ffma"),
+           "roofline_us": round(bound * 1e6, 2), "frac": round(bound / (ms * 1e-3), 4), "rotating_sets": sets,
+           "timing": "CUDA graph replay"}
+    del bufs, calls
+    torch.cuda.empty_cache()
+    return row
+
+
+def per_op_table(sg, peaks, seed):
+    specs = op_specs(sg, seed)
+    return [measure_op(sg, peaks, specs[name]) for name in specs if name != "matmul4096_bf16"]
 
 
 def cpu_baseline(target_seconds=12.0):
@@ -228,6 +274,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-per-op", action="store_true", help="skip the per-op table")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
+    ap.add_argument("--op", default=None, help="time only this op of the per-op table (used for profiler captures)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -253,6 +300,13 @@ def main():
     peaks = load_peaks()
     seed = inputs.BASE_SEED + 1
     warmup = max(args.warmup, 3)
+
+    if args.op is not None:
+        specs = op_specs(sg, seed)
+        if args.op not in specs:
+            raise SystemExit(f"--op must be one of {sorted(specs)}")
+        print(json.dumps(measure_op(sg, peaks, specs[args.op], reps=max(1, min(args.steps, 5)))), flush=True)
+        return
 
     sets = [(gpu_operand((M, K), seed, 1 + 3 * s, "uniform", "bf16"), gpu_operand((K, N), seed, 2 + 3 * s, "uniform", "bf16"),
              torch.empty(M, N, device="cuda")) for s in range(N_SETS)]
