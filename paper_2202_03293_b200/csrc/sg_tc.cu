@@ -172,24 +172,31 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_b
     return d;
 }
 
-// Instruction descriptor: f32 accumulator, bf16 A and B, A K-major, B N-major, M = 128, N = BN.
-__host__ __device__ constexpr uint32_t make_idesc_bf16(int n) {
+// Instruction descriptor: f32 accumulator, bf16 A and B, A K-major, B N-major.
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int n, int m) {
     return (1u << 4)                       // D format: f32
          | (1u << 7)                       // A format: bf16
          | (1u << 10)                      // B format: bf16
          | (0u << 15)                      // A major: K
          | (1u << 16)                      // B major: MN (filter stored [k][f], f contiguous)
          | ((uint32_t)(n >> 3) << 17)      // N / 8
-         | ((uint32_t)(BM >> 4) << 24);    // M / 16
+         | ((uint32_t)(m >> 4) << 24);     // M / 16 (128 for one CTA, 256 for a pair)
 }
 
-template <int BN>
+template <int BN, int CG>
 struct Cfg {
-    static constexpr int B_STAGE_BYTES = BK * BN * 2;
+    // CG = 1: one CTA owns a 128 x BN tile.  CG = 2: a pair of CTAs (one cluster) owns a
+    // 256 x BN tile; each CTA stages its own 128 input rows and its own BN/2 filter columns,
+    // and one tcgen05.mma.cta_group::2 per k-step feeds both SMs' tensor cores, so every
+    // filter element is staged once per pair instead of once per CTA.
+    static constexpr int B_COLS = BN / CG;                    // filter columns staged by this CTA
+    static constexpr int B_STAGE_BYTES = BK * B_COLS * 2;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-    static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
+    static constexpr int STAGES = (196608 / STAGE_BYTES) > 8 ? 8 : (196608 / STAGE_BYTES);
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // two accumulator buffers
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static_assert(B_COLS % 64 == 0 && BN % 16 == 0 && BN <= 256, "tile width");
+    static_assert(TMEM_COLS <= 512 && (TMEM_COLS & (TMEM_COLS - 1)) == 0, "TMEM columns");
 };
 
 // Static tile order: groups of 8 tile-rows, row index fastest inside a group, so that the
@@ -204,11 +211,66 @@ __device__ __forceinline__ void tile_coords(int t, int num_m_tiles, int num_n_ti
     mt = g * GM + (r - nt * rows);
 }
 
-template <int BN>
+// ---- cluster helpers (CG = 2) ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA loads whose completion may be signalled on the peer CTA's mbarrier (cta_group::2).
+__device__ __forceinline__ void tma_load_2d_cg2(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_cg2(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z, int w) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_3d_cg2(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                                       int c, int w, int n, unsigned short off_w) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2], {%6};"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(n), "h"(off_w) : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_4d_cg2(uint32_t dst, const CUtensorMap *map, uint32_t bar,
+                                                       int c, int w, int h, int n, unsigned short off_w, unsigned short off_h) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B, 256 x N x 16 across the CTA pair.
+__device__ __forceinline__ void umma_bf16_cg2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives (once the pair's MMAs issued so far have finished) on a barrier that may live in
+// either CTA of the pair; `cluster_bar` is a shared::cluster address.
+__device__ __forceinline__ void umma_commit_cg2(uint32_t cluster_bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar) : "memory");
+}
+
+template <int BN, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_flt,
                const __grid_constant__ CUtensorMap map_out, const TcParams p) {
-    using C = Cfg<BN>;
+    using C = Cfg<BN, CG>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -227,35 +289,49 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_gen + 8 * (2 * C::STAGES + 4) + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // In a pair, CTA 0 (the leader) issues the MMAs; both CTAs produce and both run epilogues.
+    const uint32_t cta_rank = CG == 2 ? cluster_ctarank() : 0u;
+    const int group_id = CG == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int num_groups = CG == 2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
+        // full: one arrive.expect_tx (by the leader's producer).  acc_empty: one arrive per epilogue
+        // warp of every CTA of the group.  empty / acc_full: one tcgen05.commit.
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 4 * CG); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {   // TMEM allocation is a warp-wide operation
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(const_cast<uint32_t *>(tmem_ptr_slot))), "r"((uint32_t)C::TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (warp == 1) {   // TMEM allocation is a warp-wide operation (the same warp in both CTAs of a pair)
+        if constexpr (CG == 2) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(const_cast<uint32_t *>(tmem_ptr_slot))), "r"((uint32_t)C::TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(const_cast<uint32_t *>(tmem_ptr_slot))), "r"((uint32_t)C::TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (CG == 2) cluster_sync_all();   // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_slot;
 
-    const int num_tiles = p.num_m_tiles * p.num_n_tiles;
+    const int num_tiles = p.num_m_tiles * p.num_n_tiles;   // tiles of (CG*128) x BN
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
         if (lane == 0) {
             int it = 0;   // k-block counter across all of this CTA's tiles
             bool ok = true;
-            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            for (int t = group_id; t < num_tiles && ok; t += num_groups) {
                 int mt, nt;
                 tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
-                const int m0 = mt * BM, n0 = nt * BN;
-                int pix_n = 0, pix_h = 0, pix_w = 0;   // first output pixel of the tile
+                const int m0 = (mt * CG + (int)cta_rank) * BM;
+                const int n0 = nt * BN + (int)cta_rank * C::B_COLS;
+                int pix_n = 0, pix_h = 0, pix_w = 0;   // first output pixel of this CTA's rows
                 if (p.a_mode != 0) {
                     int hw = p.Ho * p.Wo;
                     pix_n = m0 / hw;
@@ -269,32 +345,51 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t a_dst = stages_addr + s * C::STAGE_BYTES;
                     const uint32_t b_dst = a_dst + A_STAGE_BYTES;
-                    mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
                     const int tap = kb / p.kb_per_tap;
                     const int c0 = (kb - tap * p.kb_per_tap) * BK;
                     const int kh = tap / p.KW, kw = tap - kh * p.KW;
-                    if (p.a_mode == 0) {
-                        tma_load_2d(a_dst, &map_in, full_bar(s), c0, m0);
-                    } else if (p.a_mode == 1) {
-                        tma_load_im2col_3d(a_dst, &map_in, full_bar(s), c0, pix_w * p.sw, pix_n,
-                                           (unsigned short)(kw * p.dw));
-                    } else {
-                        tma_load_im2col_4d(a_dst, &map_in, full_bar(s), c0, pix_w * p.sw, pix_h * p.sh, pix_n,
-                                           (unsigned short)(kw * p.dw), (unsigned short)(kh * p.dh));
-                    }
+                    if constexpr (CG == 1) {
+                        const uint32_t bar = full_bar(s);
+                        mbar_expect_tx(bar, C::STAGE_BYTES);
+                        if (p.a_mode == 0) {
+                            tma_load_2d(a_dst, &map_in, bar, c0, m0);
+                        } else if (p.a_mode == 1) {
+                            tma_load_im2col_3d(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_n, (unsigned short)(kw * p.dw));
+                        } else {
+                            tma_load_im2col_4d(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_h * p.sh, pix_n,
+                                               (unsigned short)(kw * p.dw), (unsigned short)(kh * p.dh));
+                        }
 #pragma unroll
-                    for (int j = 0; j < BN / 64; ++j)
-                        tma_load_4d(b_dst + j * (BK * 128), &map_flt, full_bar(s), n0 + j * 64, c0, kw, kh);
+                        for (int j = 0; j < C::B_COLS / 64; ++j)
+                            tma_load_4d(b_dst + j * (BK * 128), &map_flt, bar, n0 + j * 64, c0, kw, kh);
+                    } else {
+                        // both CTAs' bytes are counted on the leader's barrier, which its MMA thread waits
+                        // on; the leader alone arms it, for the pair's total (a remote arrive by the
+                        // peer would order it after its own loads in flight and serialise the ring)
+                        const uint32_t bar = map_to_cta(full_bar(s), 0);
+                        if (cta_rank == 0) mbar_expect_tx(full_bar(s), CG * C::STAGE_BYTES);
+                        if (p.a_mode == 0) {
+                            tma_load_2d_cg2(a_dst, &map_in, bar, c0, m0);
+                        } else if (p.a_mode == 1) {
+                            tma_load_im2col_3d_cg2(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_n, (unsigned short)(kw * p.dw));
+                        } else {
+                            tma_load_im2col_4d_cg2(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_h * p.sh, pix_n,
+                                                   (unsigned short)(kw * p.dw), (unsigned short)(kh * p.dh));
+                        }
+#pragma unroll
+                        for (int j = 0; j < C::B_COLS / 64; ++j)
+                            tma_load_4d_cg2(b_dst + j * (BK * 128), &map_flt, bar, n0 + j * 64, c0, kw, kh);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(BN);
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && cta_rank == 0) {
+            constexpr uint32_t idesc = make_idesc_bf16(BN, CG * BM);
             int it = 0, tl = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tl) {
+            for (int t = group_id; t < num_tiles && ok; t += num_groups, ++tl) {
                 const int buf = tl & 1;
                 if (!mbar_wait(acc_empty_bar(buf), ((tl >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -314,12 +409,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     const uint64_t b_desc = make_smem_desc(b_addr, BK * 128, 1024);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
-                        umma_bf16(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc,
-                                  (kb > 0 || k > 0) ? 1u : 0u);
+                        const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+                        if constexpr (CG == 1) umma_bf16(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc, acc);
+                        else umma_bf16_cg2(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc, acc);
                     }
-                    umma_commit(empty_bar(s));   // the stage is free once these MMAs have read it
+                    // the stage is free (in every CTA of the group) once these MMAs have read it
+                    if constexpr (CG == 1) {
+                        umma_commit(empty_bar(s));
+                    } else {
+                        umma_commit_cg2(map_to_cta(empty_bar(s), 0));
+                        umma_commit_cg2(map_to_cta(empty_bar(s), 1));
+                    }
                 }
-                if (ok) umma_commit(acc_full_bar(buf));
+                if (ok) {
+                    if constexpr (CG == 1) {
+                        umma_commit(acc_full_bar(buf));
+                    } else {
+                        umma_commit_cg2(map_to_cta(acc_full_bar(buf), 0));
+                        umma_commit_cg2(map_to_cta(acc_full_bar(buf), 1));
+                    }
+                }
             }
         }
     } else {
@@ -329,10 +438,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         uint8_t *stg_gen = staging_gen + (warp - 2) * 8192;
         int tl = 0, chunk_count = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tl) {
+        for (int t = group_id; t < num_tiles && ok; t += num_groups, ++tl) {
             int mt, nt;
             tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
-            const int m0 = mt * BM, n0 = nt * BN;
+            const int m0 = (mt * CG + (int)cta_rank) * BM, n0 = nt * BN;
             const int buf = tl & 1;
             if (!mbar_wait(acc_full_bar(buf), (tl >> 1) & 1, abort_flag)) { ok = false; break; }
             tc_fence_after();
@@ -362,10 +471,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     bulk_commit();
                 }
             }
-            // every tcgen05.ld of this buffer has completed: hand it back to the MMA warp
+            // every tcgen05.ld of this buffer has completed: hand it back to the MMA thread
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty_bar(buf));
+            if (lane == 0) {
+                if constexpr (CG == 1) mbar_arrive(acc_empty_bar(buf));
+                else mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));
+            }
         }
         if (lane == 0) bulk_wait_all();
     }
@@ -377,9 +489,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         for (int i = 0; i < 200; ++i) __nanosleep(5000);
         __syncthreads();
     }
+    // a pair leaves together: the leader's MMAs read the peer's shared memory and both CTAs
+    // signal barriers in each other's shared memory
+    if constexpr (CG == 2) cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS) : "memory");
+        if constexpr (CG == 2)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS) : "memory");
     }
 }
 
@@ -397,12 +515,13 @@ struct Driver {
     EncodeIm2colFn im2col = nullptr;
     int num_sms = 0;
     int device = -1;
-    bool attr_set[3] = {false, false, false};
+    bool attr_set[8] = {};
     bool ok = false;
 };
 std::mutex g_mu;
 Driver g_drv;
-int g_bn_override = -1;   // -1: not read yet; 0: automatic
+int g_bn_override = -1;   // tile width forced by SG_TC_BN (-1: not read yet; 0: automatic)
+int g_cg_override = 0;    // CTAs per tile forced by SG_TC_CG (0: automatic)
 
 bool init_driver() {
     int dev = 0;
@@ -427,20 +546,41 @@ bool init_driver() {
 
 inline bool mult(int64_t v, int64_t q) { return v % q == 0; }
 
-template <int BN>
-sg_status launch_bn(const CUtensorMap &mi, const CUtensorMap &mf, const CUtensorMap &mo, const TcParams &tp,
-                    int slot, cudaStream_t stream) {
-    using C = Cfg<BN>;
+struct Variant { int bn, cg; double step_cost; };
+// Relative cost of one 16-deep k-step of a tile per variant (measured on large problems):
+// narrow tiles pay more shared-memory traffic per flop, CTA pairs stage the filter once.
+constexpr Variant kVariants[] = {{64, 1, 80.0}, {128, 1, 102.0}, {256, 1, 128.0}, {128, 2, 95.0}, {256, 2, 120.0}};
+constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
+
+template <int BN, int CG>
+sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUtensorMap &mo, TcParams tp, int M, int N,
+                         int slot, cudaStream_t stream) {
+    using C = Cfg<BN, CG>;
     if (!g_drv.attr_set[slot]) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
             return SG_ERR_CUDA;
         g_drv.attr_set[slot] = true;
     }
-    int tiles = tp.num_m_tiles * tp.num_n_tiles;
-    int grid = tiles < g_drv.num_sms ? tiles : g_drv.num_sms;
-    tc_gemm_kernel<BN><<<grid, NUM_THREADS, C::SMEM_BYTES, stream>>>(mi, mf, mo, tp);
+    tp.num_m_tiles = (M + CG * BM - 1) / (CG * BM);
+    tp.num_n_tiles = (N + BN - 1) / BN;
+    const int tiles = tp.num_m_tiles * tp.num_n_tiles;
+    const int groups = g_drv.num_sms / CG;
+    const int grid = CG * (tiles < groups ? tiles : groups);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CG;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<BN, CG>, mi, mf, mo, tp);
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? SG_OK : SG_ERR_CUDA;
+    return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
 }
 
 }  // namespace
@@ -467,6 +607,8 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     if (g_bn_override < 0) {
         const char *e = getenv("SG_TC_BN");
         g_bn_override = e ? atoi(e) : 0;
+        e = getenv("SG_TC_CG");
+        g_cg_override = e ? atoi(e) : 0;
     }
 
     alignas(64) CUtensorMap map_in, map_flt, map_out;
@@ -550,26 +692,36 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
     }
 
-    // ---- tile width: fewest (waves x per-tile cost); narrower tiles cost more shared-memory
-    //      traffic per flop, wider ones quantise worse ----
-    int bn = g_bn_override;
-    if (bn != 64 && bn != 128 && bn != 256) {
+    // ---- tile variant: fewest (waves x per-tile cost); narrower tiles cost more shared-memory
+    //      traffic per flop, wider ones and CTA pairs quantise worse on small problems ----
+    int pick = -1;
+    if (g_bn_override > 0) {
+        for (int i = 0; i < kNumVariants; ++i)
+            if (kVariants[i].bn == g_bn_override && kVariants[i].cg == (g_cg_override > 0 ? g_cg_override : 1)) pick = i;
+    }
+    for (int pass = 0; pass < 2 && pick < 0; ++pass) {   // pass 1 drops a forced group size that does not fit
         double best = 1e300;
-        const int cand[3] = {64, 128, 256};
-        const double step_cost[3] = {48.0, 64.0, 128.0};
-        for (int i = 0; i < 3; ++i) {
-            if (cand[i] > 64 && cand[i] / 2 >= p.N) continue;   // at most half of the tile would be used
-            int64_t tiles = (int64_t)((p.M + BM - 1) / BM) * ((p.N + cand[i] - 1) / cand[i]);
-            int64_t waves = (tiles + g_drv.num_sms - 1) / g_drv.num_sms;
-            double cost = (double)waves * step_cost[i];
-            if (cost < best) { best = cost; bn = cand[i]; }
+        for (int i = 0; i < kNumVariants; ++i) {
+            const Variant &v = kVariants[i];
+            if (pass == 0 && g_cg_override > 0 && v.cg != g_cg_override) continue;
+            if (v.bn > 64 && v.bn / 2 >= p.N) continue;          // at most half of the tile would be used
+            if (v.cg == 2 && p.M <= BM) continue;                // the second CTA would have no rows
+            int64_t tiles = (int64_t)((p.M + v.cg * BM - 1) / (v.cg * BM)) * ((p.N + v.bn - 1) / v.bn);
+            int64_t groups = g_drv.num_sms / v.cg;
+            int64_t waves = (tiles + groups - 1) / groups;
+            // a pair pays a fixed price (cluster launch, cross-CTA signalling) worth ~6 k-blocks
+            double cost = (double)waves * tp.num_kb * v.step_cost + (v.cg == 2 ? 760.0 : 0.0);
+            if (cost < best) { best = cost; pick = i; }
         }
     }
-    tp.num_m_tiles = (p.M + BM - 1) / BM;
-    tp.num_n_tiles = (p.N + bn - 1) / bn;
-    if (bn == 64) return launch_bn<64>(map_in, map_flt, map_out, tp, 0, stream);
-    if (bn == 128) return launch_bn<128>(map_in, map_flt, map_out, tp, 1, stream);
-    return launch_bn<256>(map_in, map_flt, map_out, tp, 2, stream);
+    if (pick < 0) return SG_ERR_INTERNAL;
+    switch (pick) {
+        case 0: return launch_variant<64, 1>(map_in, map_flt, map_out, tp, p.M, p.N, 0, stream);
+        case 1: return launch_variant<128, 1>(map_in, map_flt, map_out, tp, p.M, p.N, 1, stream);
+        case 2: return launch_variant<256, 1>(map_in, map_flt, map_out, tp, p.M, p.N, 2, stream);
+        case 3: return launch_variant<128, 2>(map_in, map_flt, map_out, tp, p.M, p.N, 3, stream);
+        default: return launch_variant<256, 2>(map_in, map_flt, map_out, tp, p.M, p.N, 4, stream);
+    }
 }
 
 sg_status tensor_read_status(cudaStream_t stream) {

@@ -66,22 +66,28 @@ def test_matmul_f32_shapes(M, N, K):
     assert_within_bound(C, want, S, f"matmul f32 {M}x{N}x{K}")
 
 
-@pytest.mark.parametrize("bn", ["64", "128", "256"])
-def test_matmul_bf16_every_tile_width(bn, monkeypatch):
-    # the tile width is normally chosen from the shape; exercise each instantiation on a
-    # shape with ragged edges in m, n and k.  SG_TC_BN is read once per process, so these
-    # run in a child interpreter.
+@pytest.mark.parametrize("bn,cg", [("64", "1"), ("128", "1"), ("256", "1"), ("128", "2"), ("256", "2")])
+def test_tensor_path_every_tile_variant(bn, cg):
+    # the tile variant (width, one CTA or a CTA pair) is normally chosen from the shape; exercise
+    # each instantiation on shapes with ragged edges in m, n and k, several tiles per CTA, and
+    # on both convolutions.  The override is read once per process, so these run in a child.
     import subprocess, sys, os
     code = (
         "import sys; sys.path.insert(0, 'tests'); sys.path.insert(0, '.');"
         "import test_gpu_parity as t;"
         "from helpers import assert_within_bound;"
         "C, want, S = t.run_matmul(400, 520, 200, 'bf16', family=t.TENSOR, seed=t.SEED + 7);"
-        "assert_within_bound(C, want, S, 'bn');"
+        "assert_within_bound(C, want, S, 'ragged');"
         "C, want, S = t.run_matmul(400, 520, 200, 'bf16', family=t.TENSOR, accumulate=True, seed=t.SEED + 7);"
-        "assert_within_bound(C, want, S, 'bn acc'); t.sg.sg_check(); print('child-ok')"
+        "assert_within_bound(C, want, S, 'ragged acc');"
+        "C, want, S = t.run_matmul(2048 + 136, 2304, 328, 'bf16', family=t.TENSOR, seed=t.SEED + 7);"
+        "assert_within_bound(C, want, S, 'many tiles per CTA');"
+        "O, want, S = t.run_conv2d(5, 30, 27, 72, 3, 3, 136, (1, 1), (1, 1), 'bf16', family=t.TENSOR, seed=t.SEED + 7);"
+        "assert_within_bound(O, want, S, 'conv2d');"
+        "O, want, S = t.run_conv1d(3, 700, 64, 3, 200, 2, 2, 'bf16', family=t.TENSOR, seed=t.SEED + 7);"
+        "assert_within_bound(O, want, S, 'conv1d'); t.sg.sg_check(); print('child-ok')"
     )
-    env = dict(os.environ, SG_TC_BN=bn)
+    env = dict(os.environ, SG_TC_BN=bn, SG_TC_CG=cg)
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     out = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
     assert out.returncode == 0 and "child-ok" in out.stdout, out.stdout + out.stderr
