@@ -288,7 +288,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2202_03293_b200 import binding as sg
-    from paper_2202_03293_b200 import inputs
+    from paper_2202_03293_b200 import inputs, sharding
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -335,11 +335,7 @@ def main():
     launches = sg.sg_launch_count() - launches0
     clocks = sampler.stop()
     sg.sg_check()
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = sharding.max_over_ranks(e0.elapsed_time(e1), device="cuda")
     ms_per_step = ms_total / args.steps
     value = world * FLOPS_PER_STEP / (ms_per_step * 1e-3) / 1e9      # GFLOP/s, all ranks
 
@@ -364,11 +360,7 @@ def main():
         e2e_step(i)
     e1.record()
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = sharding.max_over_ranks(e0.elapsed_time(e1), device="cuda")
     e2e_value = world * FLOPS_PER_STEP / (e2e_ms / e2e_steps * 1e-3) / 1e9
 
     if rank != 0:
