@@ -21,6 +21,14 @@
 //                          filter is stored [k][f] with f contiguous, so it is consumed as
 //                          an MN-major operand instead of being transposed.
 //
+// f32 inputs run on the same pipeline as three tf32 products per k-step ("3xTF32"): the TMA
+// writes the raw f32 tiles into its ring, four converter warps split every element x into two
+// tf32 values hi = rn(x) and lo = rn(x - hi) and write them to a second ring of two slots
+// (transposing the filter tile to K-major on the way, which kind::tf32 needs), and the MMA
+// thread accumulates lo*hi + hi*lo + hi*hi in f32: the dropped terms are below 2^-21 |a*b|, so
+// f32 accuracy is kept.  Raw tiles are 128 rows x 32 f32 (input) and 32 k-rows x 32 f32
+// sub-tiles (filter), again 128 bytes per row.
+//
 // Every wait in this file is bounded: a wait that expires sets an abort flag in shared
 // memory and a bit in the device status word, every role then leaves its loop, the CTA
 // drains its copies, frees its TMEM and returns.
@@ -34,10 +42,10 @@ namespace sg {
 namespace {
 
 constexpr int BM = 128;           // rows of an output tile = lanes of TMEM = M of one MMA
-constexpr int BK = 64;            // bf16 elements per k-block = one 128-byte swizzle row
-constexpr int UMMA_K = 16;        // k extent of one tcgen05.mma for 16-bit inputs
-constexpr int NUM_THREADS = 192;  // 6 warps: producer, MMA, 4 epilogue
-constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int ROW_BYTES = 128;    // one k-block = one 128-byte swizzle row: 64 bf16 or 32 f32
+constexpr int K_STEPS = 4;        // tcgen05.mma per k-block and product: 32 bytes of k each
+constexpr int A_STAGE_BYTES = BM * ROW_BYTES;
+constexpr int CONVERTER_THREADS = 128;        // f32 path: 4 warps splitting tiles into hi and lo
 constexpr int STAGING_BYTES = 4 * 2 * 4096;   // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
 constexpr long long WAIT_BUDGET_CYCLES = 2000000000LL;   // ~1 s: far beyond any legitimate wait
 
@@ -76,12 +84,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// Same test with cluster-scope acquire: the barrier was signalled by threads of the peer CTA
+// whose shared-memory writes must be visible afterwards.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait.  Returns false when the budget expired or another role already aborted.
+template <bool CLUSTER_SCOPE = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
+    auto test = [&]() { return CLUSTER_SCOPE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+    if (test()) return true;
     const long long t0 = clock64();
     for (uint32_t it = 0;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (test()) return true;
         if ((it & 63u) == 63u) {
             if (*abort_flag) return false;
             if (clock64() - t0 > WAIT_BUDGET_CYCLES) {
@@ -142,6 +163,14 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Same shape with tf32 inputs (f32 words in shared memory, k extent 8).
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 // Arrives on the mbarrier once every tcgen05.mma issued so far by this thread has finished.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -172,31 +201,68 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_b
     return d;
 }
 
-// Instruction descriptor: f32 accumulator, bf16 A and B, A K-major, B N-major.
-__host__ __device__ constexpr uint32_t make_idesc_bf16(int n, int m) {
+// Instruction descriptor: f32 accumulator, A and B both bf16 (kind::f16) or both tf32
+// (kind::tf32), A K-major, B N-major.
+__host__ __device__ constexpr uint32_t make_idesc(int n, int m, bool tf32) {
     return (1u << 4)                       // D format: f32
-         | (1u << 7)                       // A format: bf16
-         | (1u << 10)                      // B format: bf16
+         | ((tf32 ? 2u : 1u) << 7)         // A format: bf16 = 1 in kind::f16, tf32 = 2 in kind::tf32
+         | ((tf32 ? 2u : 1u) << 10)        // B format: the same type as A
          | (0u << 15)                      // A major: K
-         | (1u << 16)                      // B major: MN (filter stored [k][f], f contiguous)
+         | ((tf32 ? 0u : 1u) << 16)        // B major: MN for bf16 (filter stored [k][f], f contiguous, read as
+                                           // is); kind::tf32 takes K-major operands only (an N-major
+                                           // descriptor makes the MMA a no-op), so the f32 path
+                                           // transposes the filter tile while splitting it
          | ((uint32_t)(n >> 3) << 17)      // N / 8
          | ((uint32_t)(m >> 4) << 24);     // M / 16 (128 for one CTA, 256 for a pair)
 }
 
-template <int BN, int CG>
+// 3xTF32 split of an f32 word x into two tf32 values (low 13 mantissa bits zero, so whatever
+// rounding the tensor core applies to its inputs leaves them unchanged): hi = x rounded to
+// nearest, lo = (x - hi) rounded to nearest; x - hi is exact in f32 and |x - hi - lo| <=
+// 2^-22 |x|.  Infinities and NaNs stay in hi alone; a finite x that would round up to
+// infinity is truncated instead.
+__device__ __forceinline__ uint32_t cvt_rna_tf32(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ uint32_t split_hi(uint32_t x) {
+    const uint32_t h = cvt_rna_tf32(__uint_as_float(x));
+    return (h & 0x7F800000u) == 0x7F800000u ? (x & 0xFFFFE000u) : h;
+}
+__device__ __forceinline__ uint32_t split_lo(uint32_t x, uint32_t hi) {
+    const uint32_t l = cvt_rna_tf32(__uint_as_float(x) - __uint_as_float(hi));
+    return (x & 0x7F800000u) == 0x7F800000u ? 0u : l;
+}
+
+template <int BN, int CG, bool F32>
 struct Cfg {
     // CG = 1: one CTA owns a 128 x BN tile.  CG = 2: a pair of CTAs (one cluster) owns a
     // 256 x BN tile; each CTA stages its own 128 input rows and its own BN/2 filter columns,
     // and one tcgen05.mma.cta_group::2 per k-step feeds both SMs' tensor cores, so every
     // filter element is staged once per pair instead of once per CTA.
+    static constexpr int ELT = F32 ? 4 : 2;                   // bytes per input element
+    static constexpr int BK = ROW_BYTES / ELT;                // elements per k-block
+    static constexpr int SUB_COLS = ROW_BYTES / ELT;          // filter columns per sub-tile (one 128-byte row)
+    static constexpr int SUB_BYTES = BK * ROW_BYTES;          // one filter sub-tile: BK k-rows
     static constexpr int B_COLS = BN / CG;                    // filter columns staged by this CTA
-    static constexpr int B_STAGE_BYTES = BK * B_COLS * 2;
-    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-    static constexpr int STAGES = (196608 / STAGE_BYTES) > 8 ? 8 : (196608 / STAGE_BYTES);
+    static constexpr int B_STAGE_BYTES = B_COLS * ROW_BYTES;  // = BK * B_COLS * ELT
+    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;   // written by TMA per stage
+    // bf16: one ring of stages, TMA -> MMA.  f32: the TMA ring holds raw tiles; a second ring of
+    // two slots holds what the converter warps make of them, [input hi | input lo | filter hi |
+    // filter lo], the filter transposed to K-major on the way (kind::tf32 takes no N-major operand).
+    static constexpr int SPLIT_SLOTS = F32 ? 2 : 0;
+    static constexpr int SPLIT_BYTES = 2 * STAGE_BYTES;
+    static constexpr int RING_BUDGET = 196608 - SPLIT_SLOTS * SPLIT_BYTES;
+    static constexpr int STAGES = (RING_BUDGET / STAGE_BYTES) > 8 ? 8 : (RING_BUDGET / STAGE_BYTES);
+    static constexpr int THREADS = 192 + (F32 ? CONVERTER_THREADS : 0);   // producer, MMA, 4 epilogue (, 4 converter) warps
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // two accumulator buffers
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SPLIT_SLOTS * SPLIT_BYTES + STAGING_BYTES +
+                                      1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int B_KSTEP_DESC = 16 * ROW_BYTES / 16;   // bf16 filter tile, N-major: 16 k-rows per k-step
     static_assert(B_COLS % 64 == 0 && BN % 16 == 0 && BN <= 256, "tile width");
     static_assert(TMEM_COLS <= 512 && (TMEM_COLS & (TMEM_COLS - 1)) == 0, "TMEM columns");
+    static_assert(STAGES >= 2 && STAGES <= 8, "ring depth");
 };
 
 // Static tile order: groups of 8 tile-rows, row index fastest inside a group, so that the
@@ -260,33 +326,43 @@ __device__ __forceinline__ void umma_bf16_cg2(uint32_t d_tmem, uint64_t a_desc, 
         "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+__device__ __forceinline__ void umma_tf32_cg2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 // Arrives (once the pair's MMAs issued so far have finished) on a barrier that may live in
 // either CTA of the pair; `cluster_bar` is a shared::cluster address.
 __device__ __forceinline__ void umma_commit_cg2(uint32_t cluster_bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar) : "memory");
 }
 
-template <int BN, int CG>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+template <int BN, int CG, bool F32>
+__global__ void __launch_bounds__(Cfg<BN, CG, F32>::THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_flt,
                const __grid_constant__ CUtensorMap map_out, const TcParams p) {
-    using C = Cfg<BN, CG>;
+    using C = Cfg<BN, CG, F32>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
 
     const uint32_t stages_addr = smem_base;
-    const uint32_t staging_addr = smem_base + C::STAGES * C::STAGE_BYTES;
-    uint8_t *staging_gen = smem_gen + C::STAGES * C::STAGE_BYTES;
+    const uint32_t split_addr = smem_base + C::STAGES * C::STAGE_BYTES;      // f32 only: hi/lo slots
+    const uint32_t staging_addr = split_addr + C::SPLIT_SLOTS * C::SPLIT_BYTES;
+    uint8_t *staging_gen = smem_gen + C::STAGES * C::STAGE_BYTES + C::SPLIT_SLOTS * C::SPLIT_BYTES;
     const uint32_t bars_addr = staging_addr + STAGING_BYTES;
     uint8_t *bars_gen = staging_gen + STAGING_BYTES;
-    // barrier block: full[STAGES] | empty[STAGES] | acc_full[2] | acc_empty[2] | tmem_ptr | abort
+    // barrier block: full[8] | empty[8] | split_full[2] | split_empty[2] | acc_full[2] | acc_empty[2] | tmem_ptr | abort
     auto full_bar = [&](int s) { return bars_addr + 8u * s; };
-    auto empty_bar = [&](int s) { return bars_addr + 8u * (C::STAGES + s); };
-    auto acc_full_bar = [&](int b) { return bars_addr + 8u * (2 * C::STAGES + b); };
-    auto acc_empty_bar = [&](int b) { return bars_addr + 8u * (2 * C::STAGES + 2 + b); };
-    volatile uint32_t *tmem_ptr_slot = reinterpret_cast<volatile uint32_t *>(bars_gen + 8 * (2 * C::STAGES + 4));
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_gen + 8 * (2 * C::STAGES + 4) + 4);
+    auto empty_bar = [&](int s) { return bars_addr + 8u * (8 + s); };
+    auto split_full_bar = [&](int s) { return bars_addr + 8u * (16 + s); };
+    auto split_empty_bar = [&](int s) { return bars_addr + 8u * (18 + s); };
+    auto acc_full_bar = [&](int b) { return bars_addr + 8u * (20 + b); };
+    auto acc_empty_bar = [&](int b) { return bars_addr + 8u * (22 + b); };
+    volatile uint32_t *tmem_ptr_slot = reinterpret_cast<volatile uint32_t *>(bars_gen + 8 * 24);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_gen + 8 * 24 + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // In a pair, CTA 0 (the leader) issues the MMAs; both CTAs produce and both run epilogues.
@@ -295,9 +371,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     const int num_groups = CG == 2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
-        // full: one arrive.expect_tx (by the leader's producer).  acc_empty: one arrive per epilogue
-        // warp of every CTA of the group.  empty / acc_full: one tcgen05.commit.
-        for (int s = 0; s < C::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        // full: one arrive.expect_tx by a producer.  empty: one tcgen05.commit (bf16) or one arrive per
+        // converter warp of this CTA (f32).  split_full: one arrive per converter warp of every CTA
+        // of the group.  split_empty / acc_full: one tcgen05.commit.  acc_empty: one arrive per
+        // epilogue warp of every CTA of the group.
+        for (int s = 0; s < C::STAGES; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), F32 ? CONVERTER_THREADS / 32 : 1);
+        }
+        for (int s = 0; s < C::SPLIT_SLOTS; ++s) {
+            mbar_init(split_full_bar(s), (CONVERTER_THREADS / 32) * CG);
+            mbar_init(split_empty_bar(s), 1);
+        }
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), 4 * CG); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -320,6 +405,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     const uint32_t tmem_base = *tmem_ptr_slot;
 
     const int num_tiles = p.num_m_tiles * p.num_n_tiles;   // tiles of (CG*128) x BN
+    // bf16 pairs count both CTAs' TMA bytes on the leader's barrier, which its MMA thread waits
+    // on.  f32 pairs signal each CTA's own barrier (its converter warps wait there) and the
+    // leader's MMA thread waits on the split barrier instead.
+    constexpr bool REMOTE_FULL = (CG == 2) && !F32;
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -346,9 +435,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     const uint32_t a_dst = stages_addr + s * C::STAGE_BYTES;
                     const uint32_t b_dst = a_dst + A_STAGE_BYTES;
                     const int tap = kb / p.kb_per_tap;
-                    const int c0 = (kb - tap * p.kb_per_tap) * BK;
+                    const int c0 = (kb - tap * p.kb_per_tap) * C::BK;
                     const int kh = tap / p.KW, kw = tap - kh * p.KW;
-                    if constexpr (CG == 1) {
+                    if constexpr (!REMOTE_FULL) {
                         const uint32_t bar = full_bar(s);
                         mbar_expect_tx(bar, C::STAGE_BYTES);
                         if (p.a_mode == 0) {
@@ -360,11 +449,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                                                (unsigned short)(kw * p.dw), (unsigned short)(kh * p.dh));
                         }
 #pragma unroll
-                        for (int j = 0; j < C::B_COLS / 64; ++j)
-                            tma_load_4d(b_dst + j * (BK * 128), &map_flt, bar, n0 + j * 64, c0, kw, kh);
+                        for (int j = 0; j < C::B_COLS / C::SUB_COLS; ++j)
+                            tma_load_4d(b_dst + j * C::SUB_BYTES, &map_flt, bar, n0 + j * C::SUB_COLS, c0, kw, kh);
                     } else {
-                        // both CTAs' bytes are counted on the leader's barrier, which its MMA thread waits
-                        // on; the leader alone arms it, for the pair's total (a remote arrive by the
+                        // the leader alone arms its barrier, for the pair's total (a remote arrive by the
                         // peer would order it after its own loads in flight and serialise the ring)
                         const uint32_t bar = map_to_cta(full_bar(s), 0);
                         if (cta_rank == 0) mbar_expect_tx(full_bar(s), CG * C::STAGE_BYTES);
@@ -377,8 +465,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                                                    (unsigned short)(kw * p.dw), (unsigned short)(kh * p.dh));
                         }
 #pragma unroll
-                        for (int j = 0; j < C::B_COLS / 64; ++j)
-                            tma_load_4d_cg2(b_dst + j * (BK * 128), &map_flt, bar, n0 + j * 64, c0, kw, kh);
+                        for (int j = 0; j < C::B_COLS / C::SUB_COLS; ++j)
+                            tma_load_4d_cg2(b_dst + j * C::SUB_BYTES, &map_flt, bar, n0 + j * C::SUB_COLS, c0, kw, kh);
                     }
                 }
             }
@@ -386,7 +474,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && cta_rank == 0) {
-            constexpr uint32_t idesc = make_idesc_bf16(BN, CG * BM);
+            constexpr uint32_t idesc = make_idesc(BN, CG * BM, F32);
+            auto mma = [&](uint32_t d, uint64_t ad, uint64_t bd, uint32_t acc) {
+                if constexpr (F32) {
+                    if constexpr (CG == 1) umma_tf32(d, ad, bd, idesc, acc); else umma_tf32_cg2(d, ad, bd, idesc, acc);
+                } else {
+                    if constexpr (CG == 1) umma_bf16(d, ad, bd, idesc, acc); else umma_bf16_cg2(d, ad, bd, idesc, acc);
+                }
+            };
             int it = 0, tl = 0;
             bool ok = true;
             for (int t = group_id; t < num_tiles && ok; t += num_groups, ++tl) {
@@ -395,30 +490,54 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
-                    const int s = it % C::STAGES;
-                    const uint32_t ph = (it / C::STAGES) & 1;
-                    if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_addr = stages_addr + s * C::STAGE_BYTES;
-                    const uint32_t b_addr = a_addr + A_STAGE_BYTES;
-                    // input tile, K-major: 8-row groups are 1024 B apart; a k-step of 16 bf16 is 32 B
-                    // inside the swizzled 128-byte row.
-                    const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024);
-                    // filter tile, N-major: 64-column sub-tiles are BK*128 B apart (leading offset),
-                    // 8-row k groups 1024 B apart (stride offset); a k-step of 16 rows is 2048 B.
-                    const uint64_t b_desc = make_smem_desc(b_addr, BK * 128, 1024);
+                    if constexpr (F32) {
+                        const int s = it & 1;
+                        if (!mbar_wait<CG == 2>(split_full_bar(s), (it >> 1) & 1, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        // slot: [input hi | input lo | filter hi | filter lo], all K-major: 8-row groups
+                        // 1024 B apart, a k-step of 8 f32 is 32 B inside the swizzled 128-byte row
+                        const uint32_t a_hi = split_addr + s * C::SPLIT_BYTES;
+                        const uint64_t ah = make_smem_desc(a_hi, 16, 1024);
+                        const uint64_t al = make_smem_desc(a_hi + A_STAGE_BYTES, 16, 1024);
+                        const uint64_t bh = make_smem_desc(a_hi + 2 * A_STAGE_BYTES, 16, 1024);
+                        const uint64_t bl = make_smem_desc(a_hi + 2 * A_STAGE_BYTES + C::B_STAGE_BYTES, 16, 1024);
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-                        if constexpr (CG == 1) umma_bf16(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc, acc);
-                        else umma_bf16_cg2(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc, acc);
-                    }
-                    // the stage is free (in every CTA of the group) once these MMAs have read it
-                    if constexpr (CG == 1) {
-                        umma_commit(empty_bar(s));
+                        for (int k = 0; k < K_STEPS; ++k) {
+                            const uint64_t o = (uint64_t)(k * 2);
+                            mma(d_tmem, al + o, bh + o, (kb > 0 || k > 0) ? 1u : 0u);   // small terms first
+                            mma(d_tmem, ah + o, bl + o, 1u);
+                            mma(d_tmem, ah + o, bh + o, 1u);
+                        }
+                        if constexpr (CG == 1) {
+                            umma_commit(split_empty_bar(s));
+                        } else {
+                            umma_commit_cg2(map_to_cta(split_empty_bar(s), 0));
+                            umma_commit_cg2(map_to_cta(split_empty_bar(s), 1));
+                        }
                     } else {
-                        umma_commit_cg2(map_to_cta(empty_bar(s), 0));
-                        umma_commit_cg2(map_to_cta(empty_bar(s), 1));
+                        const int s = it % C::STAGES;
+                        const uint32_t ph = (it / C::STAGES) & 1;
+                        if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a_addr = stages_addr + s * C::STAGE_BYTES;
+                        const uint32_t b_addr = a_addr + A_STAGE_BYTES;
+                        // input tile, K-major: 8-row groups are 1024 B apart; a k-step of 16 bf16 is 32 B
+                        // inside the swizzled 128-byte row.
+                        const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024);
+                        // filter tile, N-major: 64-column sub-tiles are SUB_BYTES apart (leading offset),
+                        // 8-row k groups 1024 B apart (stride offset); a k-step of 16 rows is 2048 B.
+                        const uint64_t b_desc = make_smem_desc(b_addr, C::SUB_BYTES, 1024);
+#pragma unroll
+                        for (int k = 0; k < K_STEPS; ++k)
+                            mma(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * C::B_KSTEP_DESC),
+                                (kb > 0 || k > 0) ? 1u : 0u);
+                        // the stage is free (in every CTA of the group) once these MMAs have read it
+                        if constexpr (CG == 1) {
+                            umma_commit(empty_bar(s));
+                        } else {
+                            umma_commit_cg2(map_to_cta(empty_bar(s), 0));
+                            umma_commit_cg2(map_to_cta(empty_bar(s), 1));
+                        }
                     }
                 }
                 if (ok) {
@@ -427,6 +546,82 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     } else {
                         umma_commit_cg2(map_to_cta(acc_full_bar(buf), 0));
                         umma_commit_cg2(map_to_cta(acc_full_bar(buf), 1));
+                    }
+                }
+            }
+        }
+    } else if (warp >= 6) {
+        // ------------------------------------------------------------ converter (f32 only)
+        if constexpr (F32) {
+            const int cw = warp - 6;                       // converter warp 0..3
+            const int ct = (int)threadIdx.x - 192;         // converter thread 0..127
+            int it = 0;
+            bool ok = true;
+            for (int t = group_id; t < num_tiles && ok; t += num_groups) {
+                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                    const int r = it % C::STAGES, s = it & 1;
+                    if (!mbar_wait(full_bar(r), (it / C::STAGES) & 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait<CG == 2>(split_empty_bar(s), ((it >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint8_t *raw = smem_gen + r * C::STAGE_BYTES;
+                    uint8_t *slot = smem_gen + C::STAGES * C::STAGE_BYTES + s * C::SPLIT_BYTES;
+                    // input tile: elementwise, the swizzled placement of the elements is kept
+                    {
+                        const uint4 *src = reinterpret_cast<const uint4 *>(raw) + ct;
+                        uint4 *hi = reinterpret_cast<uint4 *>(slot) + ct;
+                        uint4 *lo = hi + A_STAGE_BYTES / 16;
+                        constexpr int N = A_STAGE_BYTES / 16 / CONVERTER_THREADS;   // 8 chunks per thread
+                        uint4 v[N];
+#pragma unroll
+                        for (int i = 0; i < N; ++i) v[i] = src[i * CONVERTER_THREADS];
+#pragma unroll
+                        for (int i = 0; i < N; ++i) {
+                            uint4 h, l;
+                            h.x = split_hi(v[i].x); l.x = split_lo(v[i].x, h.x);
+                            h.y = split_hi(v[i].y); l.y = split_lo(v[i].y, h.y);
+                            h.z = split_hi(v[i].z); l.z = split_lo(v[i].z, h.z);
+                            h.w = split_hi(v[i].w); l.w = split_lo(v[i].w, h.w);
+                            hi[i * CONVERTER_THREADS] = h;
+                            lo[i * CONVERTER_THREADS] = l;
+                        }
+                    }
+                    // filter tile: raw sub-tiles are [32 k][32 f] rows of 128 B, not swizzled; the split
+                    // tiles are K-major, [f][32 k] rows of 128 B in 8-row groups with the 128-byte swizzle
+                    // (16-byte chunk c of row f sits at chunk c ^ (f & 7)).  A unit is half a sub-tile
+                    // (16 k); lane = f reads a column (one 128-byte row per load across the warp) and
+                    // writes 4 chunks of its row.
+                    {
+                        const float *braw = reinterpret_cast<const float *>(raw + A_STAGE_BYTES);
+                        uint8_t *bhi = slot + 2 * A_STAGE_BYTES;
+                        uint8_t *blo = bhi + C::B_STAGE_BYTES;
+                        constexpr int UNITS = 2 * C::B_COLS / 32;
+#pragma unroll
+                        for (int u = cw; u < UNITS; u += CONVERTER_THREADS / 32) {
+                            const int j = u >> 1, half = u & 1;
+                            const float *col = braw + j * (C::SUB_BYTES / 4) + half * 16 * 32 + lane;
+                            uint32_t x[16];
+#pragma unroll
+                            for (int k = 0; k < 16; ++k) x[k] = __float_as_uint(col[k * 32]);
+                            const int f = j * 32 + lane;
+                            const int row_off = (f >> 3) * 1024 + (f & 7) * 128;
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                uint4 h, l;
+                                h.x = split_hi(x[4 * c]);     l.x = split_lo(x[4 * c], h.x);
+                                h.y = split_hi(x[4 * c + 1]); l.y = split_lo(x[4 * c + 1], h.y);
+                                h.z = split_hi(x[4 * c + 2]); l.z = split_lo(x[4 * c + 2], h.z);
+                                h.w = split_hi(x[4 * c + 3]); l.w = split_lo(x[4 * c + 3], h.w);
+                                const int off = row_off + (((half * 4 + c) ^ (f & 7)) << 4);
+                                *reinterpret_cast<uint4 *>(bhi + off) = h;
+                                *reinterpret_cast<uint4 *>(blo + off) = l;
+                            }
+                        }
+                    }
+                    fence_async_smem();     // generic-proxy writes -> visible to the tensor core's reads
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(empty_bar(r));          // the raw stage may be refilled
+                        if constexpr (CG == 1) mbar_arrive(split_full_bar(s));
+                        else mbar_arrive_cluster(map_to_cta(split_full_bar(s), 0));
                     }
                 }
             }
@@ -515,7 +710,7 @@ struct Driver {
     EncodeIm2colFn im2col = nullptr;
     int num_sms = 0;
     int device = -1;
-    bool attr_set[8] = {};
+    bool attr_set[16] = {};
     bool ok = false;
 };
 std::mutex g_mu;
@@ -546,18 +741,23 @@ bool init_driver() {
 
 inline bool mult(int64_t v, int64_t q) { return v % q == 0; }
 
-struct Variant { int bn, cg; double step_cost; };
-// Relative cost of one 16-deep k-step of a tile per variant (measured on large problems):
-// narrow tiles pay more shared-memory traffic per flop, CTA pairs stage the filter once.
-constexpr Variant kVariants[] = {{64, 1, 80.0}, {128, 1, 102.0}, {256, 1, 128.0}, {128, 2, 95.0}, {256, 2, 120.0}};
+struct Variant { int bn, cg; double step_cost, step_cost_f32; };
+// Relative cost of one k-block of a tile per variant.  bf16: measured on large problems; narrow
+// tiles pay more shared-memory traffic per flop, CTA pairs stage the filter once.  f32: the
+// shared-memory cycles of one k-block (TMA fill, hi/lo split, operand reads of the 12 MMAs).
+constexpr Variant kVariants[] = {{64, 1, 80.0, 1344.0}, {128, 1, 102.0, 1792.0}, {256, 1, 128.0, 2688.0},
+                                 {128, 2, 95.0, 1344.0}, {256, 2, 120.0, 1792.0}};
 constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
 
-template <int BN, int CG>
+template <int BN, int CG, bool F32>
 sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUtensorMap &mo, TcParams tp, int M, int N,
                          int slot, cudaStream_t stream) {
-    using C = Cfg<BN, CG>;
+  if constexpr (F32 && BN == 256 && CG == 1) {
+    return SG_ERR_INTERNAL;   // the split slots of a 128 x 256 f32 tile do not fit beside a TMA ring
+  } else {
+    using C = Cfg<BN, CG, F32>;
     if (!g_drv.attr_set[slot]) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, CG, F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
             return SG_ERR_CUDA;
         g_drv.attr_set[slot] = true;
     }
@@ -568,7 +768,7 @@ sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUt
     const int grid = CG * (tiles < groups ? tiles : groups);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
-    cfg.blockDim = dim3(NUM_THREADS, 1, 1);
+    cfg.blockDim = dim3(C::THREADS, 1, 1);
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -578,9 +778,10 @@ sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUt
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<BN, CG>, mi, mf, mo, tp);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<BN, CG, F32>, mi, mf, mo, tp);
     count_launch();
     return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
+  }
 }
 
 }  // namespace
@@ -588,8 +789,10 @@ sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUt
 sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float *O, cudaStream_t stream) {
     // ---- layout rules of the TMA descriptors (bytes): unit inner stride, 16-byte aligned
     //      bases and pitches; output rows uniformly strided so that O is one 2-D matrix ----
-    if (!p.in_bf16) return SG_ERR_UNSUPPORTED;
-    const int64_t es = 2;
+    const bool f32 = !p.in_bf16;
+    const int64_t es = f32 ? 4 : 2;
+    const int BK = ROW_BYTES / (int)es;          // elements per k-block
+    const CUtensorMapDataType in_type = f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     if (p.i_c != 1 || p.k_f != 1 || p.o_f != 1) return SG_ERR_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(In) % 16 || reinterpret_cast<uintptr_t>(Flt) % 16 ||
         reinterpret_cast<uintptr_t>(O) % 16) return SG_ERR_UNSUPPORTED;
@@ -627,8 +830,8 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         tp.a_mode = 0;
         cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)p.M};
         cuuint64_t strides[1] = {(cuuint64_t)(p.i_w * es)};
-        cuuint32_t box[2] = {BK, BM};
-        r = g_drv.tiled(&map_in, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(In), dims, strides, box, ones,
+        cuuint32_t box[2] = {(cuuint32_t)BK, BM};
+        r = g_drv.tiled(&map_in, in_type, 2, const_cast<void *>(In), dims, strides, box, ones,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
@@ -651,7 +854,7 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
             cuuint64_t strides[2] = {(cuuint64_t)(p.i_w * es), (cuuint64_t)((p.batch > 1 ? p.i_n : used_w * p.i_w) * es)};
             int lower[1] = {0}, upper[1] = {(int)-span_w};
             cuuint32_t trav[3] = {1, (cuuint32_t)p.sw, 1};
-            r = g_drv.im2col(&map_in, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(In), dims, strides, lower,
+            r = g_drv.im2col(&map_in, in_type, 3, const_cast<void *>(In), dims, strides, lower,
                              upper, BK, BM, trav, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         } else {
@@ -663,21 +866,24 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
                                      (cuuint64_t)((p.batch > 1 ? p.i_n : used_h * p.i_h) * es)};
             int lower[2] = {0, 0}, upper[2] = {(int)-span_w, (int)-span_h};
             cuuint32_t trav[4] = {1, (cuuint32_t)p.sw, (cuuint32_t)p.sh, 1};
-            r = g_drv.im2col(&map_in, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(In), dims, strides, lower,
+            r = g_drv.im2col(&map_in, in_type, 4, const_cast<void *>(In), dims, strides, lower,
                              upper, BK, BM, trav, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         }
         if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
     }
-    // ---- filter operand: 4-D {f, c, kw, kh}, one 64 x 64 box per load ----
+    // ---- filter operand: 4-D {f, c, kw, kh}, one sub-tile per load ----
     {
         cuuint64_t dims[4] = {(cuuint64_t)p.N, (cuuint64_t)p.C, (cuuint64_t)p.KW, (cuuint64_t)p.KH};
         int64_t s_kw = p.KW > 1 ? p.k_kw : (int64_t)p.C * p.k_c;
         int64_t s_kh = p.KH > 1 ? p.k_kh : (int64_t)p.KW * s_kw;
         cuuint64_t strides[3] = {(cuuint64_t)(p.k_c * es), (cuuint64_t)(s_kw * es), (cuuint64_t)(s_kh * es)};
-        cuuint32_t box[4] = {64, BK, 1, 1};
-        r = g_drv.tiled(&map_flt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(Flt), dims, strides, box, ones,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+        cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)BK, 1, 1};   // one sub-tile: a 128-byte row of columns x BK k-rows
+        // bf16 sub-tiles are consumed by the tensor core as they land (128-byte swizzle); f32
+        // sub-tiles are read by the converter warps, one 128-byte row per load: no swizzle
+        r = g_drv.tiled(&map_flt, in_type, 4, const_cast<void *>(Flt), dims, strides, box, ones,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, f32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
     }
@@ -697,31 +903,38 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     int pick = -1;
     if (g_bn_override > 0) {
         for (int i = 0; i < kNumVariants; ++i)
-            if (kVariants[i].bn == g_bn_override && kVariants[i].cg == (g_cg_override > 0 ? g_cg_override : 1)) pick = i;
+            if (kVariants[i].bn == g_bn_override && kVariants[i].cg == (g_cg_override > 0 ? g_cg_override : 1) &&
+                !(f32 && kVariants[i].bn == 256 && kVariants[i].cg == 1)) pick = i;
     }
     for (int pass = 0; pass < 2 && pick < 0; ++pass) {   // pass 1 drops a forced group size that does not fit
         double best = 1e300;
         for (int i = 0; i < kNumVariants; ++i) {
             const Variant &v = kVariants[i];
             if (pass == 0 && g_cg_override > 0 && v.cg != g_cg_override) continue;
+            if (f32 && v.bn == 256 && v.cg == 1) continue;       // not built (shared-memory budget)
             if (v.bn > 64 && v.bn / 2 >= p.N) continue;          // at most half of the tile would be used
             if (v.cg == 2 && p.M <= BM) continue;                // the second CTA would have no rows
             int64_t tiles = (int64_t)((p.M + v.cg * BM - 1) / (v.cg * BM)) * ((p.N + v.bn - 1) / v.bn);
             int64_t groups = g_drv.num_sms / v.cg;
             int64_t waves = (tiles + groups - 1) / groups;
             // a pair pays a fixed price (cluster launch, cross-CTA signalling) worth ~6 k-blocks
-            double cost = (double)waves * tp.num_kb * v.step_cost + (v.cg == 2 ? 760.0 : 0.0);
+            double cost = (double)waves * tp.num_kb * (f32 ? v.step_cost_f32 : v.step_cost) + (v.cg == 2 ? (f32 ? 6000.0 : 760.0) : 0.0);
             if (cost < best) { best = cost; pick = i; }
         }
     }
     if (pick < 0) return SG_ERR_INTERNAL;
+    const int slot = pick + (f32 ? kNumVariants : 0);
+#define SG_LAUNCH(BN_, CG_)                                                                              \
+    (f32 ? launch_variant<BN_, CG_, true>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)          \
+         : launch_variant<BN_, CG_, false>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream))
     switch (pick) {
-        case 0: return launch_variant<64, 1>(map_in, map_flt, map_out, tp, p.M, p.N, 0, stream);
-        case 1: return launch_variant<128, 1>(map_in, map_flt, map_out, tp, p.M, p.N, 1, stream);
-        case 2: return launch_variant<256, 1>(map_in, map_flt, map_out, tp, p.M, p.N, 2, stream);
-        case 3: return launch_variant<128, 2>(map_in, map_flt, map_out, tp, p.M, p.N, 3, stream);
-        default: return launch_variant<256, 2>(map_in, map_flt, map_out, tp, p.M, p.N, 4, stream);
+        case 0: return SG_LAUNCH(64, 1);
+        case 1: return SG_LAUNCH(128, 1);
+        case 2: return SG_LAUNCH(256, 1);
+        case 3: return SG_LAUNCH(128, 2);
+        default: return SG_LAUNCH(256, 2);
     }
+#undef SG_LAUNCH
 }
 
 sg_status tensor_read_status(cudaStream_t stream) {

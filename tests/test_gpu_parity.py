@@ -42,11 +42,22 @@ def run_matmul(M, N, K, dtype, family=None, accumulate=False, dist="uniform", se
 
 # ------------------------------------------------------------------ config 1: matmul 128^3 f32
 
+# f32 inputs on the tensor-core path are three tf32 products per term (hi*hi + hi*lo + lo*hi):
+# the result must stay at f32 accuracy, far inside the parity bound.
+F32_TENSOR_RATIO = 4e-6
+
+
 @pytest.mark.parametrize("accumulate", [False, True])
-def test_c1_matmul_128_f32(accumulate):
-    C, want, S = run_matmul(128, 128, 128, "f32", accumulate=accumulate, seed=SEED + 0)
-    assert sg.sg_last_kernel() == FFMA
+@pytest.mark.parametrize("family", [FFMA, TENSOR])
+def test_c1_matmul_128_f32(accumulate, family):
+    C, want, S = run_matmul(128, 128, 128, "f32", family=family, accumulate=accumulate, seed=SEED + 0)
+    assert sg.sg_last_kernel() == family
     assert_within_bound(C, want, S, "matmul 128^3 f32")
+
+
+def test_c1_default_selection_is_tensor_path():
+    C, want, S = run_matmul(128, 128, 128, "f32", seed=SEED + 0)
+    assert sg.sg_last_kernel() == TENSOR
 
 
 # ------------------------------------------------------------------ matmul, both kernel families
@@ -64,6 +75,18 @@ def test_matmul_bf16_shapes(M, N, K, family):
 def test_matmul_f32_shapes(M, N, K):
     C, want, S = run_matmul(M, N, K, "f32", seed=SEED + 1)
     assert_within_bound(C, want, S, f"matmul f32 {M}x{N}x{K}")
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (256, 256, 256), (300, 200, 136), (129, 72, 8), (1, 8, 8),
+                                   (515, 264, 1000), (128, 64, 4096), (384, 520, 72), (1024, 768, 36)])
+def test_matmul_f32_tensor_path_keeps_f32_accuracy(M, N, K):
+    C, want, S = run_matmul(M, N, K, "f32", family=TENSOR, seed=SEED + 1)
+    assert sg.sg_last_kernel() == TENSOR
+    ratio = assert_within_bound(C, want, S, f"matmul f32 3xTF32 {M}x{N}x{K}")
+    assert ratio < F32_TENSOR_RATIO, ratio
+    # normal-distributed values exercise every exponent, not just [-1, 1)
+    C, want, S = run_matmul(M, N, K, "f32", family=TENSOR, dist="normal", seed=SEED + 9)
+    assert assert_within_bound(C, want, S, "normal inputs") < F32_TENSOR_RATIO
 
 
 @pytest.mark.parametrize("bn,cg", [("64", "1"), ("128", "1"), ("256", "1"), ("128", "2"), ("256", "2")])
@@ -85,7 +108,18 @@ def test_tensor_path_every_tile_variant(bn, cg):
         "O, want, S = t.run_conv2d(5, 30, 27, 72, 3, 3, 136, (1, 1), (1, 1), 'bf16', family=t.TENSOR, seed=t.SEED + 7);"
         "assert_within_bound(O, want, S, 'conv2d');"
         "O, want, S = t.run_conv1d(3, 700, 64, 3, 200, 2, 2, 'bf16', family=t.TENSOR, seed=t.SEED + 7);"
-        "assert_within_bound(O, want, S, 'conv1d'); t.sg.sg_check(); print('child-ok')"
+        "assert_within_bound(O, want, S, 'conv1d');"
+        "C, want, S = t.run_matmul(400, 520, 200, 'f32', family=t.TENSOR, seed=t.SEED + 7);"
+        "assert assert_within_bound(C, want, S, 'f32 ragged') < t.F32_TENSOR_RATIO;"
+        "C, want, S = t.run_matmul(400, 520, 200, 'f32', family=t.TENSOR, accumulate=True, seed=t.SEED + 7);"
+        "assert_within_bound(C, want, S, 'f32 ragged acc');"
+        "C, want, S = t.run_matmul(2048 + 136, 2304, 164, 'f32', family=t.TENSOR, seed=t.SEED + 7);"
+        "assert assert_within_bound(C, want, S, 'f32 many tiles per CTA') < t.F32_TENSOR_RATIO;"
+        "O, want, S = t.run_conv2d(5, 30, 27, 72, 3, 3, 136, (1, 1), (1, 1), 'f32', family=t.TENSOR, seed=t.SEED + 7);"
+        "assert assert_within_bound(O, want, S, 'f32 conv2d') < t.F32_TENSOR_RATIO;"
+        "O, want, S = t.run_conv1d(3, 700, 64, 3, 200, 2, 2, 'f32', family=t.TENSOR, seed=t.SEED + 7);"
+        "assert assert_within_bound(O, want, S, 'f32 conv1d') < t.F32_TENSOR_RATIO;"
+        " t.sg.sg_check(); print('child-ok')"
     )
     env = dict(os.environ, SG_TC_BN=bn, SG_TC_CG=cg)
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -94,10 +128,12 @@ def test_tensor_path_every_tile_variant(bn, cg):
 
 
 @pytest.mark.parametrize("family", [FFMA, TENSOR])
-def test_matmul_integer_inputs_are_bit_exact(family):
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_matmul_integer_inputs_are_bit_exact(family, dtype):
     # integers in [-2,2]: every product and partial sum is exact in f32, so every summation
-    # order gives the same bits as the f64 oracle.
-    C, want, S = run_matmul(256, 192, 320, "bf16", family=family, dist="ints", seed=SEED + 2)
+    # order (and the hi/lo split of the f32 tensor-core path) gives the bits of the f64 oracle.
+    C, want, S = run_matmul(256, 192, 320, dtype, family=family, dist="ints", seed=SEED + 2)
+    assert sg.sg_last_kernel() == family
     assert np.array_equal(C.cpu().numpy().astype(np.float64), want)
 
 
@@ -225,10 +261,13 @@ def run_conv2d(N, Ho, Wo, C, KH, KW, F, st, dl, dtype, family=None, accumulate=F
     return O, want, S
 
 
-def test_c3_conv1d_f32_full():
+@pytest.mark.parametrize("family", [FFMA, TENSOR])
+def test_c3_conv1d_f32_full(family):
     # config 3: N=32, W=1026, C=64, KW=3, F=128, stride 1, f32, uniform[-1,1)
-    O, want, S = run_conv1d(32, 1024, 64, 3, 128, 1, 1, "f32", seed=SEED + 2)
-    assert_within_bound(O, want, S, "conv1d config 3")
+    O, want, S = run_conv1d(32, 1024, 64, 3, 128, 1, 1, "f32", family=family, seed=SEED + 2)
+    assert sg.sg_last_kernel() == family
+    ratio = assert_within_bound(O, want, S, "conv1d config 3")
+    assert ratio < F32_TENSOR_RATIO
 
 
 def test_c4_conv2d_bf16_full():
@@ -266,6 +305,24 @@ def test_conv2d_bf16(family, N, Ho, Wo, C, KH, KW, F, st, dl):
 def test_conv2d_f32(N, Ho, Wo, C, KH, KW, F, st, dl):
     O, want, S = run_conv2d(N, Ho, Wo, C, KH, KW, F, st, dl, "f32", seed=SEED + 6)
     assert_within_bound(O, want, S, "conv2d f32")
+
+
+@pytest.mark.parametrize("N,Ho,Wo,C,KH,KW,F,st,dl", [(3, 20, 20, 64, 3, 3, 128, (1, 1), (1, 1)),
+                                                      (4, 13, 17, 72, 2, 3, 40, (1, 1), (1, 1)),
+                                                      (2, 20, 19, 64, 3, 3, 64, (2, 2), (1, 1)),
+                                                      (1, 55, 55, 32, 3, 3, 64, (2, 2), (2, 2))])
+def test_conv2d_f32_tensor_path(N, Ho, Wo, C, KH, KW, F, st, dl):
+    O, want, S = run_conv2d(N, Ho, Wo, C, KH, KW, F, st, dl, "f32", family=TENSOR, seed=SEED + 6)
+    assert sg.sg_last_kernel() == TENSOR
+    assert assert_within_bound(O, want, S, "conv2d f32 3xTF32") < F32_TENSOR_RATIO
+
+
+@pytest.mark.parametrize("N,Wo,C,KW,F,sw,dw", [(4, 300, 64, 3, 128, 1, 1), (3, 333, 72, 5, 40, 1, 1),
+                                               (2, 500, 64, 3, 64, 2, 1), (5, 97, 200, 2, 136, 3, 2)])
+def test_conv1d_f32_tensor_path(N, Wo, C, KW, F, sw, dw):
+    O, want, S = run_conv1d(N, Wo, C, KW, F, sw, dw, "f32", family=TENSOR, seed=SEED + 4)
+    assert sg.sg_last_kernel() == TENSOR
+    assert assert_within_bound(O, want, S, "conv1d f32 3xTF32") < F32_TENSOR_RATIO
 
 
 @pytest.mark.parametrize("family", [FFMA, TENSOR])
@@ -343,8 +400,8 @@ def test_full_size_bf16_matmul_sampled(M, N, K, cfg):
     assert torch.allclose(C.double().sum(dim=1), rs, rtol=1e-6, atol=1e-2 * K ** 0.5)
 
 
-def test_full_size_f32_matmul_sampled():
-    M = N = K = 1024
+@pytest.mark.parametrize("M,N,K", [(1024, 1024, 1024), (4096, 4096, 4096), (256, 4096, 2048)])
+def test_full_size_f32_matmul_sampled(M, N, K):
     A, a = operand((M, K), SEED + 1, 1, "uniform", "f32")
     B, b = operand((K, N), SEED + 1, 2, "uniform", "f32")
     C = torch.full((M, N), float("nan"), device="cuda")
@@ -353,5 +410,6 @@ def test_full_size_f32_matmul_sampled():
     pm, pn = sample_points(M, N, 4096, 98)
     want, S = ref.matmul_points(a, b, pm, pn)
     got = C[torch.from_numpy(pm).cuda(), torch.from_numpy(pn).cuda()]
-    assert_within_bound(got, want, S, "sampled f32 1024^3")
+    assert sg.sg_last_kernel() == TENSOR
+    assert assert_within_bound(got, want, S, f"sampled f32 {M}x{N}x{K}") < F32_TENSOR_RATIO
     assert not torch.isnan(C).any()
