@@ -23,7 +23,7 @@
 //
 // f32 inputs run on the same pipeline as three tf32 products per k-step ("3xTF32"): the TMA
 // writes the raw f32 tiles into its ring, four converter warps split every element x into two
-// tf32 values hi = rn(x) and lo = rn(x - hi) and write them to a second ring of two slots
+// values hi = x rounded to tf32 and lo = x - hi and write them to a second ring of two slots
 // (transposing the filter tile to K-major on the way, which kind::tf32 needs), and the MMA
 // thread accumulates lo*hi + hi*lo + hi*hi in f32: the dropped terms are below 2^-21 |a*b|, so
 // f32 accuracy is kept.  Raw tiles are 128 rows x 32 f32 (input) and 32 k-rows x 32 f32
@@ -45,7 +45,7 @@ constexpr int BM = 128;           // rows of an output tile = lanes of TMEM = M 
 constexpr int ROW_BYTES = 128;    // one k-block = one 128-byte swizzle row: 64 bf16 or 32 f32
 constexpr int K_STEPS = 4;        // tcgen05.mma per k-block and product: 32 bytes of k each
 constexpr int A_STAGE_BYTES = BM * ROW_BYTES;
-constexpr int CONVERTER_THREADS = 128;        // f32 path: 4 warps splitting tiles into hi and lo
+constexpr int CONVERTER_THREADS = 256;        // f32 path: 8 warps splitting tiles into hi and lo
 constexpr int STAGING_BYTES = 4 * 2 * 4096;   // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
 constexpr long long WAIT_BUDGET_CYCLES = 2000000000LL;   // ~1 s: far beyond any legitimate wait
 
@@ -216,23 +216,29 @@ __host__ __device__ constexpr uint32_t make_idesc(int n, int m, bool tf32) {
          | ((uint32_t)(m >> 4) << 24);     // M / 16 (128 for one CTA, 256 for a pair)
 }
 
-// 3xTF32 split of an f32 word x into two tf32 values (low 13 mantissa bits zero, so whatever
-// rounding the tensor core applies to its inputs leaves them unchanged): hi = x rounded to
-// nearest, lo = (x - hi) rounded to nearest; x - hi is exact in f32 and |x - hi - lo| <=
-// 2^-22 |x|.  Infinities and NaNs stay in hi alone; a finite x that would round up to
-// infinity is truncated instead.
-__device__ __forceinline__ uint32_t cvt_rna_tf32(float x) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return r;
-}
-__device__ __forceinline__ uint32_t split_hi(uint32_t x) {
-    const uint32_t h = cvt_rna_tf32(__uint_as_float(x));
-    return (h & 0x7F800000u) == 0x7F800000u ? (x & 0xFFFFE000u) : h;
-}
-__device__ __forceinline__ uint32_t split_lo(uint32_t x, uint32_t hi) {
-    const uint32_t l = cvt_rna_tf32(__uint_as_float(x) - __uint_as_float(hi));
-    return (x & 0x7F800000u) == 0x7F800000u ? 0u : l;
+// 3xTF32 split of four f32 words.  hi = x rounded to the nearest tf32 value (10 mantissa bits;
+// done on the bit pattern: add half an ulp, clear the low 13 bits); x - hi is exact in f32 and
+// lo is that difference rounded to tf32 the same way, so x - hi - lo is below 2^-22 |x|.  The
+// low bits of hi and lo are zero, so whatever rounding the tensor core applies to its inputs
+// leaves them unchanged.  Words of magnitude >= 2^127 (where rounding up
+// could reach infinity), infinities and NaNs take a slow path: hi truncated, lo = 0 unless
+// finite.
+__device__ __forceinline__ void split4(const uint4 v, uint4 &h, uint4 &l) {
+    const float fx = __uint_as_float(v.x), fy = __uint_as_float(v.y), fz = __uint_as_float(v.z), fw = __uint_as_float(v.w);
+    const float big = fmaxf(fmaxf(fabsf(fx), fabsf(fy)), fmaxf(fabsf(fz), fabsf(fw)));
+    if (big < 1.7014118e38f) {
+        h.x = (v.x + 0x1000u) & 0xFFFFE000u; l.x = (__float_as_uint(fx - __uint_as_float(h.x)) + 0x1000u) & 0xFFFFE000u;
+        h.y = (v.y + 0x1000u) & 0xFFFFE000u; l.y = (__float_as_uint(fy - __uint_as_float(h.y)) + 0x1000u) & 0xFFFFE000u;
+        h.z = (v.z + 0x1000u) & 0xFFFFE000u; l.z = (__float_as_uint(fz - __uint_as_float(h.z)) + 0x1000u) & 0xFFFFE000u;
+        h.w = (v.w + 0x1000u) & 0xFFFFE000u; l.w = (__float_as_uint(fw - __uint_as_float(h.w)) + 0x1000u) & 0xFFFFE000u;
+    } else {
+        auto one = [](uint32_t x, uint32_t &hi, uint32_t &lo) {
+            hi = x & 0xFFFFE000u;
+            const float d = __uint_as_float(x) - __uint_as_float(hi);
+            lo = (x & 0x7F800000u) == 0x7F800000u ? 0u : __float_as_uint(d);
+        };
+        one(v.x, h.x, l.x); one(v.y, h.y, l.y); one(v.z, h.z, l.z); one(v.w, h.w, l.w);
+    }
 }
 
 template <int BN, int CG, bool F32>
@@ -255,7 +261,7 @@ struct Cfg {
     static constexpr int SPLIT_BYTES = 2 * STAGE_BYTES;
     static constexpr int RING_BUDGET = 196608 - SPLIT_SLOTS * SPLIT_BYTES;
     static constexpr int STAGES = (RING_BUDGET / STAGE_BYTES) > 8 ? 8 : (RING_BUDGET / STAGE_BYTES);
-    static constexpr int THREADS = 192 + (F32 ? CONVERTER_THREADS : 0);   // producer, MMA, 4 epilogue (, 4 converter) warps
+    static constexpr int THREADS = 192 + (F32 ? CONVERTER_THREADS : 0);   // producer, MMA, 4 epilogue (, 8 converter) warps
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // two accumulator buffers
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SPLIT_SLOTS * SPLIT_BYTES + STAGING_BYTES +
                                       1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -289,8 +295,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
+// Arrive on a barrier of another CTA of the cluster.  Default semantics (release at CTA scope):
+// what the arriving thread wrote before goes to its own CTA's shared memory, which the
+// tensor core reads after a proxy fence; a cluster-scope release costs a full memory barrier
+// per arrive (measured: 1.6x on the whole f32 kernel) and orders nothing more that is needed.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -553,8 +563,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     } else if (warp >= 6) {
         // ------------------------------------------------------------ converter (f32 only)
         if constexpr (F32) {
-            const int cw = warp - 6;                       // converter warp 0..3
-            const int ct = (int)threadIdx.x - 192;         // converter thread 0..127
+            const int cw = warp - 6;                       // converter warp
+            const int ct = (int)threadIdx.x - 192;         // converter thread
             int it = 0;
             bool ok = true;
             for (int t = group_id; t < num_tiles && ok; t += num_groups) {
@@ -569,48 +579,42 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                         const uint4 *src = reinterpret_cast<const uint4 *>(raw) + ct;
                         uint4 *hi = reinterpret_cast<uint4 *>(slot) + ct;
                         uint4 *lo = hi + A_STAGE_BYTES / 16;
-                        constexpr int N = A_STAGE_BYTES / 16 / CONVERTER_THREADS;   // 8 chunks per thread
+                        constexpr int N = A_STAGE_BYTES / 16 / CONVERTER_THREADS;   // 16-byte chunks per thread
                         uint4 v[N];
 #pragma unroll
                         for (int i = 0; i < N; ++i) v[i] = src[i * CONVERTER_THREADS];
 #pragma unroll
                         for (int i = 0; i < N; ++i) {
                             uint4 h, l;
-                            h.x = split_hi(v[i].x); l.x = split_lo(v[i].x, h.x);
-                            h.y = split_hi(v[i].y); l.y = split_lo(v[i].y, h.y);
-                            h.z = split_hi(v[i].z); l.z = split_lo(v[i].z, h.z);
-                            h.w = split_hi(v[i].w); l.w = split_lo(v[i].w, h.w);
+                            split4(v[i], h, l);
                             hi[i * CONVERTER_THREADS] = h;
                             lo[i * CONVERTER_THREADS] = l;
                         }
                     }
                     // filter tile: raw sub-tiles are [32 k][32 f] rows of 128 B, not swizzled; the split
                     // tiles are K-major, [f][32 k] rows of 128 B in 8-row groups with the 128-byte swizzle
-                    // (16-byte chunk c of row f sits at chunk c ^ (f & 7)).  A unit is half a sub-tile
-                    // (16 k); lane = f reads a column (one 128-byte row per load across the warp) and
-                    // writes 4 chunks of its row.
+                    // (16-byte chunk c of row f sits at chunk c ^ (f & 7)).  A unit is a quarter of a
+                    // sub-tile (8 k); lane = f reads a column (one 128-byte row per load across the warp)
+                    // and writes 2 chunks of its row.
                     {
                         const float *braw = reinterpret_cast<const float *>(raw + A_STAGE_BYTES);
                         uint8_t *bhi = slot + 2 * A_STAGE_BYTES;
                         uint8_t *blo = bhi + C::B_STAGE_BYTES;
-                        constexpr int UNITS = 2 * C::B_COLS / 32;
+                        constexpr int UNITS = 4 * C::B_COLS / 32;
 #pragma unroll
                         for (int u = cw; u < UNITS; u += CONVERTER_THREADS / 32) {
-                            const int j = u >> 1, half = u & 1;
-                            const float *col = braw + j * (C::SUB_BYTES / 4) + half * 16 * 32 + lane;
-                            uint32_t x[16];
+                            const int j = u >> 2, quarter = u & 3;
+                            const float *col = braw + j * (C::SUB_BYTES / 4) + quarter * 8 * 32 + lane;
+                            uint32_t x[8];
 #pragma unroll
-                            for (int k = 0; k < 16; ++k) x[k] = __float_as_uint(col[k * 32]);
+                            for (int k = 0; k < 8; ++k) x[k] = __float_as_uint(col[k * 32]);
                             const int f = j * 32 + lane;
                             const int row_off = (f >> 3) * 1024 + (f & 7) * 128;
 #pragma unroll
-                            for (int c = 0; c < 4; ++c) {
+                            for (int c = 0; c < 2; ++c) {
                                 uint4 h, l;
-                                h.x = split_hi(x[4 * c]);     l.x = split_lo(x[4 * c], h.x);
-                                h.y = split_hi(x[4 * c + 1]); l.y = split_lo(x[4 * c + 1], h.y);
-                                h.z = split_hi(x[4 * c + 2]); l.z = split_lo(x[4 * c + 2], h.z);
-                                h.w = split_hi(x[4 * c + 3]); l.w = split_lo(x[4 * c + 3], h.w);
-                                const int off = row_off + (((half * 4 + c) ^ (f & 7)) << 4);
+                                split4(make_uint4(x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]), h, l);
+                                const int off = row_off + (((quarter * 2 + c) ^ (f & 7)) << 4);
                                 *reinterpret_cast<uint4 *>(bhi + off) = h;
                                 *reinterpret_cast<uint4 *>(blo + off) = l;
                             }

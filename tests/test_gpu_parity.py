@@ -413,3 +413,29 @@ def test_full_size_f32_matmul_sampled(M, N, K):
     assert sg.sg_last_kernel() == TENSOR
     assert assert_within_bound(got, want, S, f"sampled f32 {M}x{N}x{K}") < F32_TENSOR_RATIO
     assert not torch.isnan(C).any()
+
+
+def test_f32_tensor_path_special_values():
+    # the hi/lo split must not turn a large finite value into infinity; an infinite or NaN input
+    # gives a non-finite output (inf * lo with lo = 0 is NaN: the 3xTF32 path does not keep
+    # the sign of an infinity, which the header documents)
+    M, N, K = 128, 64, 32
+    A = torch.zeros(M, K, device="cuda")
+    B = torch.zeros(K, N, device="cuda")
+    fmax = torch.finfo(torch.float32).max
+    A[0, 0] = fmax                    # rounding hi up would overflow
+    A[1, 0] = float("inf")
+    A[2, 0] = float("nan")
+    A[3, 0] = -fmax
+    A[4, 0] = 1.0 + 2.0 ** -23        # lo carries the last bit
+    B[0, :] = 0.25
+    C = torch.empty(M, N, device="cuda")
+    sg.sg_set_kernel_override(TENSOR)
+    sg.sg_matmul(A, B, C)
+    torch.cuda.synchronize()
+    assert sg.sg_last_kernel() == TENSOR
+    assert torch.all(torch.isfinite(C[0])) and torch.allclose(C[0], torch.full_like(C[0], fmax * 0.25), rtol=1e-6, atol=0)
+    assert torch.allclose(C[3], torch.full_like(C[3], -fmax * 0.25), rtol=1e-6, atol=0)
+    assert not torch.isfinite(C[1]).any() and not torch.isfinite(C[2]).any()
+    assert torch.all(C[4] == (1.0 + 2.0 ** -23) * 0.25)
+    assert torch.all(C[5:] == 0)
