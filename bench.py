@@ -2,11 +2,13 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-One "step" is one call of the hot path on the headline workload: the bf16 matmul
-C[4096,4096] = A[4096,4096] . B[4096,4096] with f32 accumulation and f32 output (the largest
-point of the matmul sweep).  Rank 0 prints ONE JSON line.  The line also carries, under
-"per_op", the GFLOP/s and roofline fraction of the other configured ops (f32 matmul, both
-convolutions, the large and the skinny matmul), each timed the same way on fewer iterations.
+One "step" is one pass over the matmul sweep: C[M,N] = A[M,K] . B[K,N] for every M, N, K in
+{256, 512, 1024, 2048, 4096} (125 shapes), once with bf16 inputs and once with f32 inputs, f32
+accumulation and f32 output: 250 calls of sg_matmul on dense row-major buffers that stay
+resident in HBM (6.3 GB, far beyond the L2).  Rank 0 prints ONE JSON line.  Its "roofline"
+object describes the kernel that takes most of the step (the f32 tensor-core kernel); "per_op"
+lists the other configured ops (the sweep's 4096^3 corner in both dtypes, config 1, both
+convolutions, the large and the skinny matmul), each timed on its own by CUDA-graph replay.
 
 Multi-GPU (torchrun, one process per GPU): the op has no exchange step, so each rank runs
 the same workload on its own device ("weak" scaling, no data-path collective); the value is
@@ -30,14 +32,20 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-M = N = K = 4096
-WORKLOAD = "matmul 4096x4096x4096, bf16 inputs uniform[-1,1), f32 accumulate and output (largest point of the matmul sweep)"
-FLOPS_PER_STEP = 2.0 * M * N * K
-N_SETS = 3            # rotating (A, B, C) sets: 3 x 128 MB > the 126 MB L2
+SWEEP = (256, 512, 1024, 2048, 4096)
+SHAPES = [(m, n, k) for m in SWEEP for n in SWEEP for k in SWEEP]
+M = N = K = 4096          # the sweep's largest point (CPU sample, per-op table)
+WORKLOAD = ("matmul sweep M,N,K in {256,512,1024,2048,4096} (125 shapes), bf16 inputs and again f32 inputs, "
+            "uniform[-1,1), f32 accumulate and output")
+FLOPS_PER_DTYPE = sum(2.0 * m * n * k for m, n, k in SHAPES)
+FLOPS_PER_STEP = 2 * FLOPS_PER_DTYPE
 
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture; None when the
 # kernel changed after the capture was taken.
 NCU_TRAFFIC_BYTES = None
+# tf32 : bf16 dense tensor throughput (nominal 1.1 : 2.25 PFLOP/s; the issue rate measured on
+# this chip is exactly half)
+TF32_OVER_BF16 = 0.5
 
 
 def load_peaks():
@@ -203,7 +211,8 @@ def measure_op(sg, peaks, spec, reps=None):
     ms = time_graph(calls, reps)
     host_ms = time_launches(lambda i: call(*bufs[i % sets]), max(3, min(100, ncalls * 2)), 2)
     tf = flops / (ms * 1e-3) / 1e12
-    t_compute = flops / ((peaks["bf16_tflops"] if fam == sg.SG_KERNEL_TENSOR else ffma_peak) * 1e12)
+    tensor_peak = peaks["bf16_tflops"] * (TF32_OVER_BF16 if dtype == "f32" else 1.0)
+    t_compute = flops / ((tensor_peak if fam == sg.SG_KERNEL_TENSOR else ffma_peak) * 1e12)
     t_bytes = bytes_ / (peaks["hbm_gbs"] * 1e9)
     bound = max(t_compute, t_bytes)
     row = {"op": label, "dtype": dtype, "kernel": "tensor" if fam == sg.SG_KERNEL_TENSOR else "ffma",
@@ -212,6 +221,9 @@ def measure_op(sg, peaks, spec, reps=None):
            "bound": "hbm" if t_bytes > t_compute else ("tensor" if fam == sg.SG_KERNEL_TENSOR else "ffma"),
            "roofline_us": round(bound * 1e6, 2), "frac": round(bound / (ms * 1e-3), 4), "rotating_sets": sets,
            "timing": "CUDA graph replay"}
+    if dtype == "f32" and fam == sg.SG_KERNEL_TENSOR:
+        # the f32 path issues three tf32 products per term: its own ceiling is a third of the tf32 peak
+        row["frac_of_3xtf32_ceiling"] = round(max(3 * t_compute, t_bytes) / (ms * 1e-3), 4)
     del bufs, calls
     torch.cuda.empty_cache()
     return row
@@ -219,7 +231,7 @@ def measure_op(sg, peaks, spec, reps=None):
 
 def per_op_table(sg, peaks, seed):
     specs = op_specs(sg, seed)
-    return [measure_op(sg, peaks, specs[name]) for name in specs if name != "matmul4096_bf16"]
+    return [measure_op(sg, peaks, specs[name]) for name in specs]
 
 
 def cpu_baseline(target_seconds=12.0):
@@ -257,24 +269,64 @@ def run_reference(args, rank):
             vals.append(info["value"])
     value = statistics.mean(vals)
     info["value"] = round(value, 3)
-    line = {"impl": "reference", "metric": "matmul GFLOP/s (4096^3 bf16-valued inputs, f64 CPU oracle)", "value": round(value, 3),
+    line = {"impl": "reference", "metric": "matmul sweep GFLOP/s (f64 CPU oracle on a bounded sample)", "value": round(value, 3),
             "unit": "GFLOP/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": round(FLOPS_PER_STEP / (value * 1e9) * 1e3, 1), "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD},
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": "leading rows of the sweep's 4096^3 point, bf16-valued inputs"},
             "cpu_baseline": info, "e2e": {"value": round(value, 3), "unit": "GFLOP/s", "h2d_bytes_per_step": 0,
                                            "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
 
+def sweep_buffers(torch, seed):
+    """Dense device buffers for every shape of the sweep, both dtypes: sub-blocks of one seeded
+    4096 x 4096 sample per operand, copied out so that every matrix is contiguous."""
+    import numpy as np
+    from paper_2202_03293_b200 import inputs
+    full = {}
+    for dtype in ("bf16", "f32"):
+        for name, tid in (("A", 1), ("B", 2)):
+            payload, _ = inputs.make((4096, 4096), seed, tid, "uniform", dtype)
+            t = torch.from_numpy(payload.view(np.int16) if dtype == "bf16" else payload).cuda()
+            full[dtype, name] = t.view(torch.bfloat16) if dtype == "bf16" else t
+    bufs = {}
+    for dtype in ("bf16", "f32"):
+        for (m, n, k) in SHAPES:
+            bufs[dtype, m, n, k] = (full[dtype, "A"][:m, :k].contiguous(), full[dtype, "B"][:k, :n].contiguous(),
+                                    torch.empty(m, n, device="cuda"))
+    return bufs
+
+
+def sweep_table(sg, peaks, bufs, torch):
+    """Per-shape device time (CUDA events around a few back-to-back launches) and roofline fraction."""
+    rows = []
+    for dtype in ("bf16", "f32"):
+        es = 2 if dtype == "bf16" else 4
+        peak = peaks["bf16_tflops"] * (TF32_OVER_BF16 if dtype == "f32" else 1.0) * 1e12
+        for (m, n, k) in SHAPES:
+            a, b, c = bufs[dtype, m, n, k]
+            flops = 2.0 * m * n * k
+            reps = int(max(3, min(40, 2e-3 / max(flops / 3e14, 8e-6))))
+            ms = time_launches(lambda i: sg.sg_matmul(a, b, c), reps, 2)
+            t_c, t_b = flops / peak, ((m * k + k * n) * es + m * n * 4) / (peaks["hbm_gbs"] * 1e9)
+            rows.append({"dtype": dtype, "M": m, "N": n, "K": k, "us": round(ms * 1e3, 2),
+                         "gflops": round(flops / (ms * 1e-3) / 1e9, 1), "bound": "hbm" if t_b > t_c else "tensor",
+                         "frac": round(max(t_c, t_b) / (ms * 1e-3), 4)})
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-per-op", action="store_true", help="skip the per-op table")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--op", default=None, help="time only this op of the per-op table (used for profiler captures)")
+    ap.add_argument("--sweep-table", default=None, help="also time every shape of the sweep on its own and write the table to this JSON file")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -308,12 +360,19 @@ def main():
         print(json.dumps(measure_op(sg, peaks, specs[args.op], reps=max(1, min(args.steps, 5)))), flush=True)
         return
 
-    sets = [(gpu_operand((M, K), seed, 1 + 3 * s, "uniform", "bf16"), gpu_operand((K, N), seed, 2 + 3 * s, "uniform", "bf16"),
-             torch.empty(M, N, device="cuda")) for s in range(N_SETS)]
+    bufs = sweep_buffers(torch, seed)
+    # large shapes first, so that the host's call overhead of the small ones hides behind them
+    order = sorted(SHAPES, key=lambda s: -s[0] * s[1] * s[2])
+    halves = {dt: [bufs[dt, m, n, k] for (m, n, k) in order] for dt in ("f32", "bf16")}
+    mid = torch.cuda.Event(enable_timing=True)
 
-    def step(i):
-        a, b, c = sets[i % N_SETS]
-        sg.sg_matmul(a, b, c)
+    def step(mark=None):
+        for a, b, c in halves["f32"]:
+            sg.sg_matmul(a, b, c)
+        if mark is not None:
+            mark.record()
+        for a, b, c in halves["bf16"]:
+            sg.sg_matmul(a, b, c)
 
     def barrier():
         if world > 1:
@@ -321,15 +380,20 @@ def main():
         torch.cuda.synchronize()
 
     for i in range(warmup):
-        step(i)
+        step()
     barrier()
+    # one step split at the dtype boundary: which kernel dominates, and its average launch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(); step(mid); e1.record()
+    torch.cuda.synchronize()
+    f32_ms, bf16_ms = e0.elapsed_time(mid), mid.elapsed_time(e1)
+
     sampler = ClockSampler(local_rank)
     sampler.start()
     launches0 = sg.sg_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(args.steps):
-        step(i)
+        step()
     e1.record()
     barrier()
     launches = sg.sg_launch_count() - launches0
@@ -340,28 +404,33 @@ def main():
     value = world * FLOPS_PER_STEP / (ms_per_step * 1e-3) / 1e9      # GFLOP/s, all ranks
 
     # ---- end to end through the public call, host buffers, copies inside the timed region ----
-    a_h = sets[0][0].cpu().pin_memory()
-    b_h = sets[0][1].cpu().pin_memory()
-    c_h = torch.empty(M, N).pin_memory()
-    e2e_steps = max(3, min(20, args.steps))
+    e2e = None
+    if not args.no_e2e:
+        host = {key: (a.cpu().pin_memory(), b.cpu().pin_memory(), torch.empty(c.shape).pin_memory())
+                for key, (a, b, c) in bufs.items()}
+        e2e_steps = max(2, min(5, args.steps))
+        h2d = sum(a.numel() * a.element_size() + b.numel() * b.element_size() for a, b, _ in host.values())
+        d2h = sum(c.numel() * 4 for _, _, c in host.values())
 
-    def e2e_step(i):
-        a, b, c = sets[i % N_SETS]
-        a.copy_(a_h, non_blocking=True)
-        b.copy_(b_h, non_blocking=True)
-        sg.sg_matmul(a, b, c)
-        c_h.copy_(c, non_blocking=True)
+        def e2e_step():
+            for key, (a, b, c) in bufs.items():
+                ah, bh, ch = host[key]
+                a.copy_(ah, non_blocking=True)
+                b.copy_(bh, non_blocking=True)
+                sg.sg_matmul(a, b, c)
+                ch.copy_(c, non_blocking=True)
 
-    for i in range(3):
-        e2e_step(i)
-    barrier()
-    e0.record()
-    for i in range(e2e_steps):
-        e2e_step(i)
-    e1.record()
-    barrier()
-    e2e_ms = sharding.max_over_ranks(e0.elapsed_time(e1), device="cuda")
-    e2e_value = world * FLOPS_PER_STEP / (e2e_ms / e2e_steps * 1e-3) / 1e9
+        e2e_step()
+        barrier()
+        e0.record()
+        for i in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = sharding.max_over_ranks(e0.elapsed_time(e1), device="cuda")
+        e2e = {"value": round(world * FLOPS_PER_STEP / (e2e_ms / e2e_steps * 1e-3) / 1e9, 1), "unit": "GFLOP/s",
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+        del host
 
     if rank != 0:
         if world > 1:
@@ -369,31 +438,42 @@ def main():
             dist.destroy_process_group()
         return
 
-    # the timed loop is one kernel launch per step, so the kernel's average duration is the
-    # step time measured above (CUDA events on the launching stream)
+    # dominant kernel: the f32 tensor-core kernel (three tf32 products per term).  Its launches in a
+    # step are the 125 f32 shapes; achieved = their algorithmic flops over their device time.
     timed_seconds = ms_total * 1e-3
     peak_kind = "bf16_tflops_sustained" if timed_seconds >= 1.0 else "bf16_tflops"
-    achieved_tf = FLOPS_PER_STEP / (ms_per_step * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "achieved": round(achieved_tf, 1), "peak": peaks[peak_kind], "unit": "TFLOP/s",
-                "frac": round(achieved_tf / peaks[peak_kind], 4), "traffic": NCU_TRAFFIC_BYTES,
-                "peak_source": f"{peaks['source']} {peak_kind} (timed region {timed_seconds:.2f} s)",
-                "kernel": "tc_gemm_kernel", "algorithmic_flops_per_launch": FLOPS_PER_STEP,
-                "frac_of_burst": round(achieved_tf / peaks["bf16_tflops"], 4),
-                "frac_of_sustained": round(achieved_tf / peaks["bf16_tflops_sustained"], 4)}
+    tf32_peak = peaks[peak_kind] * TF32_OVER_BF16
+    share_f32 = f32_ms / (f32_ms + bf16_ms)
+    f32_tf = FLOPS_PER_DTYPE / (ms_per_step * share_f32 * 1e-3) / 1e12
+    bf16_tf = FLOPS_PER_DTYPE / (ms_per_step * (1 - share_f32) * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "achieved": round(f32_tf, 1), "peak": round(tf32_peak, 1), "unit": "TFLOP/s",
+                "frac": round(f32_tf / tf32_peak, 4), "traffic": NCU_TRAFFIC_BYTES,
+                "kernel": "tc_gemm_kernel<BN, CG, f32> (125 launches per step, %.0f%% of the step)" % (100 * share_f32),
+                "peak_source": f"{peaks['source']} {peak_kind} x {TF32_OVER_BF16} (tf32 : bf16 tensor rate); timed region {timed_seconds:.2f} s",
+                "algorithmic_flops_per_step": FLOPS_PER_DTYPE, "avg_launch_us": round(ms_per_step * share_f32 * 1e3 / len(SHAPES), 2),
+                "note": "f32 accuracy costs three tf32 products per term, so this kernel's own ceiling is frac = 0.333",
+                "frac_of_3xtf32_ceiling": round(3 * f32_tf / tf32_peak, 4),
+                "bf16_half": {"achieved": round(bf16_tf, 1), "peak": peaks[peak_kind], "frac": round(bf16_tf / peaks[peak_kind], 4),
+                              "share_of_step": round(1 - share_f32, 4)}}
 
-    line = {"metric": "matmul GFLOP/s (and fraction of the tensor-core roofline) on B200", "value": round(value, 1),
+    line = {"metric": "matmul sweep GFLOP/s (and fraction of the tensor-core roofline) on B200", "value": round(value, 1),
             "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
             "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "M": M, "N": N, "K": K,
-                       "l2": f"inputs rotate over {N_SETS} buffer sets ({N_SETS * 128} MB) > 126 MB L2",
+            "dtype": "bf16+f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "calls_per_step": 2 * len(SHAPES),
+                       "l2": "every shape has its own buffers, 6.3 GB per step > 126 MB L2",
                        "parallelism": f"replicas x{world}, no collective"},
-            "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches),
-            "e2e": {"value": round(e2e_value, 1), "unit": "GFLOP/s", "h2d_bytes_per_step": 2 * M * K * 2,
-                    "d2h_bytes_per_step": M * N * 4, "steps": e2e_steps}}
+            "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e}
+    if args.sweep_table:
+        rows = sweep_table(sg, peaks, bufs, torch)
+        with open(args.sweep_table, "w") as f:
+            json.dump(rows, f)
+        for dt in ("bf16", "f32"):
+            fr = sorted(r["frac"] for r in rows if r["dtype"] == dt)
+            line.setdefault("sweep_fractions", {})[dt] = {"min": fr[0], "median": fr[len(fr) // 2], "max": fr[-1]}
+    del bufs, halves
+    torch.cuda.empty_cache()
     if not args.no_per_op:
-        del sets
-        torch.cuda.empty_cache()
         line["per_op"] = per_op_table(sg, peaks, seed)
     if not args.no_cpu and world == 1:
         line["cpu_baseline"] = cpu_baseline()[0]

@@ -151,6 +151,21 @@ int64_t sg_launch_count(void);
  */
 sg_status sg_set_kernel_override(int kernel_family);
 
+/*
+ * Tensor-core path only, for testing and benchmarking: force the output tile width (64, 128
+ * or 256 columns), the number of CTAs that share a tile (1, or 2 = a CTA pair working on 256
+ * rows) and the number of contiguous k ranges a tile's reduction is dealt out in (partial
+ * sums then meet in the output by reduce-add; an overwriting call clears the output first).
+ * 0 leaves a choice to the library's cost estimate.  A combination that does not exist (256
+ * columns on one CTA with f32 inputs) or does not fit the shape falls back to that estimate.
+ * Returns SG_ERR_INVALID_ARG for other values.  The environment variables SG_TC_BN, SG_TC_CG
+ * and SG_TC_SPLIT, read at the first call, set the same three values.
+ */
+sg_status sg_set_tile_override(int tile_n, int ctas_per_tile, int k_splits);
+
+/* {tile width, CTAs per tile, k ranges} of the most recent tensor-core launch of the process. */
+void sg_last_tile_choice(int out[3]);
+
 /* Drops cached tensor maps and other host-side state.  Safe to call twice. */
 void sg_shutdown(void);
 

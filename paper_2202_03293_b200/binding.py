@@ -23,7 +23,8 @@ SG_KERNEL_AUTO, SG_KERNEL_FFMA, SG_KERNEL_TENSOR = 0, 1, 2
 
 EXPORTS = [
     "sg_matmul", "sg_conv1d_nwc_wcf", "sg_conv2d_nhwc_hwcf", "sg_check", "sg_status_string",
-    "sg_version", "sg_last_kernel", "sg_launch_count", "sg_set_kernel_override", "sg_shutdown",
+    "sg_version", "sg_last_kernel", "sg_launch_count", "sg_set_kernel_override", "sg_set_tile_override",
+    "sg_last_tile_choice", "sg_shutdown",
 ]
 
 
@@ -58,6 +59,10 @@ def lib() -> ctypes.CDLL:
         L.sg_launch_count.restype = i64
         L.sg_set_kernel_override.argtypes = [ci]
         L.sg_set_kernel_override.restype = ci
+        L.sg_set_tile_override.argtypes = [ci, ci, ci]
+        L.sg_set_tile_override.restype = ci
+        L.sg_last_tile_choice.argtypes = [ctypes.POINTER(ctypes.c_int)]
+        L.sg_last_tile_choice.restype = None
         L.sg_shutdown.restype = None
         _lib = L
     return _lib
@@ -163,6 +168,18 @@ def sg_set_kernel_override(kernel_family: int) -> None:
     rc = lib().sg_set_kernel_override(int(kernel_family))
     if rc != SG_OK:
         raise SgError(rc, "sg_set_kernel_override")
+
+
+def sg_set_tile_override(tile_n: int = 0, ctas_per_tile: int = 0, k_splits: int = 0) -> None:
+    rc = lib().sg_set_tile_override(int(tile_n), int(ctas_per_tile), int(k_splits))
+    if rc != SG_OK:
+        raise SgError(rc, "sg_set_tile_override")
+
+
+def sg_last_tile_choice():
+    out = (ctypes.c_int * 3)()
+    lib().sg_last_tile_choice(out)
+    return out[0], out[1], out[2]
 
 
 def sg_shutdown() -> None:

@@ -176,6 +176,17 @@ sg_status sg_set_kernel_override(int kernel_family) {
     return SG_OK;
 }
 
+sg_status sg_set_tile_override(int tile_n, int ctas_per_tile, int k_splits) {
+    if (tile_n != 0 && tile_n != 64 && tile_n != 128 && tile_n != 256) return SG_ERR_INVALID_ARG;
+    if (ctas_per_tile < 0 || ctas_per_tile > 2 || k_splits < 0 || k_splits > 64) return SG_ERR_INVALID_ARG;
+    tensor_set_tile_override(tile_n, ctas_per_tile, k_splits);
+    return SG_OK;
+}
+
+void sg_last_tile_choice(int out[3]) {
+    if (out) tensor_last_choice(out);
+}
+
 void sg_shutdown(void) { tensor_shutdown(); }
 
 }  // extern "C"

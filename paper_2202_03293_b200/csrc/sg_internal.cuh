@@ -40,6 +40,8 @@ cudaError_t launch_zero_fill(const Problem &p, float *O, cudaStream_t stream);
 sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float *O,
                         cudaStream_t stream);
 void tensor_shutdown();
+void tensor_set_tile_override(int bn, int cg, int splits);
+void tensor_last_choice(int out[3]);
 // Reads and clears the current device's status word (written by kernels whose bounded
 // waits expire); the caller has already synchronised the stream.
 sg_status tensor_read_status(cudaStream_t stream);

@@ -55,6 +55,8 @@ struct TcParams {
     int M, N;
     int num_m_tiles, num_n_tiles;
     int num_kb;          // k-blocks per tile = taps * kb_per_tap
+    int splits;          // work items per tile: the k-blocks are dealt out in `splits` contiguous ranges
+    int kb_per_split;    // ceil(num_kb / splits); partial sums meet in the output by reduce-add
     int kb_per_tap;      // ceil(C / 64)
     int KW;              // taps are ordered (kh, kw)
     int a_mode;          // 0: tiled 2-D (matmul), 1: im2col 3-D (conv1d), 2: im2col 4-D (conv2d)
@@ -414,7 +416,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_slot;
 
-    const int num_tiles = p.num_m_tiles * p.num_n_tiles;   // tiles of (CG*128) x BN
+    // work items: (tile of (CG*128) x BN, k range); the splits of one tile are neighbours in the
+    // order, so they run at the same time and their operands meet in L2
+    const int num_tiles = p.num_m_tiles * p.num_n_tiles * p.splits;
+    auto item_range = [&](int t, int &tile, int &kb0, int &kb1) {
+        tile = t / p.splits;
+        kb0 = (t - tile * p.splits) * p.kb_per_split;
+        kb1 = kb0 + p.kb_per_split < p.num_kb ? kb0 + p.kb_per_split : p.num_kb;
+    };
     // bf16 pairs count both CTAs' TMA bytes on the leader's barrier, which its MMA thread waits
     // on.  f32 pairs signal each CTA's own barrier (its converter warps wait there) and the
     // leader's MMA thread waits on the split barrier instead.
@@ -426,8 +435,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
             int it = 0;   // k-block counter across all of this CTA's tiles
             bool ok = true;
             for (int t = group_id; t < num_tiles && ok; t += num_groups) {
-                int mt, nt;
-                tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+                int mt, nt, tile, kb0, kb1;
+                item_range(t, tile, kb0, kb1);
+                tile_coords(tile, p.num_m_tiles, p.num_n_tiles, mt, nt);
                 const int m0 = (mt * CG + (int)cta_rank) * BM;
                 const int n0 = nt * BN + (int)cta_rank * C::B_COLS;
                 int pix_n = 0, pix_h = 0, pix_w = 0;   // first output pixel of this CTA's rows
@@ -438,7 +448,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     pix_h = r / p.Wo;
                     pix_w = r - pix_h * p.Wo;
                 }
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int s = it % C::STAGES;
                     const uint32_t ph = (it / C::STAGES) & 1;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -499,7 +509,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                 if (!mbar_wait(acc_empty_bar(buf), ((tl >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                int tile, kb0, kb1;
+                item_range(t, tile, kb0, kb1);
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     if constexpr (F32) {
                         const int s = it & 1;
                         if (!mbar_wait<CG == 2>(split_full_bar(s), (it >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -514,7 +526,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
 #pragma unroll
                         for (int k = 0; k < K_STEPS; ++k) {
                             const uint64_t o = (uint64_t)(k * 2);
-                            mma(d_tmem, al + o, bh + o, (kb > 0 || k > 0) ? 1u : 0u);   // small terms first
+                            mma(d_tmem, al + o, bh + o, (kb > kb0 || k > 0) ? 1u : 0u);   // small terms first
                             mma(d_tmem, ah + o, bl + o, 1u);
                             mma(d_tmem, ah + o, bh + o, 1u);
                         }
@@ -540,7 +552,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
 #pragma unroll
                         for (int k = 0; k < K_STEPS; ++k)
                             mma(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * C::B_KSTEP_DESC),
-                                (kb > 0 || k > 0) ? 1u : 0u);
+                                (kb > kb0 || k > 0) ? 1u : 0u);
                         // the stage is free (in every CTA of the group) once these MMAs have read it
                         if constexpr (CG == 1) {
                             umma_commit(empty_bar(s));
@@ -568,7 +580,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
             int it = 0;
             bool ok = true;
             for (int t = group_id; t < num_tiles && ok; t += num_groups) {
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                int tile, kb0, kb1;
+                item_range(t, tile, kb0, kb1);
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int r = it % C::STAGES, s = it & 1;
                     if (!mbar_wait(full_bar(r), (it / C::STAGES) & 1, abort_flag)) { ok = false; break; }
                     if (!mbar_wait<CG == 2>(split_empty_bar(s), ((it >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
@@ -639,7 +653,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         bool ok = true;
         for (int t = group_id; t < num_tiles && ok; t += num_groups, ++tl) {
             int mt, nt;
-            tile_coords(t, p.num_m_tiles, p.num_n_tiles, mt, nt);
+            tile_coords(t / p.splits, p.num_m_tiles, p.num_n_tiles, mt, nt);
             const int m0 = (mt * CG + (int)cta_rank) * BM, n0 = nt * BN;
             const int buf = tl & 1;
             if (!mbar_wait(acc_full_bar(buf), (tl >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -719,8 +733,10 @@ struct Driver {
 };
 std::mutex g_mu;
 Driver g_drv;
-int g_bn_override = -1;   // tile width forced by SG_TC_BN (-1: not read yet; 0: automatic)
-int g_cg_override = 0;    // CTAs per tile forced by SG_TC_CG (0: automatic)
+int g_bn_override = -1;   // tile width forced by SG_TC_BN or sg_set_tile_override (-1: not read yet; 0: automatic)
+int g_cg_override = 0;    // CTAs per tile (0: automatic)
+int g_split_override = 0; // k ranges per tile (0: automatic)
+int g_last_choice[3] = {0, 0, 0};
 
 bool init_driver() {
     int dev = 0;
@@ -745,13 +761,36 @@ bool init_driver() {
 
 inline bool mult(int64_t v, int64_t q) { return v % q == 0; }
 
-struct Variant { int bn, cg; double step_cost, step_cost_f32; };
-// Relative cost of one k-block of a tile per variant.  bf16: measured on large problems; narrow
-// tiles pay more shared-memory traffic per flop, CTA pairs stage the filter once.  f32: the
-// shared-memory cycles of one k-block (TMA fill, hi/lo split, operand reads of the 12 MMAs).
-constexpr Variant kVariants[] = {{64, 1, 80.0, 1344.0}, {128, 1, 102.0, 1792.0}, {256, 1, 128.0, 2688.0},
-                                 {128, 2, 95.0, 1344.0}, {256, 2, 120.0, 1792.0}};
+struct Variant { int bn, cg; double mma_ns, mma_ns_f32; };
+// Time one CTA's tensor core (bf16) or shared memory (f32: TMA fill, hi/lo split and the operand
+// reads of 12 MMAs share it) needs for one k-block of a tile, in ns.
+constexpr Variant kVariants[] = {{64, 1, 100.0, 750.0}, {128, 1, 135.0, 1000.0}, {256, 1, 270.0, 1500.0},
+                                 {128, 2, 135.0, 750.0}, {256, 2, 270.0, 1000.0}};
 constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
+
+// Estimated kernel time in ns of `tiles` tiles dealt out in `sp` k ranges each over `groups`
+// CTAs or CTA pairs.  A k-block costs the slowest of: the CTA's own MMA / shared-memory
+// time, the CTA's share of the L2 -> shared memory fill rate of the whole chip (what bounds
+// every large problem here: about 10 TB/s), and the fill rate one SM reaches alone.  The
+// constants were fitted to timings of every variant and split on the 125 shapes
+// {256..4096}^3 in both dtypes; the choices they lead to are within 1 % of the best
+// per-shape choice in total time.
+double estimate_ns(const Variant &v, bool f32, int64_t tiles, int64_t groups, int num_kb, int sp, bool accumulate) {
+    const int64_t items = tiles * sp;
+    const int64_t waves = (items + groups - 1) / groups;
+    const int kbs = (num_kb + sp - 1) / sp;
+    const double active = (double)((items < groups ? items : groups) * v.cg);
+    const double stage_bytes = A_STAGE_BYTES + (double)(v.bn / v.cg) * ROW_BYTES;
+    const double chip_fill = f32 ? 9000.0 : 10500.0, sm_fill = f32 ? 40.0 : 90.0;      // bytes per ns
+    double kb_ns = f32 ? v.mma_ns_f32 : v.mma_ns;
+    if (active * stage_bytes / chip_fill > kb_ns) kb_ns = active * stage_bytes / chip_fill;
+    if (stage_bytes / sm_fill > kb_ns) kb_ns = stage_bytes / sm_fill;
+    const double item_ns = 1500.0 + (double)v.bn * (f32 ? 24.0 : 12.0);                // pipeline fill + epilogue of one item
+    double t = (double)waves * kbs * kb_ns + item_ns + (double)(waves - 1) * (f32 ? 0.0 : 0.3) * item_ns;
+    if (v.cg == 2) t += f32 ? 800.0 : 2000.0;                                          // cluster launch, cross-CTA signalling
+    if (sp > 1) t += (f32 ? 4000.0 : 2500.0) - (accumulate ? 1500.0 : 0.0);            // reduce-add traffic, the clearing launch
+    return t;
+}
 
 template <int BN, int CG, bool F32>
 sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUtensorMap &mo, TcParams tp, int M, int N,
@@ -767,7 +806,7 @@ sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUt
     }
     tp.num_m_tiles = (M + CG * BM - 1) / (CG * BM);
     tp.num_n_tiles = (N + BN - 1) / BN;
-    const int tiles = tp.num_m_tiles * tp.num_n_tiles;
+    const int tiles = tp.num_m_tiles * tp.num_n_tiles * tp.splits;
     const int groups = g_drv.num_sms / CG;
     const int grid = CG * (tiles < groups ? tiles : groups);
     cudaLaunchConfig_t cfg = {};
@@ -816,6 +855,8 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         g_bn_override = e ? atoi(e) : 0;
         e = getenv("SG_TC_CG");
         g_cg_override = e ? atoi(e) : 0;
+        e = getenv("SG_TC_SPLIT");
+        g_split_override = e ? atoi(e) : 0;
     }
 
     alignas(64) CUtensorMap map_in, map_flt, map_out;
@@ -902,31 +943,47 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
     }
 
-    // ---- tile variant: fewest (waves x per-tile cost); narrower tiles cost more shared-memory
-    //      traffic per flop, wider ones and CTA pairs quantise worse on small problems ----
-    int pick = -1;
+    // ---- tile variant and k split: lowest estimated time ----
+    int pick = -1, splits = 1;
     if (g_bn_override > 0) {
         for (int i = 0; i < kNumVariants; ++i)
             if (kVariants[i].bn == g_bn_override && kVariants[i].cg == (g_cg_override > 0 ? g_cg_override : 1) &&
                 !(f32 && kVariants[i].bn == 256 && kVariants[i].cg == 1)) pick = i;
     }
-    for (int pass = 0; pass < 2 && pick < 0; ++pass) {   // pass 1 drops a forced group size that does not fit
+    auto valid_split = [&](int s) {      // every range of ceil(num_kb / s) k-blocks must be non-empty
+        const int per = (tp.num_kb + s - 1) / s;
+        return s >= 1 && (s - 1) * per < tp.num_kb;
+    };
+    if (pick >= 0) {
+        splits = g_split_override > 0 && valid_split(g_split_override) ? g_split_override : 1;
+    } else {
         double best = 1e300;
         for (int i = 0; i < kNumVariants; ++i) {
             const Variant &v = kVariants[i];
-            if (pass == 0 && g_cg_override > 0 && v.cg != g_cg_override) continue;
+            if (g_cg_override > 0 && v.cg != g_cg_override && !(v.cg == 1 && p.M <= BM)) continue;
             if (f32 && v.bn == 256 && v.cg == 1) continue;       // not built (shared-memory budget)
             if (v.bn > 64 && v.bn / 2 >= p.N) continue;          // at most half of the tile would be used
             if (v.cg == 2 && p.M <= BM) continue;                // the second CTA would have no rows
-            int64_t tiles = (int64_t)((p.M + v.cg * BM - 1) / (v.cg * BM)) * ((p.N + v.bn - 1) / v.bn);
-            int64_t groups = g_drv.num_sms / v.cg;
-            int64_t waves = (tiles + groups - 1) / groups;
-            // a pair pays a fixed price (cluster launch, cross-CTA signalling) worth ~6 k-blocks
-            double cost = (double)waves * tp.num_kb * (f32 ? v.step_cost_f32 : v.step_cost) + (v.cg == 2 ? (f32 ? 6000.0 : 760.0) : 0.0);
-            if (cost < best) { best = cost; pick = i; }
+            const int64_t tiles = (int64_t)((p.M + v.cg * BM - 1) / (v.cg * BM)) * ((p.N + v.bn - 1) / v.bn);
+            const int64_t groups = g_drv.num_sms / v.cg;
+            for (int sp = 1; sp <= 32; sp *= 2) {
+                if (g_split_override > 0 && sp != g_split_override) continue;
+                if (!valid_split(sp)) break;
+                if (sp > 1 && tiles * (sp / 2) >= 2 * groups) break;   // already two waves without this split
+                const double c = estimate_ns(v, f32, tiles, groups, tp.num_kb, sp, p.accumulate != 0);
+                if (c < best) { best = c; pick = i; splits = sp; }
+            }
         }
     }
     if (pick < 0) return SG_ERR_INTERNAL;
+    tp.splits = splits;
+    tp.kb_per_split = (tp.num_kb + splits - 1) / splits;
+    if (splits > 1) {
+        // partial sums meet in the output by TMA reduce-add: an overwriting call clears it first
+        if (!p.accumulate && launch_zero_fill(p, O, stream) != cudaSuccess) return SG_ERR_CUDA;
+        tp.accumulate = 1;
+    }
+    g_last_choice[0] = kVariants[pick].bn; g_last_choice[1] = kVariants[pick].cg; g_last_choice[2] = splits;
     const int slot = pick + (f32 ? kNumVariants : 0);
 #define SG_LAUNCH(BN_, CG_)                                                                              \
     (f32 ? launch_variant<BN_, CG_, true>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)          \
@@ -953,6 +1010,16 @@ sg_status tensor_read_status(cudaStream_t stream) {
         return SG_ERR_DEVICE_TIMEOUT;
     }
     return SG_OK;
+}
+
+void tensor_set_tile_override(int bn, int cg, int splits) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    g_bn_override = bn; g_cg_override = cg; g_split_override = splits;
+}
+
+void tensor_last_choice(int out[3]) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    out[0] = g_last_choice[0]; out[1] = g_last_choice[1]; out[2] = g_last_choice[2];
 }
 
 void tensor_shutdown() {

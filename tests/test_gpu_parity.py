@@ -17,8 +17,10 @@ FFMA, TENSOR = sg.SG_KERNEL_FFMA, sg.SG_KERNEL_TENSOR
 @pytest.fixture(autouse=True)
 def _reset_override():
     sg.sg_set_kernel_override(sg.SG_KERNEL_AUTO)
+    sg.sg_set_tile_override(0, 0, 0)
     yield
     sg.sg_set_kernel_override(sg.SG_KERNEL_AUTO)
+    sg.sg_set_tile_override(0, 0, 0)
     sg.sg_check()      # no kernel of the test gave up on a bounded wait
 
 
@@ -125,6 +127,45 @@ def test_tensor_path_every_tile_variant(bn, cg):
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     out = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
     assert out.returncode == 0 and "child-ok" in out.stdout, out.stdout + out.stderr
+
+
+# ------------------------------------------------------------------ reduction dealt out in k ranges
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("bn,cg,splits", [(64, 1, 2), (64, 1, 5), (128, 1, 4), (128, 2, 3), (256, 2, 8), (256, 1, 16)])
+@pytest.mark.parametrize("accumulate", [False, True])
+def test_matmul_split_reduction(dtype, bn, cg, splits, accumulate):
+    if dtype == "f32" and (bn, cg) == (256, 1):
+        pytest.skip("no such f32 instantiation")
+    # ragged in m, n and k; the last k range is shorter than the others
+    M, N, K = 300, 328, 2000 if dtype == "bf16" else 1000
+    sg.sg_set_tile_override(bn, cg, splits)
+    C, want, S = run_matmul(M, N, K, dtype, family=TENSOR, accumulate=accumulate, seed=SEED + 11)
+    assert sg.sg_last_tile_choice() == (bn, cg, splits)
+    ratio = assert_within_bound(C, want, S, f"split {splits} of {dtype} {bn}x{cg}")
+    assert ratio < F32_TENSOR_RATIO
+
+
+def test_split_reduction_is_chosen_for_few_tiles_and_long_k():
+    for dtype in ("bf16", "f32"):
+        C, want, S = run_matmul(256, 256, 4096, dtype, seed=SEED + 12)
+        assert sg.sg_last_kernel() == TENSOR and sg.sg_last_tile_choice()[2] > 1
+        assert_within_bound(C, want, S, "256x256x4096")
+        # integer inputs: every order of the partial sums gives the same bits
+        C, want, S = run_matmul(256, 256, 4096, dtype, dist="ints", seed=SEED + 12)
+        assert np.array_equal(C.cpu().numpy().astype(np.float64), want)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_conv_split_reduction(dtype):
+    sg.sg_set_tile_override(128, 1, 3)
+    O, want, S = run_conv2d(3, 20, 20, 64, 3, 3, 128, (1, 1), (1, 1), dtype, family=TENSOR, seed=SEED + 13)
+    assert sg.sg_last_tile_choice() == (128, 1, 3)
+    assert_within_bound(O, want, S, "conv2d split over taps")
+    sg.sg_set_tile_override(64, 1, 2)
+    O, want, S = run_conv1d(4, 300, 136, 3, 128, 1, 1, dtype, family=TENSOR, accumulate=True, seed=SEED + 13)
+    assert sg.sg_last_tile_choice() == (64, 1, 2)
+    assert_within_bound(O, want, S, "conv1d split, accumulate")
 
 
 @pytest.mark.parametrize("family", [FFMA, TENSOR])
