@@ -62,6 +62,7 @@ struct TcParams {
     int a_mode;          // 0: tiled 2-D (matmul), 1: im2col 3-D (conv1d), 2: im2col 4-D (conv2d)
     int Ho, Wo, sh, sw, dh, dw;
     int accumulate;
+    int b_blocked;       // 1: the filter map is blocked by sub-tile columns: one TMA load fetches the whole filter tile
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -263,7 +264,9 @@ struct Cfg {
     static constexpr int SPLIT_BYTES = 2 * STAGE_BYTES;
     static constexpr int RING_BUDGET = 196608 - SPLIT_SLOTS * SPLIT_BYTES;
     static constexpr int STAGES = (RING_BUDGET / STAGE_BYTES) > 8 ? 8 : (RING_BUDGET / STAGE_BYTES);
-    static constexpr int THREADS = 192 + (F32 ? CONVERTER_THREADS : 0);   // producer, MMA, 4 epilogue (, 8 converter) warps
+    // warps: input producer, MMA, 4 epilogue (, 8 converter), filter producer
+    static constexpr int THREADS = 192 + (F32 ? CONVERTER_THREADS : 0) + 32;
+    static constexpr int FLT_WARP = THREADS / 32 - 1;
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // two accumulator buffers
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SPLIT_SLOTS * SPLIT_BYTES + STAGING_BYTES +
                                       1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -330,6 +333,23 @@ __device__ __forceinline__ void tma_load_im2col_4d_cg2(uint32_t dst, const CUten
         "cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
 }
+// Rank-5 tiled load.  CG2: the mbarrier may belong to the peer CTA of a pair.  One TMA
+// instruction costs the issuing thread several hundred cycles whatever the size of its box
+// (measured: ~550 cycles, boxes of 8 to 64 KB), so operand tiles are fetched with as few and as
+// large boxes as the layout allows, and the two operands are issued by different warps.
+template <bool CG2>
+__device__ __forceinline__ void tma_tile_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z, int w, int v) {
+    if constexpr (CG2)
+        asm volatile("cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+                     ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v) : "memory");
+    else
+        asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+                     ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v) : "memory");
+}
+// Starts the fetch of a tensor map (a kernel parameter) ahead of its first use.
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
 // D[tmem of both CTAs] (+)= A * B, 256 x N x 16 across the CTA pair.
 __device__ __forceinline__ void umma_bf16_cg2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
@@ -377,18 +397,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_gen + 8 * 24 + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) { prefetch_tensormap(&map_in); prefetch_tensormap(&map_flt); prefetch_tensormap(&map_out); }
     // In a pair, CTA 0 (the leader) issues the MMAs; both CTAs produce and both run epilogues.
     const uint32_t cta_rank = CG == 2 ? cluster_ctarank() : 0u;
     const int group_id = CG == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int num_groups = CG == 2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
-        // full: one arrive.expect_tx by a producer.  empty: one tcgen05.commit (bf16) or one arrive per
+        // full: one arrive.expect_tx by each of the two producers.  empty: one tcgen05.commit (bf16) or one arrive per
         // converter warp of this CTA (f32).  split_full: one arrive per converter warp of every CTA
         // of the group.  split_empty / acc_full: one tcgen05.commit.  acc_empty: one arrive per
         // epilogue warp of every CTA of the group.
         for (int s = 0; s < C::STAGES; ++s) {
-            mbar_init(full_bar(s), 1);
+            mbar_init(full_bar(s), 2);
             mbar_init(empty_bar(s), F32 ? CONVERTER_THREADS / 32 : 1);
         }
         for (int s = 0; s < C::SPLIT_SLOTS; ++s) {
@@ -429,9 +450,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     // leader's MMA thread waits on the split barrier instead.
     constexpr bool REMOTE_FULL = (CG == 2) && !F32;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ producer
+    if (warp == 0 || warp == C::FLT_WARP) {
+        // ------------------------------------------------------------ producers: warp 0 fetches the
+        // input tiles, the last warp the filter tiles; both arm the stage's barrier for their bytes
         if (lane == 0) {
+            const bool input_side = warp == 0;
             int it = 0;   // k-block counter across all of this CTA's tiles
             bool ok = true;
             for (int t = group_id; t < num_tiles && ok; t += num_groups) {
@@ -457,36 +480,40 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     const int tap = kb / p.kb_per_tap;
                     const int c0 = (kb - tap * p.kb_per_tap) * C::BK;
                     const int kh = tap / p.KW, kw = tap - kh * p.KW;
-                    if constexpr (!REMOTE_FULL) {
-                        const uint32_t bar = full_bar(s);
-                        mbar_expect_tx(bar, C::STAGE_BYTES);
-                        if (p.a_mode == 0) {
-                            tma_load_2d(a_dst, &map_in, bar, c0, m0);
-                        } else if (p.a_mode == 1) {
-                            tma_load_im2col_3d(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_n, (unsigned short)(kw * p.dw));
-                        } else {
-                            tma_load_im2col_4d(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_h * p.sh, pix_n,
-                                               (unsigned short)(kw * p.dw), (unsigned short)(kh * p.dh));
-                        }
-#pragma unroll
-                        for (int j = 0; j < C::B_COLS / C::SUB_COLS; ++j)
-                            tma_load_4d(b_dst + j * C::SUB_BYTES, &map_flt, bar, n0 + j * C::SUB_COLS, c0, kw, kh);
-                    } else {
-                        // the leader alone arms its barrier, for the pair's total (a remote arrive by the
-                        // peer would order it after its own loads in flight and serialise the ring)
-                        const uint32_t bar = map_to_cta(full_bar(s), 0);
-                        if (cta_rank == 0) mbar_expect_tx(full_bar(s), CG * C::STAGE_BYTES);
-                        if (p.a_mode == 0) {
-                            tma_load_2d_cg2(a_dst, &map_in, bar, c0, m0);
-                        } else if (p.a_mode == 1) {
-                            tma_load_im2col_3d_cg2(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_n, (unsigned short)(kw * p.dw));
-                        } else {
-                            tma_load_im2col_4d_cg2(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_h * p.sh, pix_n,
+                    // bf16 pairs: the leader alone arms its barrier, for the pair's total (a remote arrive by
+                    // the peer would order it after its own loads in flight and serialise the ring)
+                    const uint32_t bar = REMOTE_FULL ? map_to_cta(full_bar(s), 0) : full_bar(s);
+                    const uint32_t my_bytes = input_side ? A_STAGE_BYTES : C::B_STAGE_BYTES;
+                    if (!REMOTE_FULL || cta_rank == 0) mbar_expect_tx(full_bar(s), (REMOTE_FULL ? CG : 1) * my_bytes);
+                    if (input_side) {
+                        if constexpr (!REMOTE_FULL) {
+                            if (p.a_mode == 0) {
+                                tma_load_2d(a_dst, &map_in, bar, c0, m0);
+                            } else if (p.a_mode == 1) {
+                                tma_load_im2col_3d(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_n, (unsigned short)(kw * p.dw));
+                            } else {
+                                tma_load_im2col_4d(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_h * p.sh, pix_n,
                                                    (unsigned short)(kw * p.dw), (unsigned short)(kh * p.dh));
+                            }
+                        } else {
+                            if (p.a_mode == 0) {
+                                tma_load_2d_cg2(a_dst, &map_in, bar, c0, m0);
+                            } else if (p.a_mode == 1) {
+                                tma_load_im2col_3d_cg2(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_n, (unsigned short)(kw * p.dw));
+                            } else {
+                                tma_load_im2col_4d_cg2(a_dst, &map_in, bar, c0, pix_w * p.sw, pix_h * p.sh, pix_n,
+                                                       (unsigned short)(kw * p.dw), (unsigned short)(kh * p.dh));
+                            }
                         }
+                    } else if (p.b_blocked) {
+                        // box {sub-tile columns, BK channels, B_COLS / SUB_COLS column blocks, 1, 1}
+                        tma_tile_5d<REMOTE_FULL>(b_dst, &map_flt, bar, 0, c0, n0 / C::SUB_COLS, kw, kh);
+                    } else {
 #pragma unroll
-                        for (int j = 0; j < C::B_COLS / C::SUB_COLS; ++j)
-                            tma_load_4d_cg2(b_dst + j * C::SUB_BYTES, &map_flt, bar, n0 + j * C::SUB_COLS, c0, kw, kh);
+                        for (int j = 0; j < C::B_COLS / C::SUB_COLS; ++j) {
+                            if constexpr (REMOTE_FULL) tma_load_4d_cg2(b_dst + j * C::SUB_BYTES, &map_flt, bar, n0 + j * C::SUB_COLS, c0, kw, kh);
+                            else tma_load_4d(b_dst + j * C::SUB_BYTES, &map_flt, bar, n0 + j * C::SUB_COLS, c0, kw, kh);
+                        }
                     }
                 }
             }
@@ -573,7 +600,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
             }
         }
     } else if (warp >= 6) {
-        // ------------------------------------------------------------ converter (f32 only)
+        // ------------------------------------------------------------ converter (f32 only; warps 6 to 13)
         if constexpr (F32) {
             const int cw = warp - 6;                       // converter warp
             const int ct = (int)threadIdx.x - 192;         // converter thread
@@ -917,21 +944,6 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         }
         if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
     }
-    // ---- filter operand: 4-D {f, c, kw, kh}, one sub-tile per load ----
-    {
-        cuuint64_t dims[4] = {(cuuint64_t)p.N, (cuuint64_t)p.C, (cuuint64_t)p.KW, (cuuint64_t)p.KH};
-        int64_t s_kw = p.KW > 1 ? p.k_kw : (int64_t)p.C * p.k_c;
-        int64_t s_kh = p.KH > 1 ? p.k_kh : (int64_t)p.KW * s_kw;
-        cuuint64_t strides[3] = {(cuuint64_t)(p.k_c * es), (cuuint64_t)(s_kw * es), (cuuint64_t)(s_kh * es)};
-        cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)BK, 1, 1};   // one sub-tile: a 128-byte row of columns x BK k-rows
-        // bf16 sub-tiles are consumed by the tensor core as they land (128-byte swizzle); f32
-        // sub-tiles are read by the converter warps, one 128-byte row per load: no swizzle
-        r = g_drv.tiled(&map_flt, in_type, 4, const_cast<void *>(Flt), dims, strides, box, ones,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, f32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
-                        CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
-    }
     // ---- output: 2-D {f, m} f32, stored in 32 x 32 boxes ----
     {
         cuuint64_t dims[2] = {(cuuint64_t)p.N, (cuuint64_t)p.M};
@@ -976,6 +988,33 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         }
     }
     if (pick < 0) return SG_ERR_INTERNAL;
+    // ---- filter operand ----
+    {
+        const int64_t s_kw = p.KW > 1 ? p.k_kw : (int64_t)p.C * p.k_c;
+        const int64_t s_kh = p.KH > 1 ? p.k_kh : (int64_t)p.KW * s_kw;
+        // bf16 sub-tiles are consumed by the tensor core as they land (128-byte swizzle); f32
+        // sub-tiles are read by the converter warps, one 128-byte row per load: no swizzle
+        const CUtensorMapSwizzle swz = f32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B;
+        const int sub_cols = BK;      // columns of one sub-tile: a 128-byte row
+        tp.b_blocked = p.N % sub_cols == 0;
+        if (tp.b_blocked) {
+            // whole sub-tile column blocks: 5-D {column in block, c, column block, kw, kh}; one box
+            // {sub_cols, BK, blocks of this CTA, 1, 1} is the CTA's whole filter tile of a k-block
+            cuuint64_t dims[5] = {(cuuint64_t)sub_cols, (cuuint64_t)p.C, (cuuint64_t)(p.N / sub_cols), (cuuint64_t)p.KW, (cuuint64_t)p.KH};
+            cuuint64_t strides[4] = {(cuuint64_t)(p.k_c * es), (cuuint64_t)ROW_BYTES, (cuuint64_t)(s_kw * es), (cuuint64_t)(s_kh * es)};
+            cuuint32_t box[5] = {(cuuint32_t)sub_cols, (cuuint32_t)BK, (cuuint32_t)(kVariants[pick].bn / kVariants[pick].cg / sub_cols), 1, 1};
+            r = g_drv.tiled(&map_flt, in_type, 5, const_cast<void *>(Flt), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        } else {
+            // 4-D {f, c, kw, kh}, one sub-tile per load
+            cuuint64_t dims[4] = {(cuuint64_t)p.N, (cuuint64_t)p.C, (cuuint64_t)p.KW, (cuuint64_t)p.KH};
+            cuuint64_t strides[3] = {(cuuint64_t)(p.k_c * es), (cuuint64_t)(s_kw * es), (cuuint64_t)(s_kh * es)};
+            cuuint32_t box[4] = {(cuuint32_t)sub_cols, (cuuint32_t)BK, 1, 1};
+            r = g_drv.tiled(&map_flt, in_type, 4, const_cast<void *>(Flt), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        }
+        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
+    }
     tp.splits = splits;
     tp.kb_per_split = (tp.num_kb + splits - 1) / splits;
     if (splits > 1) {
