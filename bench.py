@@ -379,29 +379,62 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(warmup):
+    # The 250 calls of a step are captured once into two CUDA graphs (the f32 half and the bf16
+    # half) and a step replays them: the launch mechanism a fixed sweep would use in production.
+    # The same step issued call by call is timed as well ("eager_ms_per_step").
+    for i in range(2):
         step()
     barrier()
-    # one step split at the dtype boundary: which kernel dominates, and its average launch
+    side = torch.cuda.Stream()
+    graphs = {}
+    launches_per_step = 0
+    for dt in ("f32", "bf16"):
+        g = torch.cuda.CUDAGraph()
+        n0 = sg.sg_launch_count()
+        with torch.cuda.graph(g, stream=side):
+            for a, b, c in halves[dt]:
+                sg.sg_matmul(a, b, c)
+        launches_per_step += sg.sg_launch_count() - n0
+        graphs[dt] = g
+
+    def graph_step(mark=None):
+        graphs["f32"].replay()
+        if mark is not None:
+            mark.record()
+        graphs["bf16"].replay()
+
+    for i in range(warmup):
+        graph_step()
+    barrier()
+    # a few steps split at the dtype boundary: which kernel dominates, and its average launch
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(); step(mid); e1.record()
-    torch.cuda.synchronize()
-    f32_ms, bf16_ms = e0.elapsed_time(mid), mid.elapsed_time(e1)
+    f32_ms = bf16_ms = 0.0
+    for i in range(3):
+        e0.record(); graph_step(mid); e1.record()
+        torch.cuda.synchronize()
+        f32_ms += e0.elapsed_time(mid); bf16_ms += mid.elapsed_time(e1)
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    launches0 = sg.sg_launch_count()
     e0.record()
     for i in range(args.steps):
-        step()
+        graph_step()
     e1.record()
     barrier()
-    launches = sg.sg_launch_count() - launches0
+    launches = launches_per_step * args.steps
     clocks = sampler.stop()
     sg.sg_check()
     ms_total = sharding.max_over_ranks(e0.elapsed_time(e1), device="cuda")
     ms_per_step = ms_total / args.steps
     value = world * FLOPS_PER_STEP / (ms_per_step * 1e-3) / 1e9      # GFLOP/s, all ranks
+
+    eager_steps = max(3, min(20, args.steps))
+    e0.record()
+    for i in range(eager_steps):
+        step()
+    e1.record()
+    barrier()
+    eager_ms = sharding.max_over_ranks(e0.elapsed_time(e1), device="cuda") / eager_steps
 
     # ---- end to end through the public call, host buffers, copies inside the timed region ----
     e2e = None
@@ -461,9 +494,11 @@ def main():
             "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16+f32", "data": "synthetic",
             "config": {"workload": WORKLOAD, "calls_per_step": 2 * len(SHAPES),
+                       "launch": "each step replays two CUDA graphs holding the step's 250 library calls",
                        "l2": "every shape has its own buffers, 6.3 GB per step > 126 MB L2",
                        "parallelism": f"replicas x{world}, no collective"},
-            "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e}
+            "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches),
+            "eager_ms_per_step": round(eager_ms, 5), "e2e": e2e}
     if args.sweep_table:
         rows = sweep_table(sg, peaks, bufs, torch)
         with open(args.sweep_table, "w") as f:
