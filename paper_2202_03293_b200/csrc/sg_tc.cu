@@ -244,7 +244,7 @@ __device__ __forceinline__ void split4(const uint4 v, uint4 &h, uint4 &l) {
     }
 }
 
-template <int BN, int CG, bool F32>
+template <int BN, int CG, bool F32, int KPS = 1>
 struct Cfg {
     // CG = 1: one CTA owns a 128 x BN tile.  CG = 2: a pair of CTAs (one cluster) owns a
     // 256 x BN tile; each CTA stages its own 128 input rows and its own BN/2 filter columns,
@@ -256,7 +256,9 @@ struct Cfg {
     static constexpr int SUB_BYTES = BK * ROW_BYTES;          // one filter sub-tile: BK k-rows
     static constexpr int B_COLS = BN / CG;                    // filter columns staged by this CTA
     static constexpr int B_STAGE_BYTES = B_COLS * ROW_BYTES;  // = BK * B_COLS * ELT
-    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;   // written by TMA per stage
+    // KPS k-blocks travel together in one stage: [input tile of each k-block | filter tile: sub-tiles of
+    // KPS*BK k-rows], fetched by ONE load per operand (a TMA instruction costs the same whatever its size)
+    static constexpr int STAGE_BYTES = KPS * (A_STAGE_BYTES + B_STAGE_BYTES);   // written by TMA per stage
     // bf16: one ring of stages, TMA -> MMA.  f32: the TMA ring holds raw tiles; a second ring of
     // two slots holds what the converter warps make of them, [input hi | input lo | filter hi |
     // filter lo], the filter transposed to K-major on the way (kind::tf32 takes no N-major operand).
@@ -274,6 +276,7 @@ struct Cfg {
     static_assert(B_COLS % 64 == 0 && BN % 16 == 0 && BN <= 256, "tile width");
     static_assert(TMEM_COLS <= 512 && (TMEM_COLS & (TMEM_COLS - 1)) == 0, "TMEM columns");
     static_assert(STAGES >= 2 && STAGES <= 8, "ring depth");
+    static_assert(KPS == 1 || (KPS == 2 && !F32), "k-blocks per stage");
 };
 
 // Static tile order: groups of 8 tile-rows, row index fastest inside a group, so that the
@@ -346,6 +349,15 @@ __device__ __forceinline__ void tma_tile_5d(uint32_t dst, const CUtensorMap *map
         asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
                      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v) : "memory");
 }
+template <bool CG2>
+__device__ __forceinline__ void tma_tile_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z) {
+    if constexpr (CG2)
+        asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                     ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+    else
+        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                     ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
 // Starts the fetch of a tensor map (a kernel parameter) ahead of its first use.
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -371,11 +383,11 @@ __device__ __forceinline__ void umma_commit_cg2(uint32_t cluster_bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar) : "memory");
 }
 
-template <int BN, int CG, bool F32>
-__global__ void __launch_bounds__(Cfg<BN, CG, F32>::THREADS, 1)
+template <int BN, int CG, bool F32, int KPS>
+__global__ void __launch_bounds__(Cfg<BN, CG, F32, KPS>::THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_flt,
                const __grid_constant__ CUtensorMap map_out, const TcParams p) {
-    using C = Cfg<BN, CG, F32>;
+    using C = Cfg<BN, CG, F32, KPS>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -471,22 +483,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     pix_h = r / p.Wo;
                     pix_w = r - pix_h * p.Wo;
                 }
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                for (int kb = kb0; kb < kb1; kb += KPS, ++it) {
                     const int s = it % C::STAGES;
                     const uint32_t ph = (it / C::STAGES) & 1;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t a_dst = stages_addr + s * C::STAGE_BYTES;
-                    const uint32_t b_dst = a_dst + A_STAGE_BYTES;
+                    const uint32_t b_dst = a_dst + KPS * A_STAGE_BYTES;
                     const int tap = kb / p.kb_per_tap;
                     const int c0 = (kb - tap * p.kb_per_tap) * C::BK;
                     const int kh = tap / p.KW, kw = tap - kh * p.KW;
                     // bf16 pairs: the leader alone arms its barrier, for the pair's total (a remote arrive by
                     // the peer would order it after its own loads in flight and serialise the ring)
                     const uint32_t bar = REMOTE_FULL ? map_to_cta(full_bar(s), 0) : full_bar(s);
-                    const uint32_t my_bytes = input_side ? A_STAGE_BYTES : C::B_STAGE_BYTES;
+                    const uint32_t my_bytes = KPS * (input_side ? A_STAGE_BYTES : C::B_STAGE_BYTES);
                     if (!REMOTE_FULL || cta_rank == 0) mbar_expect_tx(full_bar(s), (REMOTE_FULL ? CG : 1) * my_bytes);
                     if (input_side) {
-                        if constexpr (!REMOTE_FULL) {
+                        if constexpr (KPS > 1) {
+                            // matmul only: the input map is blocked by k-blocks, box {BK, 128 rows, KPS k-blocks}
+                            tma_tile_3d<REMOTE_FULL>(a_dst, &map_in, bar, 0, m0, kb);
+                        } else if constexpr (!REMOTE_FULL) {
                             if (p.a_mode == 0) {
                                 tma_load_2d(a_dst, &map_in, bar, c0, m0);
                             } else if (p.a_mode == 1) {
@@ -506,7 +521,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                             }
                         }
                     } else if (p.b_blocked) {
-                        // box {sub-tile columns, BK channels, B_COLS / SUB_COLS column blocks, 1, 1}
+                        // box {sub-tile columns, KPS*BK channels, B_COLS / SUB_COLS column blocks, 1, 1}
                         tma_tile_5d<REMOTE_FULL>(b_dst, &map_flt, bar, 0, c0, n0 / C::SUB_COLS, kw, kh);
                     } else {
 #pragma unroll
@@ -538,7 +553,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 int tile, kb0, kb1;
                 item_range(t, tile, kb0, kb1);
-                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                for (int kb = kb0; kb < kb1; kb += KPS, ++it) {
                     if constexpr (F32) {
                         const int s = it & 1;
                         if (!mbar_wait<CG == 2>(split_full_bar(s), (it >> 1) & 1, abort_flag)) { ok = false; break; }
@@ -569,17 +584,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                         if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t a_addr = stages_addr + s * C::STAGE_BYTES;
-                        const uint32_t b_addr = a_addr + A_STAGE_BYTES;
-                        // input tile, K-major: 8-row groups are 1024 B apart; a k-step of 16 bf16 is 32 B
-                        // inside the swizzled 128-byte row.
-                        const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024);
-                        // filter tile, N-major: 64-column sub-tiles are SUB_BYTES apart (leading offset),
-                        // 8-row k groups 1024 B apart (stride offset); a k-step of 16 rows is 2048 B.
-                        const uint64_t b_desc = make_smem_desc(b_addr, C::SUB_BYTES, 1024);
+                        const uint32_t b_addr = a_addr + KPS * A_STAGE_BYTES;
 #pragma unroll
-                        for (int k = 0; k < K_STEPS; ++k)
-                            mma(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * C::B_KSTEP_DESC),
-                                (kb > kb0 || k > 0) ? 1u : 0u);
+                        for (int kbi = 0; kbi < KPS; ++kbi) {
+                            if (kb + kbi >= kb1) break;      // an odd k range ends inside its last stage
+                            // input tile, K-major: 8-row groups are 1024 B apart; a k-step of 16 bf16 is 32 B
+                            // inside the swizzled 128-byte row.
+                            const uint64_t a_desc = make_smem_desc(a_addr + kbi * A_STAGE_BYTES, 16, 1024);
+                            // filter tile, N-major: 64-column sub-tiles of KPS*BK k-rows are KPS*SUB_BYTES apart
+                            // (leading offset), 8-row k groups 1024 B apart (stride offset); a k-step of 16
+                            // rows is 2048 B, a k-block BK rows.
+                            const uint64_t b_desc = make_smem_desc(b_addr + kbi * C::SUB_BYTES, KPS * C::SUB_BYTES, 1024);
+#pragma unroll
+                            for (int k = 0; k < K_STEPS; ++k)
+                                mma(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * C::B_KSTEP_DESC),
+                                    (kb + kbi > kb0 || k > 0) ? 1u : 0u);
+                        }
                         // the stage is free (in every CTA of the group) once these MMAs have read it
                         if constexpr (CG == 1) {
                             umma_commit(empty_bar(s));
@@ -755,7 +775,7 @@ struct Driver {
     EncodeIm2colFn im2col = nullptr;
     int num_sms = 0;
     int device = -1;
-    bool attr_set[16] = {};
+    bool attr_set[24] = {};
     bool ok = false;
 };
 std::mutex g_mu;
@@ -763,6 +783,7 @@ Driver g_drv;
 int g_bn_override = -1;   // tile width forced by SG_TC_BN or sg_set_tile_override (-1: not read yet; 0: automatic)
 int g_cg_override = 0;    // CTAs per tile (0: automatic)
 int g_split_override = 0; // k ranges per tile (0: automatic)
+int g_kps_override = 0;   // SG_TC_KPS=1 (testing): one k-block per stage everywhere
 int g_last_choice[3] = {0, 0, 0};
 
 bool init_driver() {
@@ -819,15 +840,15 @@ double estimate_ns(const Variant &v, bool f32, int64_t tiles, int64_t groups, in
     return t;
 }
 
-template <int BN, int CG, bool F32>
+template <int BN, int CG, bool F32, int KPS>
 sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUtensorMap &mo, TcParams tp, int M, int N,
                          int slot, cudaStream_t stream) {
-  if constexpr (F32 && BN == 256 && CG == 1) {
+  if constexpr ((F32 && BN == 256 && CG == 1) || (KPS == 2 && (F32 || (BN == 256 && CG == 1)))) {
     return SG_ERR_INTERNAL;   // the split slots of a 128 x 256 f32 tile do not fit beside a TMA ring
   } else {
-    using C = Cfg<BN, CG, F32>;
+    using C = Cfg<BN, CG, F32, KPS>;
     if (!g_drv.attr_set[slot]) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, CG, F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, CG, F32, KPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
             return SG_ERR_CUDA;
         g_drv.attr_set[slot] = true;
     }
@@ -848,7 +869,7 @@ sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUt
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<BN, CG, F32>, mi, mf, mo, tp);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<BN, CG, F32, KPS>, mi, mf, mo, tp);
     count_launch();
     return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
   }
@@ -884,6 +905,8 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         g_cg_override = e ? atoi(e) : 0;
         e = getenv("SG_TC_SPLIT");
         g_split_override = e ? atoi(e) : 0;
+        e = getenv("SG_TC_KPS");
+        g_kps_override = e ? atoi(e) : 0;
     }
 
     alignas(64) CUtensorMap map_in, map_flt, map_out;
@@ -899,14 +922,7 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     CUresult r;
     // ---- input operand ----
     if (p.spatial_rank == 0) {
-        tp.a_mode = 0;
-        cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)p.M};
-        cuuint64_t strides[1] = {(cuuint64_t)(p.i_w * es)};
-        cuuint32_t box[2] = {(cuuint32_t)BK, BM};
-        r = g_drv.tiled(&map_in, in_type, 2, const_cast<void *>(In), dims, strides, box, ones,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
+        tp.a_mode = 0;      // the map is encoded below, once the tile variant is known
     } else {
         // im2col descriptors: the bounding box of base pixels is [0, used - (K-1)*d) per spatial
         // dimension, walked with the conv stride, which yields exactly W_out (H_out) base
@@ -1002,7 +1018,9 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
             // {sub_cols, BK, blocks of this CTA, 1, 1} is the CTA's whole filter tile of a k-block
             cuuint64_t dims[5] = {(cuuint64_t)sub_cols, (cuuint64_t)p.C, (cuuint64_t)(p.N / sub_cols), (cuuint64_t)p.KW, (cuuint64_t)p.KH};
             cuuint64_t strides[4] = {(cuuint64_t)(p.k_c * es), (cuuint64_t)ROW_BYTES, (cuuint64_t)(s_kw * es), (cuuint64_t)(s_kh * es)};
-            cuuint32_t box[5] = {(cuuint32_t)sub_cols, (cuuint32_t)BK, (cuuint32_t)(kVariants[pick].bn / kVariants[pick].cg / sub_cols), 1, 1};
+            // (bf16 matmuls with whole k-blocks fetch two k-blocks per load, see below)
+            const bool two = !f32 && p.spatial_rank == 0 && p.K % BK == 0 && !(kVariants[pick].bn == 256 && kVariants[pick].cg == 1) && g_kps_override != 1;
+            cuuint32_t box[5] = {(cuuint32_t)sub_cols, (cuuint32_t)(two ? 2 * BK : BK), (cuuint32_t)(kVariants[pick].bn / kVariants[pick].cg / sub_cols), 1, 1};
             r = g_drv.tiled(&map_flt, in_type, 5, const_cast<void *>(Flt), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         } else {
@@ -1015,18 +1033,43 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         }
         if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
     }
+    // bf16 matmuls with whole k-blocks move two k-blocks per stage and per TMA load
+    const int kps = (!f32 && p.spatial_rank == 0 && p.K % BK == 0 && tp.b_blocked &&
+                     !(kVariants[pick].bn == 256 && kVariants[pick].cg == 1) && g_kps_override != 1) ? 2 : 1;
+    if (p.spatial_rank == 0) {
+        if (kps == 2) {
+            // blocked by k-blocks: {k in block, m, k-block}, box {BK, 128, 2}
+            cuuint64_t dims[3] = {(cuuint64_t)BK, (cuuint64_t)p.M, (cuuint64_t)(p.K / BK)};
+            cuuint64_t strides[2] = {(cuuint64_t)(p.i_w * es), (cuuint64_t)ROW_BYTES};
+            cuuint32_t box[3] = {(cuuint32_t)BK, BM, 2};
+            r = g_drv.tiled(&map_in, in_type, 3, const_cast<void *>(In), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        } else {
+            cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)p.M};
+            cuuint64_t strides[1] = {(cuuint64_t)(p.i_w * es)};
+            cuuint32_t box[2] = {(cuuint32_t)BK, BM};
+            r = g_drv.tiled(&map_in, in_type, 2, const_cast<void *>(In), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        }
+        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
+    }
+    // k ranges are whole stages; every range keeps at least one k-block
+    int per = (tp.num_kb + splits - 1) / splits;
+    per = (per + kps - 1) / kps * kps;
+    splits = (tp.num_kb + per - 1) / per;
     tp.splits = splits;
-    tp.kb_per_split = (tp.num_kb + splits - 1) / splits;
+    tp.kb_per_split = per;
     if (splits > 1) {
         // partial sums meet in the output by TMA reduce-add: an overwriting call clears it first
         if (!p.accumulate && launch_zero_fill(p, O, stream) != cudaSuccess) return SG_ERR_CUDA;
         tp.accumulate = 1;
     }
     g_last_choice[0] = kVariants[pick].bn; g_last_choice[1] = kVariants[pick].cg; g_last_choice[2] = splits;
-    const int slot = pick + (f32 ? kNumVariants : 0);
-#define SG_LAUNCH(BN_, CG_)                                                                              \
-    (f32 ? launch_variant<BN_, CG_, true>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)          \
-         : launch_variant<BN_, CG_, false>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream))
+    const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0);
+#define SG_LAUNCH(BN_, CG_)                                                                                \
+    (f32 ? launch_variant<BN_, CG_, true, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)         \
+         : kps == 2 ? launch_variant<BN_, CG_, false, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)   \
+                    : launch_variant<BN_, CG_, false, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream))
     switch (pick) {
         case 0: return SG_LAUNCH(64, 1);
         case 1: return SG_LAUNCH(128, 1);
