@@ -812,14 +812,14 @@ inline bool mult(int64_t v, int64_t q) { return v % q == 0; }
 struct Variant { int bn, cg; double mma_ns, mma_ns_f32; };
 // Time one CTA's tensor core (bf16) or shared memory (f32: TMA fill, hi/lo split and the operand
 // reads of 12 MMAs share it) needs for one k-block of a tile, in ns.
-constexpr Variant kVariants[] = {{64, 1, 100.0, 750.0}, {128, 1, 135.0, 1000.0}, {256, 1, 270.0, 1500.0},
-                                 {128, 2, 135.0, 750.0}, {256, 2, 270.0, 1000.0}};
+constexpr Variant kVariants[] = {{64, 1, 100.0, 750.0}, {128, 1, 135.0, 1000.0}, {256, 1, 330.0, 1500.0},
+                                 {128, 2, 135.0, 750.0}, {256, 2, 330.0, 1000.0}};
 constexpr int kNumVariants = sizeof(kVariants) / sizeof(kVariants[0]);
 
 // Estimated kernel time in ns of `tiles` tiles dealt out in `sp` k ranges each over `groups`
 // CTAs or CTA pairs.  A k-block costs the slowest of: the CTA's own MMA / shared-memory
 // time, the CTA's share of the L2 -> shared memory fill rate of the whole chip (what bounds
-// every large problem here: about 10 TB/s), and the fill rate one SM reaches alone.  The
+// every large problem here: 9 to 14 TB/s), and the fill rate one SM reaches alone.  The
 // constants were fitted to timings of every variant and split on the 125 shapes
 // {256..4096}^3 in both dtypes; the choices they lead to are within 1 % of the best
 // per-shape choice in total time.
@@ -829,7 +829,7 @@ double estimate_ns(const Variant &v, bool f32, int64_t tiles, int64_t groups, in
     const int kbs = (num_kb + sp - 1) / sp;
     const double active = (double)((items < groups ? items : groups) * v.cg);
     const double stage_bytes = A_STAGE_BYTES + (double)(v.bn / v.cg) * ROW_BYTES;
-    const double chip_fill = f32 ? 9000.0 : 10500.0, sm_fill = f32 ? 40.0 : 90.0;      // bytes per ns
+    const double chip_fill = f32 ? 9000.0 : 14000.0, sm_fill = f32 ? 40.0 : 130.0;      // bytes per ns
     double kb_ns = f32 ? v.mma_ns_f32 : v.mma_ns;
     if (active * stage_bytes / chip_fill > kb_ns) kb_ns = active * stage_bytes / chip_fill;
     if (stage_bytes / sm_fill > kb_ns) kb_ns = stage_bytes / sm_fill;
