@@ -358,6 +358,12 @@ __device__ __forceinline__ void tma_tile_3d(uint32_t dst, const CUtensorMap *map
         asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
 }
+// True in exactly one lane of the (converged) warp, the same lane on every call.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
 // Starts the fetch of a tensor map (a kernel parameter) ahead of its first use.
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -535,20 +541,37 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && cta_rank == 0) {
+        // The whole warp walks the loop, so that addresses and descriptors are warp-uniform values;
+        // one elected lane issues the MMAs and the commits (a loop run by a single lane of a
+        // diverged warp pays for moving every descriptor out of per-lane registers: measured
+        // ~120 cycles per MMA, as much as a 128 x 256 x 16 MMA takes to execute).
+        if (cta_rank == 0) {
             constexpr uint32_t idesc = make_idesc(BN, CG * BM, F32);
+            const bool issuer = elect_one();
+            auto wait_all = [&](bool passed) { return __all_sync(0xffffffffu, passed) != 0; };
             auto mma = [&](uint32_t d, uint64_t ad, uint64_t bd, uint32_t acc) {
+                if (!issuer) return;
                 if constexpr (F32) {
                     if constexpr (CG == 1) umma_tf32(d, ad, bd, idesc, acc); else umma_tf32_cg2(d, ad, bd, idesc, acc);
                 } else {
                     if constexpr (CG == 1) umma_bf16(d, ad, bd, idesc, acc); else umma_bf16_cg2(d, ad, bd, idesc, acc);
                 }
             };
+            // arrive, once the MMAs issued so far have finished, on the same barrier of every CTA of the group
+            auto commit_all = [&](uint32_t bar) {
+                if (!issuer) return;
+                if constexpr (CG == 1) {
+                    umma_commit(bar);
+                } else {
+                    umma_commit_cg2(map_to_cta(bar, 0));
+                    umma_commit_cg2(map_to_cta(bar, 1));
+                }
+            };
             int it = 0, tl = 0;
             bool ok = true;
             for (int t = group_id; t < num_tiles && ok; t += num_groups, ++tl) {
                 const int buf = tl & 1;
-                if (!mbar_wait(acc_empty_bar(buf), ((tl >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
+                if (!wait_all(mbar_wait(acc_empty_bar(buf), ((tl >> 1) & 1) ^ 1u, abort_flag))) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 int tile, kb0, kb1;
@@ -556,7 +579,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                 for (int kb = kb0; kb < kb1; kb += KPS, ++it) {
                     if constexpr (F32) {
                         const int s = it & 1;
-                        if (!mbar_wait<CG == 2>(split_full_bar(s), (it >> 1) & 1, abort_flag)) { ok = false; break; }
+                        if (!wait_all(mbar_wait<CG == 2>(split_full_bar(s), (it >> 1) & 1, abort_flag))) { ok = false; break; }
                         tc_fence_after();
                         // slot: [input hi | input lo | filter hi | filter lo], all K-major: 8-row groups
                         // 1024 B apart, a k-step of 8 f32 is 32 B inside the swizzled 128-byte row
@@ -572,16 +595,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                             mma(d_tmem, ah + o, bl + o, 1u);
                             mma(d_tmem, ah + o, bh + o, 1u);
                         }
-                        if constexpr (CG == 1) {
-                            umma_commit(split_empty_bar(s));
-                        } else {
-                            umma_commit_cg2(map_to_cta(split_empty_bar(s), 0));
-                            umma_commit_cg2(map_to_cta(split_empty_bar(s), 1));
-                        }
+                        commit_all(split_empty_bar(s));
                     } else {
                         const int s = it % C::STAGES;
                         const uint32_t ph = (it / C::STAGES) & 1;
-                        if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                        if (!wait_all(mbar_wait(full_bar(s), ph, abort_flag))) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t a_addr = stages_addr + s * C::STAGE_BYTES;
                         const uint32_t b_addr = a_addr + KPS * A_STAGE_BYTES;
@@ -601,22 +619,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                                     (kb + kbi > kb0 || k > 0) ? 1u : 0u);
                         }
                         // the stage is free (in every CTA of the group) once these MMAs have read it
-                        if constexpr (CG == 1) {
-                            umma_commit(empty_bar(s));
-                        } else {
-                            umma_commit_cg2(map_to_cta(empty_bar(s), 0));
-                            umma_commit_cg2(map_to_cta(empty_bar(s), 1));
-                        }
+                        commit_all(empty_bar(s));
                     }
                 }
-                if (ok) {
-                    if constexpr (CG == 1) {
-                        umma_commit(acc_full_bar(buf));
-                    } else {
-                        umma_commit_cg2(map_to_cta(acc_full_bar(buf), 0));
-                        umma_commit_cg2(map_to_cta(acc_full_bar(buf), 1));
-                    }
-                }
+                if (ok) commit_all(acc_full_bar(buf));
             }
         }
     } else if (warp >= 6) {
