@@ -212,16 +212,18 @@ def measure_op(sg, peaks, spec, reps=None):
     host_ms = time_launches(lambda i: call(*bufs[i % sets]), max(3, min(100, ncalls * 2)), 2)
     tf = flops / (ms * 1e-3) / 1e12
     tensor_peak = peaks["bf16_tflops"] * (TF32_OVER_BF16 if dtype == "f32" else 1.0)
-    t_compute = flops / ((tensor_peak if fam == sg.SG_KERNEL_TENSOR else ffma_peak) * 1e12)
+    on_tensor = fam in (sg.SG_KERNEL_TENSOR, sg.SG_KERNEL_CONV_STRIP)
+    kernel_name = {sg.SG_KERNEL_TENSOR: "tensor", sg.SG_KERNEL_CONV_STRIP: "tensor (conv strip)"}.get(fam, "ffma")
+    t_compute = flops / ((tensor_peak if on_tensor else ffma_peak) * 1e12)
     t_bytes = bytes_ / (peaks["hbm_gbs"] * 1e9)
     bound = max(t_compute, t_bytes)
-    row = {"op": label, "dtype": dtype, "kernel": "tensor" if fam == sg.SG_KERNEL_TENSOR else "ffma",
+    row = {"op": label, "dtype": dtype, "kernel": kernel_name,
            "us": round(ms * 1e3, 2), "us_with_host_call": round(host_ms * 1e3, 2), "gflops": round(tf * 1e3, 1),
            "gbs": round(bytes_ / (ms * 1e-3) / 1e9, 1),
-           "bound": "hbm" if t_bytes > t_compute else ("tensor" if fam == sg.SG_KERNEL_TENSOR else "ffma"),
+           "bound": "hbm" if t_bytes > t_compute else ("tensor" if on_tensor else "ffma"),
            "roofline_us": round(bound * 1e6, 2), "frac": round(bound / (ms * 1e-3), 4), "rotating_sets": sets,
            "timing": "CUDA graph replay"}
-    if dtype == "f32" and fam == sg.SG_KERNEL_TENSOR:
+    if dtype == "f32" and on_tensor:
         # the f32 path issues three tf32 products per term: its own ceiling is a third of the tf32 peak
         row["frac_of_3xtf32_ceiling"] = round(max(3 * t_compute, t_bytes) / (ms * 1e-3), 4)
     del bufs, calls

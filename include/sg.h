@@ -63,7 +63,13 @@ typedef enum { SG_F32 = 0, SG_BF16 = 1 } sg_dtype;
 enum { SG_OVERWRITE = 0, SG_ACCUMULATE = 1 };
 
 /* Kernel families, for sg_set_kernel_override(). */
-enum { SG_KERNEL_AUTO = 0, SG_KERNEL_FFMA = 1, SG_KERNEL_TENSOR = 2 };
+enum {
+    SG_KERNEL_AUTO = 0,
+    SG_KERNEL_FFMA = 1,        /* strided CUDA-core kernel, any layout                                   */
+    SG_KERNEL_TENSOR = 2,      /* TMA + tcgen05 implicit GEMM (matmul; convolutions through TMA im2col)  */
+    SG_KERNEL_CONV_STRIP = 3   /* tcgen05 kernel for stride-1 bf16 convolutions: resident filter, each
+                                  input pixel fetched once per tile                                      */
+};
 
 /*
  * Matrix multiplication (paper Section 4.6.1, variant "AB"; iterators
@@ -133,7 +139,7 @@ int sg_version(void);
 
 /*
  * Which kernel family the most recent successful call on this host thread
- * selected: SG_KERNEL_FFMA or SG_KERNEL_TENSOR (0 before any call).
+ * selected: SG_KERNEL_FFMA, SG_KERNEL_TENSOR or SG_KERNEL_CONV_STRIP (0 before any call).
  */
 int sg_last_kernel(void);
 
@@ -145,9 +151,11 @@ int64_t sg_launch_count(void);
 
 /*
  * Force a kernel family for later calls on this process (testing and
- * benchmarking): SG_KERNEL_AUTO restores the default selection.  Forcing
- * SG_KERNEL_TENSOR makes calls whose layout the tensor-core path cannot take
- * return SG_ERR_UNSUPPORTED instead of falling back.
+ * benchmarking): SG_KERNEL_AUTO restores the default selection (the
+ * convolution kernel where it applies, else the tensor-core GEMM, else the
+ * CUDA-core kernel).  Forcing SG_KERNEL_TENSOR or SG_KERNEL_CONV_STRIP makes
+ * calls that kernel cannot take return SG_ERR_UNSUPPORTED instead of falling
+ * back.
  */
 sg_status sg_set_kernel_override(int kernel_family);
 

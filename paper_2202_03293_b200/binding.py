@@ -19,7 +19,7 @@ _lib = None
 SG_OK = 0
 SG_F32, SG_BF16 = 0, 1
 SG_OVERWRITE, SG_ACCUMULATE = 0, 1
-SG_KERNEL_AUTO, SG_KERNEL_FFMA, SG_KERNEL_TENSOR = 0, 1, 2
+SG_KERNEL_AUTO, SG_KERNEL_FFMA, SG_KERNEL_TENSOR, SG_KERNEL_CONV_STRIP = 0, 1, 2, 3
 
 EXPORTS = [
     "sg_matmul", "sg_conv1d_nwc_wcf", "sg_conv2d_nhwc_hwcf", "sg_check", "sg_status_string",

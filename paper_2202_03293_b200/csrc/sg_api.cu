@@ -22,6 +22,12 @@ sg_status run(const Problem &p, const void *In, const void *Flt, float *O, cudaS
         return launch_zero_fill(p, O, stream) == cudaSuccess ? SG_OK : SG_ERR_CUDA;
     }
     const int force = g_override.load();
+    if (force == SG_KERNEL_AUTO || force == SG_KERNEL_CONV_STRIP) {
+        // stride-1 bf16 convolutions whose filter fits in shared memory
+        sg_status st = launch_conv_strip(p, In, Flt, O, stream);
+        if (st == SG_OK) { t_last_kernel = SG_KERNEL_CONV_STRIP; return SG_OK; }
+        if (st != SG_ERR_UNSUPPORTED || force == SG_KERNEL_CONV_STRIP) return st;
+    }
     if (force != SG_KERNEL_FFMA) {
         sg_status st = launch_tensor(p, In, Flt, O, stream);
         if (st == SG_OK) { t_last_kernel = SG_KERNEL_TENSOR; return SG_OK; }
@@ -170,7 +176,8 @@ int sg_last_kernel(void) { return t_last_kernel; }
 int64_t sg_launch_count(void) { return g_launches.load(); }
 
 sg_status sg_set_kernel_override(int kernel_family) {
-    if (kernel_family != SG_KERNEL_AUTO && kernel_family != SG_KERNEL_FFMA && kernel_family != SG_KERNEL_TENSOR)
+    if (kernel_family != SG_KERNEL_AUTO && kernel_family != SG_KERNEL_FFMA && kernel_family != SG_KERNEL_TENSOR &&
+        kernel_family != SG_KERNEL_CONV_STRIP)
         return SG_ERR_INVALID_ARG;
     g_override.store(kernel_family);
     return SG_OK;

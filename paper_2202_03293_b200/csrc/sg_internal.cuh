@@ -1,6 +1,7 @@
 // Shared declarations of the CUDA side of the library (not part of the C ABI).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -40,6 +41,17 @@ cudaError_t launch_zero_fill(const Problem &p, float *O, cudaStream_t stream);
 sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float *O,
                         cudaStream_t stream);
 void tensor_shutdown();
+// Driver entry points resolved by the tensor path, for the other tensor-core kernels: whether the
+// current device is usable (and its SM count), and a tiled tensor-map encoder (interleave none,
+// element strides 1, out-of-bounds elements read as zero).  Call with no library lock held.
+bool tensor_driver_ready(int *num_sms);
+bool tensor_encode_tiled(CUtensorMap *map, CUtensorMapDataType type, int rank, void *base, const cuuint64_t *dims,
+                         const cuuint64_t *strides, const cuuint32_t *box, CUtensorMapSwizzle swizzle,
+                         CUtensorMapL2promotion promotion);
+// Stride-1 bf16 convolutions with a resident filter (sg_conv.cu): SG_ERR_UNSUPPORTED when the
+// shape or layout does not qualify (nothing is launched then).
+sg_status launch_conv_strip(const Problem &p, const void *In, const void *Flt, float *O, cudaStream_t stream);
+sg_status conv_read_status(cudaStream_t stream);
 void tensor_set_tile_override(int bn, int cg, int splits);
 void tensor_last_choice(int out[3]);
 // Reads and clears the current device's status word (written by kernels whose bounded

@@ -37,6 +37,7 @@
 #include <mutex>
 
 #include "sg_internal.cuh"
+#include "sg_tc_ptx.cuh"
 
 namespace sg {
 namespace {
@@ -47,9 +48,7 @@ constexpr int K_STEPS = 4;        // tcgen05.mma per k-block and product: 32 byt
 constexpr int A_STAGE_BYTES = BM * ROW_BYTES;
 constexpr int CONVERTER_THREADS = 256;        // f32 path: 8 warps splitting tiles into hi and lo
 constexpr int STAGING_BYTES = 4 * 2 * 4096;   // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
-constexpr long long WAIT_BUDGET_CYCLES = 2000000000LL;   // ~1 s: far beyond any legitimate wait
 
-__device__ unsigned int g_status_word = 0;
 
 struct TcParams {
     int M, N;
@@ -64,160 +63,6 @@ struct TcParams {
     int accumulate;
     int b_blocked;       // 1: the filter map is blocked by sub-tile columns: one TMA load fetches the whole filter tile
 };
-
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Same test with cluster-scope acquire: the barrier was signalled by threads of the peer CTA
-// whose shared-memory writes must be visible afterwards.
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false when the budget expired or another role already aborted.
-template <bool CLUSTER_SCOPE = false>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    auto test = [&]() { return CLUSTER_SCOPE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
-    if (test()) return true;
-    const long long t0 = clock64();
-    for (uint32_t it = 0;; ++it) {
-        if (test()) return true;
-        if ((it & 63u) == 63u) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_BUDGET_CYCLES) {
-                *abort_flag = 1;
-                atomicOr(&g_status_word, 1u);
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z, int w) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
-}
-// im2col mode: coordinates name the first base pixel (c, w, [h,] n); the 16-bit offsets are
-// added to every pixel's spatial coordinates (the filter tap's kw*dw, kh*dh).
-__device__ __forceinline__ void tma_load_im2col_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
-                                                   int c, int w, int n, unsigned short off_w) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2], {%6};"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(n), "h"(off_w) : "memory");
-}
-__device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar,
-                                                   int c, int w, int h, int n, unsigned short off_w, unsigned short off_h) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
-}
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, uint32_t src, int x, int y) {
-    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// D[tmem] (+)= A[smem] * B[smem], 128 x N x 16, bf16 inputs, f32 accumulate.
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// Same shape with tf32 inputs (f32 words in shared memory, k extent 8).
-__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// Arrives on the mbarrier once every tcgen05.mma issued so far by this thread has finished.
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// This warp's 32 lanes x 32 consecutive f32 columns of TMEM -> 32 registers per thread.
-__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor (sm_100 format): start address, leading and stride byte
-// offsets (all >> 4), descriptor version 1, 128-byte swizzle.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-    d |= (uint64_t)1 << 46;   // version
-    d |= (uint64_t)2 << 61;   // SWIZZLE_128B
-    return d;
-}
-
-// Instruction descriptor: f32 accumulator, A and B both bf16 (kind::f16) or both tf32
-// (kind::tf32), A K-major, B N-major.
-__host__ __device__ constexpr uint32_t make_idesc(int n, int m, bool tf32) {
-    return (1u << 4)                       // D format: f32
-         | ((tf32 ? 2u : 1u) << 7)         // A format: bf16 = 1 in kind::f16, tf32 = 2 in kind::tf32
-         | ((tf32 ? 2u : 1u) << 10)        // B format: the same type as A
-         | (0u << 15)                      // A major: K
-         | ((tf32 ? 0u : 1u) << 16)        // B major: MN for bf16 (filter stored [k][f], f contiguous, read as
-                                           // is); kind::tf32 takes K-major operands only (an N-major
-                                           // descriptor makes the MMA a no-op), so the f32 path
-                                           // transposes the filter tile while splitting it
-         | ((uint32_t)(n >> 3) << 17)      // N / 8
-         | ((uint32_t)(m >> 4) << 24);     // M / 16 (128 for one CTA, 256 for a pair)
-}
 
 // 3xTF32 split of four f32 words.  hi = x rounded to the nearest tf32 value (10 mantissa bits;
 // done on the bit pattern: add half an ulp, clear the low 13 bits); x - hi is exact in f32 and
@@ -289,104 +134,6 @@ __device__ __forceinline__ void tile_coords(int t, int num_m_tiles, int num_n_ti
     if (rows > GM) rows = GM;
     nt = r / rows;
     mt = g * GM + (r - nt * rows);
-}
-
-// ---- cluster helpers (CG = 2) ----
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-// shared::cluster address of the same shared-memory offset in CTA `rank` of this cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-    return r;
-}
-// Arrive on a barrier of another CTA of the cluster.  Default semantics (release at CTA scope):
-// what the arriving thread wrote before goes to its own CTA's shared memory, which the
-// tensor core reads after a proxy fence; a cluster-scope release costs a full memory barrier
-// per arrive (measured: 1.6x on the whole f32 kernel) and orders nothing more that is needed.
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// TMA loads whose completion may be signalled on the peer CTA's mbarrier (cta_group::2).
-__device__ __forceinline__ void tma_load_2d_cg2(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void tma_load_4d_cg2(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z, int w) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
-}
-__device__ __forceinline__ void tma_load_im2col_3d_cg2(uint32_t dst, const CUtensorMap *map, uint32_t bar,
-                                                       int c, int w, int n, unsigned short off_w) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2], {%6};"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(n), "h"(off_w) : "memory");
-}
-__device__ __forceinline__ void tma_load_im2col_4d_cg2(uint32_t dst, const CUtensorMap *map, uint32_t bar,
-                                                       int c, int w, int h, int n, unsigned short off_w, unsigned short off_h) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
-}
-// Rank-5 tiled load.  CG2: the mbarrier may belong to the peer CTA of a pair.  One TMA
-// instruction costs the issuing thread several hundred cycles whatever the size of its box
-// (measured: ~550 cycles, boxes of 8 to 64 KB), so operand tiles are fetched with as few and as
-// large boxes as the layout allows, and the two operands are issued by different warps.
-template <bool CG2>
-__device__ __forceinline__ void tma_tile_5d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z, int w, int v) {
-    if constexpr (CG2)
-        asm volatile("cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-                     ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v) : "memory");
-    else
-        asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-                     ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v) : "memory");
-}
-template <bool CG2>
-__device__ __forceinline__ void tma_tile_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z) {
-    if constexpr (CG2)
-        asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-                     ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
-    else
-        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-                     ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
-}
-// True in exactly one lane of the (converged) warp, the same lane on every call.
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred;
-    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
-    return pred != 0;
-}
-// Starts the fetch of a tensor map (a kernel parameter) ahead of its first use.
-__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
-}
-// D[tmem of both CTAs] (+)= A * B, 256 x N x 16 across the CTA pair.
-__device__ __forceinline__ void umma_bf16_cg2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_tf32_cg2(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// Arrives (once the pair's MMAs issued so far have finished) on a barrier that may live in
-// either CTA of the pair; `cluster_bar` is a shared::cluster address.
-__device__ __forceinline__ void umma_commit_cg2(uint32_t cluster_bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(cluster_bar) : "memory");
 }
 
 template <int BN, int CG, bool F32, int KPS>
@@ -1087,17 +834,30 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
 }
 
 sg_status tensor_read_status(cudaStream_t stream) {
-    unsigned int word = 0, zero = 0;
-    if (cudaMemcpyFromSymbolAsync(&word, g_status_word, sizeof(word), 0, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
-        return SG_ERR_CUDA;
-    if (cudaStreamSynchronize(stream) != cudaSuccess) return SG_ERR_CUDA;
-    if (word != 0) {
-        if (cudaMemcpyToSymbolAsync(g_status_word, &zero, sizeof(zero), 0, cudaMemcpyHostToDevice, stream) != cudaSuccess)
-            return SG_ERR_CUDA;
-        cudaStreamSynchronize(stream);
-        return SG_ERR_DEVICE_TIMEOUT;
+    const sg_status a = read_status_word(stream);
+    const sg_status b = conv_read_status(stream);
+    return a != SG_OK ? a : b;
+}
+
+bool tensor_driver_ready(int *num_sms) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!init_driver()) return false;
+    if (num_sms) *num_sms = g_drv.num_sms;
+    return true;
+}
+
+bool tensor_encode_tiled(CUtensorMap *map, CUtensorMapDataType type, int rank, void *base, const cuuint64_t *dims,
+                         const cuuint64_t *strides, const cuuint32_t *box, CUtensorMapSwizzle swizzle,
+                         CUtensorMapL2promotion promotion) {
+    const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+    EncodeTiledFn fn;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (!init_driver()) return false;
+        fn = g_drv.tiled;
     }
-    return SG_OK;
+    return fn(map, type, (cuuint32_t)rank, base, dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, promotion,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 void tensor_set_tile_override(int bn, int cg, int splits) {

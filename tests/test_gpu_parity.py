@@ -11,7 +11,7 @@ from paper_2202_03293_b200 import inputs
 
 pytestmark = pytest.mark.gpu
 SEED = inputs.BASE_SEED
-FFMA, TENSOR = sg.SG_KERNEL_FFMA, sg.SG_KERNEL_TENSOR
+FFMA, TENSOR, STRIP = sg.SG_KERNEL_FFMA, sg.SG_KERNEL_TENSOR, sg.SG_KERNEL_CONV_STRIP
 
 
 @pytest.fixture(autouse=True)
@@ -314,8 +314,11 @@ def test_c3_conv1d_f32_full(family):
 def test_c4_conv2d_bf16_full():
     # config 4: N=16, H=W=58, C=64, 3x3, F=128, stride 1, bf16 in / f32 out, N(0,1)
     O, want, S = run_conv2d(16, 56, 56, 64, 3, 3, 128, (1, 1), (1, 1), "bf16", seed=SEED + 3)
-    assert sg.sg_last_kernel() == TENSOR
+    assert sg.sg_last_kernel() == STRIP
     assert_within_bound(O, want, S, "conv2d config 4")
+    O, want, S = run_conv2d(16, 56, 56, 64, 3, 3, 128, (1, 1), (1, 1), "bf16", family=TENSOR, seed=SEED + 3)
+    assert sg.sg_last_kernel() == TENSOR
+    assert_within_bound(O, want, S, "conv2d config 4, im2col kernel")
 
 
 @pytest.mark.parametrize("family", [FFMA, TENSOR])
@@ -339,6 +342,54 @@ def test_conv2d_bf16(family, N, Ho, Wo, C, KH, KW, F, st, dl):
     O, want, S = run_conv2d(N, Ho, Wo, C, KH, KW, F, st, dl, "bf16", family=family, seed=SEED + 5)
     assert sg.sg_last_kernel() == family
     assert_within_bound(O, want, S, "conv2d bf16")
+
+
+# the stride-1 kernel with a resident filter: ragged channels and columns, dilations, tiles that
+# wrap over image rows and images, 1-D and 2-D, more than one column tile
+@pytest.mark.parametrize("N,Ho,Wo,C,KH,KW,F,dl", [(3, 20, 20, 64, 3, 3, 128, (1, 1)), (4, 13, 17, 72, 2, 3, 40, (1, 1)),
+                                                   (3, 21, 18, 64, 3, 2, 72, (2, 2)), (2, 30, 40, 136, 1, 3, 64, (1, 3)),
+                                                   (5, 7, 40, 24, 3, 1, 200, (1, 1)), (1, 1, 300, 64, 1, 1, 128, (1, 1))])
+@pytest.mark.parametrize("accumulate", [False, True])
+def test_conv2d_strip_kernel(N, Ho, Wo, C, KH, KW, F, dl, accumulate):
+    O, want, S = run_conv2d(N, Ho, Wo, C, KH, KW, F, (1, 1), dl, "bf16", family=STRIP, accumulate=accumulate, seed=SEED + 14)
+    assert sg.sg_last_kernel() == STRIP
+    assert_within_bound(O, want, S, "conv2d strip kernel")
+
+
+@pytest.mark.parametrize("N,Wo,C,KW,F,dw", [(4, 300, 64, 3, 128, 1), (3, 333, 72, 5, 40, 1), (2, 411, 128, 3, 72, 2), (1, 5000, 64, 7, 64, 4)])
+def test_conv1d_strip_kernel(N, Wo, C, KW, F, dw):
+    O, want, S = run_conv1d(N, Wo, C, KW, F, 1, dw, "bf16", family=STRIP, seed=SEED + 15, extra_w=3)
+    assert sg.sg_last_kernel() == STRIP
+    assert_within_bound(O, want, S, "conv1d strip kernel")
+
+
+def test_conv_strip_kernel_changes_filter_inside_a_cta():
+    # two column tiles and an odd number of position tiles, more items than CTA groups: some
+    # group's run of items straddles the column tiles, so it reloads its resident filter
+    O, want, S = run_conv2d(2, 79, 79, 64, 3, 3, 200, (1, 1), (1, 1), "bf16", family=STRIP, seed=SEED + 16)
+    assert sg.sg_last_kernel() == STRIP
+    assert_within_bound(O, want, S, "two column tiles")
+
+
+def test_conv_strip_kernel_exact_and_rejections():
+    O, want, S = run_conv2d(2, 24, 24, 64, 3, 3, 64, (1, 1), (1, 1), "bf16", family=STRIP, dist="ints", seed=SEED + 7)
+    assert np.array_equal(O.cpu().numpy().astype(np.float64), want)
+    # strided convolutions, f32 inputs and filters beyond shared memory are not this kernel's
+    I = torch.zeros(1, 40, 40, 64, device="cuda", dtype=torch.bfloat16)
+    Kf = torch.zeros(3, 3, 64, 64, device="cuda", dtype=torch.bfloat16)
+    sg.sg_set_kernel_override(STRIP)
+    with pytest.raises(sg.SgError):
+        sg.sg_conv2d_nhwc_hwcf(I, Kf, torch.empty(1, 19, 19, 64, device="cuda"), (2, 2), (1, 1))
+    with pytest.raises(sg.SgError):
+        sg.sg_conv2d_nhwc_hwcf(I.float(), Kf.float(), torch.empty(1, 38, 38, 64, device="cuda"))
+    big = torch.zeros(3, 3, 512, 128, device="cuda", dtype=torch.bfloat16)
+    with pytest.raises(sg.SgError):
+        sg.sg_conv2d_nhwc_hwcf(torch.zeros(1, 40, 40, 512, device="cuda", dtype=torch.bfloat16), big,
+                               torch.empty(1, 38, 38, 128, device="cuda"))
+    sg.sg_set_kernel_override(sg.SG_KERNEL_AUTO)
+    sg.sg_conv2d_nhwc_hwcf(torch.zeros(1, 40, 40, 512, device="cuda", dtype=torch.bfloat16), big,
+                           torch.empty(1, 38, 38, 128, device="cuda"))
+    assert sg.sg_last_kernel() == TENSOR        # falls back to the im2col kernel
 
 
 @pytest.mark.parametrize("N,Ho,Wo,C,KH,KW,F,st,dl", [(1, 5, 6, 3, 2, 3, 5, (1, 1), (1, 1)), (2, 9, 7, 32, 3, 3, 64, (1, 2), (2, 1)),
@@ -390,10 +441,11 @@ def test_conv_delta_filter_is_a_shift_on_gpu():
     Kf = torch.zeros(3, 3, C, C, device="cuda", dtype=torch.bfloat16)
     Kf[2, 1] = torch.eye(C, device="cuda", dtype=torch.bfloat16)
     O = torch.empty(N, H - 2, W - 2, C, device="cuda")
-    for fam in (FFMA, TENSOR):
+    for fam in (FFMA, TENSOR, STRIP):
         sg.sg_set_kernel_override(fam)
         O.fill_(float("nan"))
         sg.sg_conv2d_nhwc_hwcf(I, Kf, O)
+        assert sg.sg_last_kernel() == fam
         torch.cuda.synchronize()
         assert torch.equal(O, I[:, 2:H, 1:W - 1, :].float())
 
