@@ -218,6 +218,16 @@ __global__ void zero_fill_kernel(Problem p, float *__restrict__ O) {
     }
 }
 
+// The output as one M x N matrix of contiguous, 16-byte aligned rows `pitch` floats apart
+// (what the tensor-core path requires of it): four columns per thread.
+__global__ void zero_fill_rows_kernel(float *__restrict__ O, int M, int n4, int64_t pitch) {
+    const int64_t total = (int64_t)M * n4;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int m = (int)(i / n4), c = (int)(i - (int64_t)m * n4);
+        reinterpret_cast<float4 *>(O + (int64_t)m * pitch)[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+}
+
 inline bool mult_of(int64_t v, int64_t q) { return v % q == 0; }
 
 template <typename T>
@@ -250,6 +260,15 @@ cudaError_t launch_ffma(const Problem &p, const void *In, const void *Flt, float
 }
 
 cudaError_t launch_zero_fill(const Problem &p, float *O, cudaStream_t stream) {
+    const bool uniform_rows = p.o_f == 1 && (p.Ho == 1 || p.o_h == (int64_t)p.Wo * p.o_w) &&
+                              (p.batch == 1 || p.o_n == (int64_t)p.Ho * p.Wo * p.o_w);
+    if (uniform_rows && p.N % 4 == 0 && p.o_w % 4 == 0 && reinterpret_cast<uintptr_t>(O) % 16 == 0) {
+        const int64_t work = (int64_t)p.M * (p.N / 4);
+        const int blocks = (int)((work + 255) / 256 < 148 * 8 ? (work + 255) / 256 : 148 * 8);
+        zero_fill_rows_kernel<<<blocks, 256, 0, stream>>>(O, p.M, p.N / 4, p.o_w);
+        count_launch();
+        return cudaGetLastError();
+    }
     int64_t total = (int64_t)p.M * p.N;
     int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
     zero_fill_kernel<<<blocks, 256, 0, stream>>>(p, O);
