@@ -47,7 +47,7 @@ constexpr int ROW_BYTES = 128;    // one k-block = one 128-byte swizzle row: 64 
 constexpr int K_STEPS = 4;        // tcgen05.mma per k-block and product: 32 bytes of k each
 constexpr int A_STAGE_BYTES = BM * ROW_BYTES;
 constexpr int CONVERTER_THREADS = 256;        // f32 path: 8 warps splitting tiles into hi and lo
-constexpr int STAGING_BYTES = 4 * 2 * 4096;   // 4 epilogue warps x 2 buffers x (32 rows x 128 B)
+constexpr int STAGING_BYTES = 2 * 16384;      // epilogue: 2 staging tiles of 128 rows x 128 B
 
 
 struct TcParams {
@@ -446,9 +446,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         }
     } else {
         // ------------------------------------------------------------ epilogue
-        const int q = warp & 3;   // TMEM lane quarter this warp may access
-        const uint32_t stg_addr = staging_addr + (warp - 2) * 8192;
-        uint8_t *stg_gen = staging_gen + (warp - 2) * 8192;
+        // The four warps share two staging tiles of 128 rows x 32 columns (16 KB, 128-byte swizzle):
+        // each writes its TMEM lane quarter's rows, then ONE TMA store (or reduce-add) moves the
+        // whole 128 x 32 chunk, issued by the warps in turn: a TMA instruction costs its thread
+        // about as much for 16 KB as for 4 KB.
+        const int q = warp & 3;        // TMEM lane quarter this warp may access
+        const int ew = warp - 2;       // 0..3: whose turn it is to issue
+        auto epi_sync = [] { asm volatile("bar.sync 1, 128;" ::: "memory"); };
         int tl = 0, chunk_count = 0;
         bool ok = true;
         for (int t = group_id; t < num_tiles && ok; t += num_groups, ++tl) {
@@ -456,6 +460,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
             tile_coords(t / p.splits, p.num_m_tiles, p.num_n_tiles, mt, nt);
             const int m0 = (mt * CG + (int)cta_rank) * BM, n0 = nt * BN;
             const int buf = tl & 1;
+            // (the barrier's phase stays complete until these warps hand the buffer back, so the four
+            // warps take the same way here and meet at every epi_sync below)
             if (!mbar_wait(acc_full_bar(buf), (tl >> 1) & 1, abort_flag)) { ok = false; break; }
             tc_fence_after();
 #pragma unroll 1
@@ -464,22 +470,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                 tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + j * 32), r);
                 tmem_ld_wait();
                 const int sb = chunk_count & 1;
-                // the bulk store issued two chunks ago must have finished reading this buffer
-                if (lane == 0) bulk_wait_read<1>();
-                __syncwarp();
-                uint8_t *row = stg_gen + sb * 4096 + lane * 128;
+                // staging tile sb was last read by the store of two chunks ago, whose issuer waited for
+                // that read before the previous chunk's epi_sync
+                uint8_t *row = staging_gen + sb * 16384 + (q * 32 + lane) * 128;
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     uint4 v = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
                     *reinterpret_cast<uint4 *>(row + ((c ^ (lane & 7)) << 4)) = v;
                 }
                 fence_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    const int x = n0 + j * 32, y = m0 + q * 32;
-                    if (x < p.N && y < p.M) {
-                        if (p.accumulate) tma_reduce_add_2d(&map_out, stg_addr + sb * 4096, x, y);
-                        else tma_store_2d(&map_out, stg_addr + sb * 4096, x, y);
+                // the issuer of the previous chunk's store makes sure that store has read its tile
+                if (lane == 0 && ew == ((chunk_count + 3) & 3)) bulk_wait_read<0>();
+                epi_sync();
+                if (lane == 0 && ew == (chunk_count & 3)) {
+                    const int x = n0 + j * 32;
+                    if (x < p.N && m0 < p.M) {
+                        if (p.accumulate) tma_reduce_add_2d(&map_out, staging_addr + sb * 16384, x, m0);
+                        else tma_store_2d(&map_out, staging_addr + sb * 16384, x, m0);
                     }
                     bulk_commit();
                 }
@@ -713,11 +720,11 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         }
         if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
     }
-    // ---- output: 2-D {f, m} f32, stored in 32 x 32 boxes ----
+    // ---- output: 2-D {f, m} f32, stored in boxes of 32 columns x 128 rows ----
     {
         cuuint64_t dims[2] = {(cuuint64_t)p.N, (cuuint64_t)p.M};
         cuuint64_t strides[1] = {(cuuint64_t)(p.o_w * 4)};
-        cuuint32_t box[2] = {32, 32};
+        cuuint32_t box[2] = {32, BM};     // one store moves a chunk of 128 rows x 32 columns
         r = g_drv.tiled(&map_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, O, dims, strides, box, ones,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
