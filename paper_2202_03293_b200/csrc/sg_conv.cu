@@ -172,7 +172,7 @@ conv_strip_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_const
         // ------------------------------------------------------------ MMA issuer (leader CTA).  The
         // whole warp walks the loop so that addresses stay warp-uniform; one elected lane issues.
         if (cta_rank == 0) {
-            constexpr uint32_t idesc = make_idesc(BN, CG * BM, false);
+            constexpr uint32_t idesc = make_idesc(BN, CG * BM, false, false, true);   // filter read as stored: N-major
             const bool issuer = elect_one();
             auto wait_all = [&](bool passed) { return __all_sync(0xffffffffu, passed) != 0; };
             // arrive, once the MMAs issued so far have finished, on the same barrier of every CTA of the group

@@ -136,11 +136,16 @@ __device__ __forceinline__ void tile_coords(int t, int num_m_tiles, int num_n_ti
     mt = g * GM + (r - nt * rows);
 }
 
-template <int BN, int CG, bool F32, int KPS>
+// LAY (bf16 matmuls, one k-block per stage): bit 0 = the input operand is stored transposed
+// ([k][m], m contiguous: A^T B of Section 4.6.1) and consumed as an M-major operand; bit 1 = the
+// filter operand is stored transposed ([n][k], k contiguous: A B^T) and consumed K-major.
+template <int BN, int CG, bool F32, int KPS, int LAY>
 __global__ void __launch_bounds__(Cfg<BN, CG, F32, KPS>::THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_flt,
                const __grid_constant__ CUtensorMap map_out, const TcParams p) {
     using C = Cfg<BN, CG, F32, KPS>;
+    constexpr bool A_MN = (LAY & 1) != 0, B_KM = (LAY & 2) != 0;
+    static_assert(LAY == 0 || (!F32 && KPS == 1), "transposed layouts: bf16, one k-block per stage");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -251,7 +256,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     const uint32_t my_bytes = KPS * (input_side ? A_STAGE_BYTES : C::B_STAGE_BYTES);
                     if (!REMOTE_FULL || cta_rank == 0) mbar_expect_tx(full_bar(s), (REMOTE_FULL ? CG : 1) * my_bytes);
                     if (input_side) {
-                        if constexpr (KPS > 1) {
+                        if constexpr (A_MN) {
+                            // transposed input: map blocked by 64 rows of m, box {64 m, BK k-rows, 2 blocks}
+                            tma_tile_3d<REMOTE_FULL>(a_dst, &map_in, bar, 0, c0, m0 / 64);
+                        } else if constexpr (KPS > 1) {
                             // matmul only: the input map is blocked by k-blocks, box {BK, 128 rows, KPS k-blocks}
                             tma_tile_3d<REMOTE_FULL>(a_dst, &map_in, bar, 0, m0, kb);
                         } else if constexpr (!REMOTE_FULL) {
@@ -273,6 +281,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                                                        (unsigned short)(kw * p.dw), (unsigned short)(kh * p.dh));
                             }
                         }
+                    } else if constexpr (B_KM) {
+                        // transposed filter: rows are columns n, k contiguous; box {BK, B_COLS rows}
+                        if constexpr (REMOTE_FULL) tma_load_2d_cg2(b_dst, &map_flt, bar, c0, n0);
+                        else tma_load_2d(b_dst, &map_flt, bar, c0, n0);
                     } else if (p.b_blocked) {
                         // box {sub-tile columns, KPS*BK channels, B_COLS / SUB_COLS column blocks, 1, 1}
                         tma_tile_5d<REMOTE_FULL>(b_dst, &map_flt, bar, 0, c0, n0 / C::SUB_COLS, kw, kh);
@@ -293,7 +305,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         // diverged warp pays for moving every descriptor out of per-lane registers: measured
         // ~120 cycles per MMA, as much as a 128 x 256 x 16 MMA takes to execute).
         if (cta_rank == 0) {
-            constexpr uint32_t idesc = make_idesc(BN, CG * BM, F32);
+            constexpr uint32_t idesc = make_idesc(BN, CG * BM, F32, A_MN, !F32 && !B_KM);
             const bool issuer = elect_one();
             auto wait_all = [&](bool passed) { return __all_sync(0xffffffffu, passed) != 0; };
             auto mma = [&](uint32_t d, uint64_t ad, uint64_t bd, uint32_t acc) {
@@ -354,15 +366,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                         for (int kbi = 0; kbi < KPS; ++kbi) {
                             if (kb + kbi >= kb1) break;      // an odd k range ends inside its last stage
                             // input tile, K-major: 8-row groups are 1024 B apart; a k-step of 16 bf16 is 32 B
-                            // inside the swizzled 128-byte row.
-                            const uint64_t a_desc = make_smem_desc(a_addr + kbi * A_STAGE_BYTES, 16, 1024);
+                            // inside the swizzled 128-byte row.  Stored transposed it is M-major like the
+                            // filter below: two 64-row sub-tiles, a k-step 16 rows of 128 B.
+                            const uint64_t a_desc = A_MN ? make_smem_desc(a_addr, C::SUB_BYTES, 1024)
+                                                         : make_smem_desc(a_addr + kbi * A_STAGE_BYTES, 16, 1024);
                             // filter tile, N-major: 64-column sub-tiles of KPS*BK k-rows are KPS*SUB_BYTES apart
                             // (leading offset), 8-row k groups 1024 B apart (stride offset); a k-step of 16
-                            // rows is 2048 B, a k-block BK rows.
-                            const uint64_t b_desc = make_smem_desc(b_addr + kbi * C::SUB_BYTES, KPS * C::SUB_BYTES, 1024);
+                            // rows is 2048 B, a k-block BK rows.  Stored transposed it is K-major like the
+                            // input tile.
+                            const uint64_t b_desc = B_KM ? make_smem_desc(b_addr, 16, 1024)
+                                                         : make_smem_desc(b_addr + kbi * C::SUB_BYTES, KPS * C::SUB_BYTES, 1024);
+                            constexpr int A_STEP = A_MN ? C::B_KSTEP_DESC : 2, B_STEP = B_KM ? 2 : C::B_KSTEP_DESC;
 #pragma unroll
                             for (int k = 0; k < K_STEPS; ++k)
-                                mma(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * C::B_KSTEP_DESC),
+                                mma(d_tmem, a_desc + (uint64_t)(k * A_STEP), b_desc + (uint64_t)(k * B_STEP),
                                     (kb + kbi > kb0 || k > 0) ? 1u : 0u);
                         }
                         // the stage is free (in every CTA of the group) once these MMAs have read it
@@ -535,7 +552,7 @@ struct Driver {
     EncodeIm2colFn im2col = nullptr;
     int num_sms = 0;
     int device = -1;
-    bool attr_set[24] = {};
+    bool attr_set[64] = {};
     bool ok = false;
 };
 std::mutex g_mu;
@@ -600,15 +617,16 @@ double estimate_ns(const Variant &v, bool f32, int64_t tiles, int64_t groups, in
     return t;
 }
 
-template <int BN, int CG, bool F32, int KPS>
+template <int BN, int CG, bool F32, int KPS, int LAY = 0>
 sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUtensorMap &mo, TcParams tp, int M, int N,
                          int slot, cudaStream_t stream) {
-  if constexpr ((F32 && BN == 256 && CG == 1) || (KPS == 2 && (F32 || (BN == 256 && CG == 1)))) {
+  if constexpr ((F32 && BN == 256 && CG == 1) || (KPS == 2 && (F32 || (BN == 256 && CG == 1))) ||
+                (LAY != 0 && (F32 || KPS != 1 || (BN == 256 && CG == 1) || (BN == 128 && CG == 2)))) {
     return SG_ERR_INTERNAL;   // the split slots of a 128 x 256 f32 tile do not fit beside a TMA ring
   } else {
     using C = Cfg<BN, CG, F32, KPS>;
     if (!g_drv.attr_set[slot]) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, CG, F32, KPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, CG, F32, KPS, LAY>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
             return SG_ERR_CUDA;
         g_drv.attr_set[slot] = true;
     }
@@ -629,7 +647,7 @@ sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUt
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<BN, CG, F32, KPS>, mi, mf, mo, tp);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<BN, CG, F32, KPS, LAY>, mi, mf, mo, tp);
     count_launch();
     return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
   }
@@ -644,17 +662,25 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     const int64_t es = f32 ? 4 : 2;
     const int BK = ROW_BYTES / (int)es;          // elements per k-block
     const CUtensorMapDataType in_type = f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-    if (p.i_c != 1 || p.k_f != 1 || p.o_f != 1) return SG_ERR_UNSUPPORTED;
+    // bf16 matmuls may hand either operand transposed through its strides (Section 4.6.1, A^T B and
+    // A B^T): the input [k][m] with m contiguous, the filter [n][k] with k contiguous
+    const bool a_mn = !f32 && p.spatial_rank == 0 && p.i_c != 1 && p.i_w == 1;
+    const bool b_km = !f32 && p.spatial_rank == 0 && p.k_f != 1 && p.k_c == 1;
+    const int lay = (a_mn ? 1 : 0) | (b_km ? 2 : 0);
+    if ((p.i_c != 1 && !a_mn) || (p.k_f != 1 && !b_km) || p.o_f != 1) return SG_ERR_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(In) % 16 || reinterpret_cast<uintptr_t>(Flt) % 16 ||
         reinterpret_cast<uintptr_t>(O) % 16) return SG_ERR_UNSUPPORTED;
-    if (!mult(p.i_w * es, 16) || !mult(p.k_c * es, 16) || !mult(p.o_w * 4, 16)) return SG_ERR_UNSUPPORTED;
+    const int64_t a_pitch = a_mn ? p.i_c : p.i_w, b_pitch = b_km ? p.k_f : p.k_c;     // elements between rows as stored
+    if (!mult(a_pitch * es, 16) || !mult(b_pitch * es, 16) || !mult(p.o_w * 4, 16)) return SG_ERR_UNSUPPORTED;
+    if (a_mn && (p.M % 64 != 0 || a_pitch < p.M)) return SG_ERR_UNSUPPORTED;   // whole 64-row blocks of m
+    if (b_km && b_pitch < p.K) return SG_ERR_UNSUPPORTED;
     if (p.Ho > 1 && p.o_h != (int64_t)p.Wo * p.o_w) return SG_ERR_UNSUPPORTED;
     if (p.batch > 1 && p.o_n != (int64_t)p.Ho * p.Wo * p.o_w) return SG_ERR_UNSUPPORTED;
     if (p.KW > 1 && !mult(p.k_kw * es, 16)) return SG_ERR_UNSUPPORTED;
     if (p.KH > 1 && !mult(p.k_kh * es, 16)) return SG_ERR_UNSUPPORTED;
-    if (p.i_w < p.C || p.k_c < p.N || p.o_w < p.N) return SG_ERR_UNSUPPORTED;   // overlapping rows
+    if ((!a_mn && p.i_w < p.C) || (!b_km && p.k_c < p.N) || p.o_w < p.N) return SG_ERR_UNSUPPORTED;   // overlapping rows
     const int64_t pitch_limit = (int64_t)1 << 40;
-    if (p.i_w * es >= pitch_limit || p.k_c * es >= pitch_limit || p.o_w * 4 >= pitch_limit) return SG_ERR_UNSUPPORTED;
+    if (a_pitch * es >= pitch_limit || b_pitch * es >= pitch_limit || p.o_w * 4 >= pitch_limit) return SG_ERR_UNSUPPORTED;
 
     std::lock_guard<std::mutex> lock(g_mu);
     if (!init_driver()) return SG_ERR_CUDA;
@@ -736,7 +762,8 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     if (g_bn_override > 0) {
         for (int i = 0; i < kNumVariants; ++i)
             if (kVariants[i].bn == g_bn_override && kVariants[i].cg == (g_cg_override > 0 ? g_cg_override : 1) &&
-                !(f32 && kVariants[i].bn == 256 && kVariants[i].cg == 1)) pick = i;
+                !(f32 && kVariants[i].bn == 256 && kVariants[i].cg == 1) &&
+                !(lay != 0 && ((kVariants[i].bn == 256 && kVariants[i].cg == 1) || (kVariants[i].bn == 128 && kVariants[i].cg == 2)))) pick = i;
     }
     auto valid_split = [&](int s) {      // every range of ceil(num_kb / s) k-blocks must be non-empty
         const int per = (tp.num_kb + s - 1) / s;
@@ -750,6 +777,7 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
             const Variant &v = kVariants[i];
             if (g_cg_override > 0 && v.cg != g_cg_override && !(v.cg == 1 && p.M <= BM)) continue;
             if (f32 && v.bn == 256 && v.cg == 1) continue;       // not built (shared-memory budget)
+            if (lay != 0 && ((v.bn == 256 && v.cg == 1) || (v.bn == 128 && v.cg == 2))) continue;   // not built for transposed operands
             if (v.bn > 64 && v.bn / 2 >= p.N) continue;          // at most half of the tile would be used
             if (v.cg == 2 && p.M <= BM) continue;                // the second CTA would have no rows
             const int64_t tiles = (int64_t)((p.M + v.cg * BM - 1) / (v.cg * BM)) * ((p.N + v.bn - 1) / v.bn);
@@ -772,14 +800,21 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         // sub-tiles are read by the converter warps, one 128-byte row per load: no swizzle
         const CUtensorMapSwizzle swz = f32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B;
         const int sub_cols = BK;      // columns of one sub-tile: a 128-byte row
-        tp.b_blocked = p.N % sub_cols == 0;
-        if (tp.b_blocked) {
+        tp.b_blocked = p.N % sub_cols == 0 && !b_km;
+        if (b_km) {
+            // stored [n][k], k contiguous: 2-D {k, n}, box {BK, columns of this CTA} lands K-major
+            cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)p.N};
+            cuuint64_t strides[1] = {(cuuint64_t)(b_pitch * es)};
+            cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)(kVariants[pick].bn / kVariants[pick].cg)};
+            r = g_drv.tiled(&map_flt, in_type, 2, const_cast<void *>(Flt), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        } else if (tp.b_blocked) {
             // whole sub-tile column blocks: 5-D {column in block, c, column block, kw, kh}; one box
             // {sub_cols, BK, blocks of this CTA, 1, 1} is the CTA's whole filter tile of a k-block
             cuuint64_t dims[5] = {(cuuint64_t)sub_cols, (cuuint64_t)p.C, (cuuint64_t)(p.N / sub_cols), (cuuint64_t)p.KW, (cuuint64_t)p.KH};
             cuuint64_t strides[4] = {(cuuint64_t)(p.k_c * es), (cuuint64_t)ROW_BYTES, (cuuint64_t)(s_kw * es), (cuuint64_t)(s_kh * es)};
             // (bf16 matmuls with whole k-blocks fetch two k-blocks per load, see below)
-            const bool two = !f32 && p.spatial_rank == 0 && p.K % BK == 0 && !(kVariants[pick].bn == 256 && kVariants[pick].cg == 1) && g_kps_override != 1;
+            const bool two = !f32 && lay == 0 && p.spatial_rank == 0 && p.K % BK == 0 && !(kVariants[pick].bn == 256 && kVariants[pick].cg == 1) && g_kps_override != 1;
             cuuint32_t box[5] = {(cuuint32_t)sub_cols, (cuuint32_t)(two ? 2 * BK : BK), (cuuint32_t)(kVariants[pick].bn / kVariants[pick].cg / sub_cols), 1, 1};
             r = g_drv.tiled(&map_flt, in_type, 5, const_cast<void *>(Flt), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -794,10 +829,17 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
     }
     // bf16 matmuls with whole k-blocks move two k-blocks per stage and per TMA load
-    const int kps = (!f32 && p.spatial_rank == 0 && p.K % BK == 0 && tp.b_blocked &&
+    const int kps = (!f32 && lay == 0 && p.spatial_rank == 0 && p.K % BK == 0 && tp.b_blocked &&
                      !(kVariants[pick].bn == 256 && kVariants[pick].cg == 1) && g_kps_override != 1) ? 2 : 1;
     if (p.spatial_rank == 0) {
-        if (kps == 2) {
+        if (a_mn) {
+            // stored [k][m], m contiguous, blocked by 64 rows of m: {m in block, k, m block}, box {64, BK, 2}
+            cuuint64_t dims[3] = {64, (cuuint64_t)p.K, (cuuint64_t)(p.M / 64)};
+            cuuint64_t strides[2] = {(cuuint64_t)(a_pitch * es), (cuuint64_t)ROW_BYTES};
+            cuuint32_t box[3] = {64, (cuuint32_t)BK, 2};
+            r = g_drv.tiled(&map_in, in_type, 3, const_cast<void *>(In), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        } else if (kps == 2) {
             // blocked by k-blocks: {k in block, m, k-block}, box {BK, 128, 2}
             cuuint64_t dims[3] = {(cuuint64_t)BK, (cuuint64_t)p.M, (cuuint64_t)(p.K / BK)};
             cuuint64_t strides[2] = {(cuuint64_t)(p.i_w * es), (cuuint64_t)ROW_BYTES};
@@ -825,11 +867,14 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         tp.accumulate = 1;
     }
     g_last_choice[0] = kVariants[pick].bn; g_last_choice[1] = kVariants[pick].cg; g_last_choice[2] = splits;
-    const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0);
+    const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0) + lay * 3 * kNumVariants;
 #define SG_LAUNCH(BN_, CG_)                                                                                \
     (f32 ? launch_variant<BN_, CG_, true, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)         \
-         : kps == 2 ? launch_variant<BN_, CG_, false, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)   \
-                    : launch_variant<BN_, CG_, false, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream))
+     : lay == 1 ? launch_variant<BN_, CG_, false, 1, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
+     : lay == 2 ? launch_variant<BN_, CG_, false, 1, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
+     : lay == 3 ? launch_variant<BN_, CG_, false, 1, 3>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
+     : kps == 2 ? launch_variant<BN_, CG_, false, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream) \
+                : launch_variant<BN_, CG_, false, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream))
     switch (pick) {
         case 0: return SG_LAUNCH(64, 1);
         case 1: return SG_LAUNCH(128, 1);

@@ -159,16 +159,15 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_b
 }
 
 // Instruction descriptor: f32 accumulator, A and B both bf16 (kind::f16) or both tf32
-// (kind::tf32), A K-major, B N-major.
-__host__ __device__ constexpr uint32_t make_idesc(int n, int m, bool tf32) {
+// (kind::tf32); each operand K-major, or MN-major (its rows/columns contiguous in shared memory
+// instead of k; kind::tf32 takes K-major operands only: an MN-major descriptor makes the MMA a
+// no-op there).
+__host__ __device__ constexpr uint32_t make_idesc(int n, int m, bool tf32, bool a_mn_major, bool b_mn_major) {
     return (1u << 4)                       // D format: f32
          | ((tf32 ? 2u : 1u) << 7)         // A format: bf16 = 1 in kind::f16, tf32 = 2 in kind::tf32
          | ((tf32 ? 2u : 1u) << 10)        // B format: the same type as A
-         | (0u << 15)                      // A major: K
-         | ((tf32 ? 0u : 1u) << 16)        // B major: MN for bf16 (filter stored [k][f], f contiguous, read as
-                                           // is); kind::tf32 takes K-major operands only (an N-major
-                                           // descriptor makes the MMA a no-op), so the f32 path
-                                           // transposes the filter tile while splitting it
+         | ((a_mn_major ? 1u : 0u) << 15)  // A major
+         | ((b_mn_major ? 1u : 0u) << 16)  // B major
          | ((uint32_t)(n >> 3) << 17)      // N / 8
          | ((uint32_t)(m >> 4) << 24);     // M / 16 (128 for one CTA, 256 for a pair)
 }

@@ -575,3 +575,68 @@ def test_sweep_shapes_in_the_benchmark_launch_configuration():
         got = C[torch.from_numpy(pm).cuda(), torch.from_numpy(pn).cuda()]
         assert_within_bound(got, want, S, f"graph replay {tuple(A.shape)} x {tuple(B.shape)} {A.dtype}")
         assert not torch.isnan(C).any()
+
+
+# ------------------------------------------------------------------ transposed operands on the tensor-core path
+
+def run_matmul_layout(M, N, K, a_t, b_t, accumulate=False, seed=SEED + 30):
+    """bf16 matmul with A stored [k][m] (a_t) and / or B stored [n][k] (b_t), handed over as strided views."""
+    A, a = operand((K, M) if a_t else (M, K), seed, 1, "uniform", "bf16")
+    B, b = operand((N, K) if b_t else (K, N), seed, 2, "uniform", "bf16")
+    if accumulate:
+        C, c0 = operand((M, N), seed, 3, "uniform", "f32")
+        C = C.clone()
+    else:
+        C, c0 = torch.full((M, N), float("nan"), device="cuda"), None
+    sg.sg_matmul(A.t() if a_t else A, B.t() if b_t else B, C, sg.SG_ACCUMULATE if accumulate else sg.SG_OVERWRITE)
+    torch.cuda.synchronize()
+    want, S = ref.matmul(np.ascontiguousarray(a.T) if a_t else a, np.ascontiguousarray(b.T) if b_t else b, C_in=c0)
+    if accumulate:
+        S = S + np.abs(c0)
+    return C, want, S
+
+
+@pytest.mark.parametrize("a_t,b_t", [(True, False), (False, True), (True, True)])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (320, 200, 136), (64, 72, 8), (512, 264, 1000), (1024, 768, 72)])
+def test_matmul_bf16_transposed_operands_tensor_path(a_t, b_t, M, N, K):
+    # Section 4.6.1: A^T B, A B^T (and both) are the same op under different strides
+    sg.sg_set_kernel_override(TENSOR)
+    C, want, S = run_matmul_layout(M, N, K, a_t, b_t)
+    assert sg.sg_last_kernel() == TENSOR
+    assert_within_bound(C, want, S, f"A^T={a_t} B^T={b_t} {M}x{N}x{K}")
+
+
+@pytest.mark.parametrize("a_t,b_t", [(True, False), (False, True), (True, True)])
+@pytest.mark.parametrize("bn,cg,splits", [(64, 1, 1), (128, 1, 3), (256, 2, 1), (256, 2, 4)])
+def test_matmul_bf16_transposed_operands_every_variant(a_t, b_t, bn, cg, splits):
+    sg.sg_set_kernel_override(TENSOR)
+    sg.sg_set_tile_override(bn, cg, splits)
+    C, want, S = run_matmul_layout(448, 520, 456, a_t, b_t, accumulate=(splits == 3))
+    assert sg.sg_last_tile_choice() == (bn, cg, splits)
+    assert_within_bound(C, want, S, "forced variant")
+    sg.sg_set_tile_override(0, 0, 0)
+    # integer inputs: exact
+    A = torch.randint(-2, 3, (256, 192), device="cuda").to(torch.bfloat16)       # stored [k][m] or [m][k]
+    B = torch.randint(-2, 3, (192, 320), device="cuda").to(torch.bfloat16)
+    Aview = A.t().contiguous().t() if a_t else A                                    # same values, transposed storage
+    Bview = B.t().contiguous().t() if b_t else B
+    C = torch.empty(256, 320, device="cuda")
+    sg.sg_matmul(Aview, Bview, C)
+    torch.cuda.synchronize()
+    assert sg.sg_last_kernel() == TENSOR
+    assert torch.equal(C, A.float() @ B.float())
+
+
+def test_matmul_bf16_transposed_full_size_sampled():
+    M = N = K = 4096
+    At, a_t = operand((K, M), SEED + 31, 1, "uniform", "bf16")
+    Bt, b_t = operand((N, K), SEED + 31, 2, "uniform", "bf16")
+    C = torch.full((M, N), float("nan"), device="cuda")
+    sg.sg_matmul(At.t(), Bt.t(), C)
+    torch.cuda.synchronize()
+    assert sg.sg_last_kernel() == TENSOR
+    pm, pn = sample_points(M, N, 2048, 96)
+    want, S = ref.matmul_points(np.ascontiguousarray(a_t.T), np.ascontiguousarray(b_t.T), pm, pn)
+    got = C[torch.from_numpy(pm).cuda(), torch.from_numpy(pn).cuda()]
+    assert_within_bound(got, want, S, "A^T B^T 4096^3")
+    assert not torch.isnan(C).any()
