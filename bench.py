@@ -169,11 +169,12 @@ def op_specs(sg, seed):
                            gpu_operand((Kx, Nx), seed, 40 + s, "uniform", dtype), torch.empty(Mx, Nx, device="cuda")),
                 lambda a, b, c: sg.sg_matmul(a, b, c))
 
-    def mm_t(Mx, Nx, Kx, a_t, b_t, label):
+    def mm_t(Mx, Nx, Kx, a_t, b_t, label, dtype="bf16"):
         # operands stored transposed and handed over as strided views (Section 4.6.1: A^T B, A B^T)
-        return (label, 2.0 * Mx * Nx * Kx, (Mx * Kx + Kx * Nx) * 2 + Mx * Nx * 4, "bf16",
-                lambda s: ((gpu_operand((Kx, Mx), seed, 10 + s, "uniform", "bf16").t() if a_t else gpu_operand((Mx, Kx), seed, 10 + s, "uniform", "bf16")),
-                           (gpu_operand((Nx, Kx), seed, 40 + s, "uniform", "bf16").t() if b_t else gpu_operand((Kx, Nx), seed, 40 + s, "uniform", "bf16")),
+        es = 2 if dtype == "bf16" else 4
+        return (label, 2.0 * Mx * Nx * Kx, (Mx * Kx + Kx * Nx) * es + Mx * Nx * 4, dtype,
+                lambda s: ((gpu_operand((Kx, Mx), seed, 10 + s, "uniform", dtype).t() if a_t else gpu_operand((Mx, Kx), seed, 10 + s, "uniform", dtype)),
+                           (gpu_operand((Nx, Kx), seed, 40 + s, "uniform", dtype).t() if b_t else gpu_operand((Kx, Nx), seed, 40 + s, "uniform", dtype)),
                            torch.empty(Mx, Nx, device="cuda")),
                 lambda a, b, c: sg.sg_matmul(a, b, c))
 
@@ -181,6 +182,8 @@ def op_specs(sg, seed):
         "matmul128_f32": mm(128, 128, 128, "f32", "matmul 128^3 f32 (config 1)"),
         "matmul4096_bf16_atb": mm_t(4096, 4096, 4096, True, False, "matmul 4096^3 bf16, A stored transposed (A^T B)"),
         "matmul4096_bf16_abt": mm_t(4096, 4096, 4096, False, True, "matmul 4096^3 bf16, B stored transposed (A B^T)"),
+        "matmul4096_f32_atb": mm_t(4096, 4096, 4096, True, False, "matmul 4096^3 f32, A stored transposed (A^T B)", "f32"),
+        "matmul4096_f32_abt": mm_t(4096, 4096, 4096, False, True, "matmul 4096^3 f32, B stored transposed (A B^T)", "f32"),
         "matmul4096_f32": mm(4096, 4096, 4096, "f32", "matmul 4096^3 f32 (sweep corner)"),
         "matmul4096_bf16": mm(4096, 4096, 4096, "bf16", "matmul 4096^3 bf16 (sweep corner)"),
         "matmul1024_bf16": mm(1024, 1024, 1024, "bf16", "matmul 1024^3 bf16 (sweep point)"),

@@ -75,9 +75,9 @@ enum {
  * Matrix multiplication (paper Section 4.6.1, variant "AB"; iterators
  * (m,n,k) = (parallel, parallel, reduction), maps A:(m,k) B:(k,n) C:(m,n)).
  * The transposed variants of the same section (A^T B, A B^T) are obtained
- * through the stride arguments alone; with bf16 inputs, 16-byte aligned
- * pitches (and M a multiple of 64 when A is stored [k][m]) they run on the
- * tensor-core path like the plain layout.
+ * through the stride arguments alone; with 16-byte aligned pitches (and M
+ * a multiple of 64 for bf16, 32 for f32, when A is stored [k][m]) they run
+ * on the tensor-core path like the plain layout.
  *   A  : M x K elements of in_dtype, element (m,k) at A[m*a_stride_m + k*a_stride_k]
  *   B  : K x N elements of in_dtype, element (k,n) at B[k*b_stride_k + n*b_stride_n]
  *   C  : M x N f32,                  element (m,n) at C[m*c_stride_m + n*c_stride_n]

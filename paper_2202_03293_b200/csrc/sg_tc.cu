@@ -35,6 +35,7 @@
 #include <cuda.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "sg_internal.cuh"
 #include "sg_tc_ptx.cuh"
@@ -145,7 +146,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                const __grid_constant__ CUtensorMap map_out, const TcParams p) {
     using C = Cfg<BN, CG, F32, KPS>;
     constexpr bool A_MN = (LAY & 1) != 0, B_KM = (LAY & 2) != 0;
-    static_assert(LAY == 0 || (!F32 && KPS == 1), "transposed layouts: bf16, one k-block per stage");
+    static_assert(LAY == 0 || KPS == 1, "transposed layouts: one k-block per stage");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -257,8 +258,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     if (!REMOTE_FULL || cta_rank == 0) mbar_expect_tx(full_bar(s), (REMOTE_FULL ? CG : 1) * my_bytes);
                     if (input_side) {
                         if constexpr (A_MN) {
-                            // transposed input: map blocked by 64 rows of m, box {64 m, BK k-rows, 2 blocks}
-                            tma_tile_3d<REMOTE_FULL>(a_dst, &map_in, bar, 0, c0, m0 / 64);
+                            // transposed input: map blocked by sub-tile rows of m (one 128-byte row: 64 bf16 or
+                            // 32 f32), box {rows in block, BK k-rows, 128 / rows-in-block blocks}
+                            tma_tile_3d<REMOTE_FULL>(a_dst, &map_in, bar, 0, c0, m0 / C::SUB_COLS);
                         } else if constexpr (KPS > 1) {
                             // matmul only: the input map is blocked by k-blocks, box {BK, 128 rows, KPS k-blocks}
                             tma_tile_3d<REMOTE_FULL>(a_dst, &map_in, bar, 0, m0, kb);
@@ -305,7 +307,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         // diverged warp pays for moving every descriptor out of per-lane registers: measured
         // ~120 cycles per MMA, as much as a 128 x 256 x 16 MMA takes to execute).
         if (cta_rank == 0) {
-            constexpr uint32_t idesc = make_idesc(BN, CG * BM, F32, A_MN, !F32 && !B_KM);
+            constexpr uint32_t idesc = make_idesc(BN, CG * BM, F32, A_MN && !F32, !F32 && !B_KM);   // f32: the converter warps hand over K-major tiles
             const bool issuer = elect_one();
             auto wait_all = [&](bool passed) { return __all_sync(0xffffffffu, passed) != 0; };
             auto mma = [&](uint32_t d, uint64_t ad, uint64_t bd, uint32_t acc) {
@@ -405,12 +407,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     if (!mbar_wait<CG == 2>(split_empty_bar(s), ((it >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
                     const uint8_t *raw = smem_gen + r * C::STAGE_BYTES;
                     uint8_t *slot = smem_gen + C::STAGES * C::STAGE_BYTES + s * C::SPLIT_BYTES;
-                    // input tile: elementwise, the swizzled placement of the elements is kept
-                    {
-                        const uint4 *src = reinterpret_cast<const uint4 *>(raw) + ct;
-                        uint4 *hi = reinterpret_cast<uint4 *>(slot) + ct;
-                        uint4 *lo = hi + A_STAGE_BYTES / 16;
-                        constexpr int N = A_STAGE_BYTES / 16 / CONVERTER_THREADS;   // 16-byte chunks per thread
+                    // An operand tile that arrives K-major (rows of 32 k, 128-byte swizzled by the TMA) is
+                    // split elementwise: the swizzled placement of the elements is kept.
+                    auto split_elementwise = [&](const uint8_t *src_tile, uint8_t *hi_tile, uint8_t *lo_tile, auto bytes_tag) {
+                        constexpr int BYTES = decltype(bytes_tag)::value;
+                        const uint4 *src = reinterpret_cast<const uint4 *>(src_tile) + ct;
+                        uint4 *hi = reinterpret_cast<uint4 *>(hi_tile) + ct;
+                        uint4 *lo = reinterpret_cast<uint4 *>(lo_tile) + ct;
+                        constexpr int N = BYTES / 16 / CONVERTER_THREADS;   // 16-byte chunks per thread
+                        static_assert(N >= 1 && BYTES % (16 * CONVERTER_THREADS) == 0, "converter chunking");
                         uint4 v[N];
 #pragma unroll
                         for (int i = 0; i < N; ++i) v[i] = src[i * CONVERTER_THREADS];
@@ -421,17 +426,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                             hi[i * CONVERTER_THREADS] = h;
                             lo[i * CONVERTER_THREADS] = l;
                         }
-                    }
-                    // filter tile: raw sub-tiles are [32 k][32 f] rows of 128 B, not swizzled; the split
-                    // tiles are K-major, [f][32 k] rows of 128 B in 8-row groups with the 128-byte swizzle
-                    // (16-byte chunk c of row f sits at chunk c ^ (f & 7)).  A unit is a quarter of a
-                    // sub-tile (8 k); lane = f reads a column (one 128-byte row per load across the warp)
-                    // and writes 2 chunks of its row.
-                    {
-                        const float *braw = reinterpret_cast<const float *>(raw + A_STAGE_BYTES);
-                        uint8_t *bhi = slot + 2 * A_STAGE_BYTES;
-                        uint8_t *blo = bhi + C::B_STAGE_BYTES;
-                        constexpr int UNITS = 4 * C::B_COLS / 32;
+                    };
+                    // An operand tile that arrives MN-major (sub-tiles of [32 k][32 rows-or-columns], 128-byte
+                    // rows, not swizzled) is transposed while it is split: the split tiles are K-major,
+                    // [row][32 k] rows of 128 B in 8-row groups with the 128-byte swizzle (16-byte chunk c of
+                    // row f sits at chunk c ^ (f & 7)).  A unit is a quarter of a sub-tile (8 k); lane = f
+                    // reads a column (one 128-byte row per load across the warp) and writes 2 chunks of its row.
+                    auto split_transpose = [&](const uint8_t *src_tile, uint8_t *hi_tile, uint8_t *lo_tile, auto cols_tag) {
+                        constexpr int COLS = decltype(cols_tag)::value;
+                        const float *braw = reinterpret_cast<const float *>(src_tile);
+                        constexpr int UNITS = 4 * COLS / 32;
 #pragma unroll
                         for (int u = cw; u < UNITS; u += CONVERTER_THREADS / 32) {
                             const int j = u >> 2, quarter = u & 3;
@@ -446,11 +450,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                                 uint4 h, l;
                                 split4(make_uint4(x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]), h, l);
                                 const int off = row_off + (((quarter * 2 + c) ^ (f & 7)) << 4);
-                                *reinterpret_cast<uint4 *>(bhi + off) = h;
-                                *reinterpret_cast<uint4 *>(blo + off) = l;
+                                *reinterpret_cast<uint4 *>(hi_tile + off) = h;
+                                *reinterpret_cast<uint4 *>(lo_tile + off) = l;
                             }
                         }
-                    }
+                    };
+                    // input: K-major as stored, M-major when stored transposed; filter: N-major as stored,
+                    // K-major when stored transposed.  kind::tf32 takes K-major operands only.
+                    if constexpr (A_MN) split_transpose(raw, slot, slot + A_STAGE_BYTES, std::integral_constant<int, BM>{});
+                    else split_elementwise(raw, slot, slot + A_STAGE_BYTES, std::integral_constant<int, A_STAGE_BYTES>{});
+                    if constexpr (B_KM)
+                        split_elementwise(raw + A_STAGE_BYTES, slot + 2 * A_STAGE_BYTES, slot + 2 * A_STAGE_BYTES + C::B_STAGE_BYTES,
+                                          std::integral_constant<int, C::B_STAGE_BYTES>{});
+                    else
+                        split_transpose(raw + A_STAGE_BYTES, slot + 2 * A_STAGE_BYTES, slot + 2 * A_STAGE_BYTES + C::B_STAGE_BYTES,
+                                        std::integral_constant<int, C::B_COLS>{});
                     fence_async_smem();     // generic-proxy writes -> visible to the tensor core's reads
                     __syncwarp();
                     if (lane == 0) {
@@ -621,7 +635,7 @@ template <int BN, int CG, bool F32, int KPS, int LAY = 0>
 sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUtensorMap &mo, TcParams tp, int M, int N,
                          int slot, cudaStream_t stream) {
   if constexpr ((F32 && BN == 256 && CG == 1) || (KPS == 2 && (F32 || (BN == 256 && CG == 1))) ||
-                (LAY != 0 && (F32 || KPS != 1 || (BN == 256 && CG == 1) || (BN == 128 && CG == 2)))) {
+                (LAY != 0 && (KPS != 1 || (BN == 256 && CG == 1) || (BN == 128 && CG == 2)))) {
     return SG_ERR_INTERNAL;   // the split slots of a 128 x 256 f32 tile do not fit beside a TMA ring
   } else {
     using C = Cfg<BN, CG, F32, KPS>;
@@ -662,17 +676,17 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     const int64_t es = f32 ? 4 : 2;
     const int BK = ROW_BYTES / (int)es;          // elements per k-block
     const CUtensorMapDataType in_type = f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-    // bf16 matmuls may hand either operand transposed through its strides (Section 4.6.1, A^T B and
+    // matmuls may hand either operand transposed through its strides (Section 4.6.1, A^T B and
     // A B^T): the input [k][m] with m contiguous, the filter [n][k] with k contiguous
-    const bool a_mn = !f32 && p.spatial_rank == 0 && p.i_c != 1 && p.i_w == 1;
-    const bool b_km = !f32 && p.spatial_rank == 0 && p.k_f != 1 && p.k_c == 1;
+    const bool a_mn = p.spatial_rank == 0 && p.i_c != 1 && p.i_w == 1;
+    const bool b_km = p.spatial_rank == 0 && p.k_f != 1 && p.k_c == 1;
     const int lay = (a_mn ? 1 : 0) | (b_km ? 2 : 0);
     if ((p.i_c != 1 && !a_mn) || (p.k_f != 1 && !b_km) || p.o_f != 1) return SG_ERR_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(In) % 16 || reinterpret_cast<uintptr_t>(Flt) % 16 ||
         reinterpret_cast<uintptr_t>(O) % 16) return SG_ERR_UNSUPPORTED;
     const int64_t a_pitch = a_mn ? p.i_c : p.i_w, b_pitch = b_km ? p.k_f : p.k_c;     // elements between rows as stored
     if (!mult(a_pitch * es, 16) || !mult(b_pitch * es, 16) || !mult(p.o_w * 4, 16)) return SG_ERR_UNSUPPORTED;
-    if (a_mn && (p.M % 64 != 0 || a_pitch < p.M)) return SG_ERR_UNSUPPORTED;   // whole 64-row blocks of m
+    if (a_mn && (p.M % BK != 0 || a_pitch < p.M)) return SG_ERR_UNSUPPORTED;   // whole sub-tile blocks of m (64 bf16 / 32 f32 rows)
     if (b_km && b_pitch < p.K) return SG_ERR_UNSUPPORTED;
     if (p.Ho > 1 && p.o_h != (int64_t)p.Wo * p.o_w) return SG_ERR_UNSUPPORTED;
     if (p.batch > 1 && p.o_n != (int64_t)p.Ho * p.Wo * p.o_w) return SG_ERR_UNSUPPORTED;
@@ -806,8 +820,8 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
             cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)p.N};
             cuuint64_t strides[1] = {(cuuint64_t)(b_pitch * es)};
             cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)(kVariants[pick].bn / kVariants[pick].cg)};
-            r = g_drv.tiled(&map_flt, in_type, 2, const_cast<void *>(Flt), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            r = g_drv.tiled(&map_flt, in_type, 2, const_cast<void *>(Flt), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         } else if (tp.b_blocked) {
             // whole sub-tile column blocks: 5-D {column in block, c, column block, kw, kh}; one box
             // {sub_cols, BK, blocks of this CTA, 1, 1} is the CTA's whole filter tile of a k-block
@@ -833,12 +847,15 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
                      !(kVariants[pick].bn == 256 && kVariants[pick].cg == 1) && g_kps_override != 1) ? 2 : 1;
     if (p.spatial_rank == 0) {
         if (a_mn) {
-            // stored [k][m], m contiguous, blocked by 64 rows of m: {m in block, k, m block}, box {64, BK, 2}
-            cuuint64_t dims[3] = {64, (cuuint64_t)p.K, (cuuint64_t)(p.M / 64)};
+            // stored [k][m], m contiguous, blocked by sub-tile rows of m (a 128-byte row: BK elements):
+            // {m in block, k, m block}, box {BK, BK, 128 / BK}.  bf16 lands as an M-major operand
+            // (swizzled); f32 is read by the converter warps, which transpose it (no swizzle).
+            cuuint64_t dims[3] = {(cuuint64_t)BK, (cuuint64_t)p.K, (cuuint64_t)(p.M / BK)};
             cuuint64_t strides[2] = {(cuuint64_t)(a_pitch * es), (cuuint64_t)ROW_BYTES};
-            cuuint32_t box[3] = {64, (cuuint32_t)BK, 2};
+            cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BK, (cuuint32_t)(BM / BK)};
             r = g_drv.tiled(&map_in, in_type, 3, const_cast<void *>(In), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                            f32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
         } else if (kps == 2) {
             // blocked by k-blocks: {k in block, m, k-block}, box {BK, 128, 2}
             cuuint64_t dims[3] = {(cuuint64_t)BK, (cuuint64_t)p.M, (cuuint64_t)(p.K / BK)};
@@ -869,7 +886,10 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     g_last_choice[0] = kVariants[pick].bn; g_last_choice[1] = kVariants[pick].cg; g_last_choice[2] = splits;
     const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0) + lay * 3 * kNumVariants;
 #define SG_LAUNCH(BN_, CG_)                                                                                \
-    (f32 ? launch_variant<BN_, CG_, true, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)         \
+    (f32 ? (lay == 0 ? launch_variant<BN_, CG_, true, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)         \
+            : lay == 1 ? launch_variant<BN_, CG_, true, 1, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
+            : lay == 2 ? launch_variant<BN_, CG_, true, 1, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
+                       : launch_variant<BN_, CG_, true, 1, 3>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream))   \
      : lay == 1 ? launch_variant<BN_, CG_, false, 1, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
      : lay == 2 ? launch_variant<BN_, CG_, false, 1, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
      : lay == 3 ? launch_variant<BN_, CG_, false, 1, 3>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \

@@ -579,10 +579,10 @@ def test_sweep_shapes_in_the_benchmark_launch_configuration():
 
 # ------------------------------------------------------------------ transposed operands on the tensor-core path
 
-def run_matmul_layout(M, N, K, a_t, b_t, accumulate=False, seed=SEED + 30):
-    """bf16 matmul with A stored [k][m] (a_t) and / or B stored [n][k] (b_t), handed over as strided views."""
-    A, a = operand((K, M) if a_t else (M, K), seed, 1, "uniform", "bf16")
-    B, b = operand((N, K) if b_t else (K, N), seed, 2, "uniform", "bf16")
+def run_matmul_layout(M, N, K, a_t, b_t, accumulate=False, seed=SEED + 30, dtype="bf16"):
+    """matmul with A stored [k][m] (a_t) and / or B stored [n][k] (b_t), handed over as strided views."""
+    A, a = operand((K, M) if a_t else (M, K), seed, 1, "uniform", dtype)
+    B, b = operand((N, K) if b_t else (K, N), seed, 2, "uniform", dtype)
     if accumulate:
         C, c0 = operand((M, N), seed, 3, "uniform", "f32")
         C = C.clone()
@@ -596,28 +596,31 @@ def run_matmul_layout(M, N, K, a_t, b_t, accumulate=False, seed=SEED + 30):
     return C, want, S
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
 @pytest.mark.parametrize("a_t,b_t", [(True, False), (False, True), (True, True)])
 @pytest.mark.parametrize("M,N,K", [(128, 128, 128), (320, 200, 136), (64, 72, 8), (512, 264, 1000), (1024, 768, 72)])
-def test_matmul_bf16_transposed_operands_tensor_path(a_t, b_t, M, N, K):
+def test_matmul_transposed_operands_tensor_path(dtype, a_t, b_t, M, N, K):
     # Section 4.6.1: A^T B, A B^T (and both) are the same op under different strides
     sg.sg_set_kernel_override(TENSOR)
-    C, want, S = run_matmul_layout(M, N, K, a_t, b_t)
+    C, want, S = run_matmul_layout(M, N, K, a_t, b_t, dtype=dtype)
     assert sg.sg_last_kernel() == TENSOR
-    assert_within_bound(C, want, S, f"A^T={a_t} B^T={b_t} {M}x{N}x{K}")
+    assert assert_within_bound(C, want, S, f"{dtype} A^T={a_t} B^T={b_t} {M}x{N}x{K}") < F32_TENSOR_RATIO
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
 @pytest.mark.parametrize("a_t,b_t", [(True, False), (False, True), (True, True)])
 @pytest.mark.parametrize("bn,cg,splits", [(64, 1, 1), (128, 1, 3), (256, 2, 1), (256, 2, 4)])
-def test_matmul_bf16_transposed_operands_every_variant(a_t, b_t, bn, cg, splits):
+def test_matmul_transposed_operands_every_variant(dtype, a_t, b_t, bn, cg, splits):
     sg.sg_set_kernel_override(TENSOR)
     sg.sg_set_tile_override(bn, cg, splits)
-    C, want, S = run_matmul_layout(448, 520, 456, a_t, b_t, accumulate=(splits == 3))
+    C, want, S = run_matmul_layout(448, 520, 456, a_t, b_t, accumulate=(splits == 3), dtype=dtype)
     assert sg.sg_last_tile_choice() == (bn, cg, splits)
     assert_within_bound(C, want, S, "forced variant")
     sg.sg_set_tile_override(0, 0, 0)
     # integer inputs: exact
-    A = torch.randint(-2, 3, (256, 192), device="cuda").to(torch.bfloat16)       # stored [k][m] or [m][k]
-    B = torch.randint(-2, 3, (192, 320), device="cuda").to(torch.bfloat16)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    A = torch.randint(-2, 3, (256, 192), device="cuda").to(tdt)       # stored [k][m] or [m][k]
+    B = torch.randint(-2, 3, (192, 320), device="cuda").to(tdt)
     Aview = A.t().contiguous().t() if a_t else A                                    # same values, transposed storage
     Bview = B.t().contiguous().t() if b_t else B
     C = torch.empty(256, 320, device="cuda")
@@ -627,10 +630,11 @@ def test_matmul_bf16_transposed_operands_every_variant(a_t, b_t, bn, cg, splits)
     assert torch.equal(C, A.float() @ B.float())
 
 
-def test_matmul_bf16_transposed_full_size_sampled():
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_matmul_transposed_full_size_sampled(dtype):
     M = N = K = 4096
-    At, a_t = operand((K, M), SEED + 31, 1, "uniform", "bf16")
-    Bt, b_t = operand((N, K), SEED + 31, 2, "uniform", "bf16")
+    At, a_t = operand((K, M), SEED + 31, 1, "uniform", dtype)
+    Bt, b_t = operand((N, K), SEED + 31, 2, "uniform", dtype)
     C = torch.full((M, N), float("nan"), device="cuda")
     sg.sg_matmul(At.t(), Bt.t(), C)
     torch.cuda.synchronize()
