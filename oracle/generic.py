@@ -71,3 +71,11 @@ def conv2d_maps(sh, sw, dh, dw):
     m_o = [[1, 0, 0, 0, 0, 0, 0], [0, 1, 0, 0, 0, 0, 0], [0, 0, 1, 0, 0, 0, 0],
            [0, 0, 0, 1, 0, 0, 0]]
     return m_in, m_k, m_o
+
+
+def depthwise_conv2d_maps(sh, sw, dh, dw):
+    # iterators (n, h, w, c, kh, kw): the channel iterator is parallel (Section 4.6.3)
+    m_in = [[1, 0, 0, 0, 0, 0], [0, sh, 0, 0, dh, 0], [0, 0, sw, 0, 0, dw], [0, 0, 0, 1, 0, 0]]
+    m_k = [[0, 0, 0, 0, 1, 0], [0, 0, 0, 0, 0, 1], [0, 0, 0, 1, 0, 0]]
+    m_o = [[1, 0, 0, 0, 0, 0], [0, 1, 0, 0, 0, 0], [0, 0, 1, 0, 0, 0], [0, 0, 0, 1, 0, 0]]
+    return m_in, m_k, m_o

@@ -160,3 +160,37 @@ def conv2d_points(I, Kf, pn, ph, pw, pf, stride=(1, 1), dilation=(1, 1), threads
                                _ptr(pts[0]), _ptr(pts[1]), _ptr(pts[2]), _ptr(pts[3]), _ptr(out),
                                _ptr(sab), ctypes.c_int(threads))
     return out, sab
+
+
+def depthwise_conv2d_nhwc_hwc(I, Kf, stride=(1, 1), dilation=(1, 1), O_in=None, out_hw=None, threads=0):
+    """O[n,h,w,c] = (O_in) + sum_{kh,kw} I[n,h*sh+kh*dh,w*sw+kw*dw,c] * Kf[kh,kw,c]  (Section 4.6.3)."""
+    I, Kf = _f32(I), _f32(Kf)
+    N, H_in, W_in, C = I.shape
+    KH, KW, C2 = Kf.shape
+    assert C == C2
+    sh, sw = stride
+    dh, dw = dilation
+    if out_hw is None:
+        out_hw = ((H_in - (KH - 1) * dh - 1) // sh + 1, (W_in - (KW - 1) * dw - 1) // sw + 1)
+    Ho, Wo = out_hw
+    mode = 0 if O_in is None else 1
+    O = np.zeros((N, Ho, Wo, C), np.float64) if O_in is None else np.array(O_in, dtype=np.float64, order="C")
+    S = np.zeros((N, Ho, Wo, C), np.float64)
+    rc = lib().sg_ref_depthwise_conv2d_nhwc_hwc(_i64(N), _i64(Ho), _i64(Wo), _i64(C), _i64(KH), _i64(KW),
+                                                _i64(H_in), _i64(W_in), _i64(sh), _i64(sw), _i64(dh), _i64(dw),
+                                                _ptr(I), _i64arr(_estrides(I)), _ptr(Kf), _i64arr(_estrides(Kf)),
+                                                _ptr(O), _i64arr([Ho * Wo * C, Wo * C, C, 1]), _ptr(S),
+                                                ctypes.c_int(mode), ctypes.c_int(threads))
+    if rc:
+        raise ValueError("sg_ref_depthwise_conv2d_nhwc_hwc rejected its arguments")
+    return O, S
+
+
+def depthwise_conv1d_nwc_wc(I, Kf, stride=1, dilation=1, O_in=None, W_out=None, threads=0):
+    """O[n,w,c] = (O_in) + sum_kw I[n,w*sw+kw*dw,c] * Kf[kw,c]: the 2-D op with H = KH = 1."""
+    I, Kf = _f32(I), _f32(Kf)
+    N, W_in, C = I.shape
+    O_in4 = None if O_in is None else np.asarray(O_in)[:, None]
+    out_hw = None if W_out is None else (1, W_out)
+    O, S = depthwise_conv2d_nhwc_hwc(I[:, None], Kf[None], (1, stride), (1, dilation), O_in4, out_hw, threads)
+    return O[:, 0], S[:, 0]

@@ -1,5 +1,6 @@
 /*
- * Reference (oracle) implementation of the three structured contraction ops.
+ * Reference (oracle) implementation of the structured contraction ops (and of the depthwise
+ * convolutions, at the end of the file).
  *
  * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a deliberately plain,
  * slow CPU evaluation of each op's definition, used only to check the CUDA
@@ -214,6 +215,52 @@ int sg_ref_conv2d_points(int64_t KH, int64_t KW, int64_t C,
                 }
         out[i] = acc;
         if (sabs) sabs[i] = sab;
+    }
+    return 0;
+}
+
+/*
+ * Depthwise convolution, NHWC input, HWC filter (Section 4.6.3, "(2-D)"; the 1-D op is the
+ * case H = KH = 1 with Sh = Dh = 1):
+ *     O[n,h,w,c] = sum_{kh,kw} I[n, h*Sh + kh*Dh, w*Sw + kw*Dw, c] * K[kh,kw,c]
+ * iterators (n,h,w,c,kh,kw) = (parallel x4, reduction x2): the channel iterator is parallel,
+ * only the window is reduced.  No padding, filter not flipped, as for the dense convolutions.
+ */
+int sg_ref_depthwise_conv2d_nhwc_hwc(int64_t N, int64_t Ho, int64_t Wo, int64_t C,
+                                     int64_t KH, int64_t KW, int64_t H_in, int64_t W_in,
+                                     int64_t sh, int64_t sw, int64_t dh, int64_t dw,
+                                     const float *I, const int64_t *is /* n,h,w,c */,
+                                     const float *Kf, const int64_t *ks /* kh,kw,c */,
+                                     double *O, const int64_t *os /* n,h,w,c */,
+                                     double *S, int mode, int threads)
+{
+    if (N < 0 || Ho < 0 || Wo < 0 || C < 0 || KH < 0 || KW < 0) return 1;
+    if (sh < 1 || sw < 1 || dh < 1 || dw < 1) return 1;
+    if (Ho > 0 && KH > 0 && H_in < (Ho - 1) * sh + (KH - 1) * dh + 1) return 1;
+    if (Wo > 0 && KW > 0 && W_in < (Wo - 1) * sw + (KW - 1) * dw + 1) return 1;
+    int nt = use_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static) collapse(2)
+    for (int64_t n = 0; n < N; ++n) {
+        for (int64_t h = 0; h < Ho; ++h) {
+            for (int64_t w = 0; w < Wo; ++w) {
+                for (int64_t c = 0; c < C; ++c) {
+                    double acc = 0.0, sab = 0.0;
+                    for (int64_t kh = 0; kh < KH; ++kh) {
+                        for (int64_t kw = 0; kw < KW; ++kw) {
+                            double p = (double)I[n * is[0] + (h * sh + kh * dh) * is[1] +
+                                                 (w * sw + kw * dw) * is[2] + c * is[3]] *
+                                       (double)Kf[kh * ks[0] + kw * ks[1] + c * ks[2]];
+                            acc += p;
+                            sab += fabs(p);
+                        }
+                    }
+                    double *o = &O[n * os[0] + h * os[1] + w * os[2] + c * os[3]];
+                    *o = (mode ? *o : 0.0) + acc;
+                    if (S) S[((n * Ho + h) * Wo + w) * C + c] = sab;
+                }
+            }
+        }
     }
     return 0;
 }
