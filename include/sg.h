@@ -126,6 +126,39 @@ sg_status sg_conv2d_nhwc_hwcf(int64_t N, int64_t H_out, int64_t W_out, int64_t F
                               sg_dtype in_dtype, int mode, sg_stream_t stream);
 
 /*
+ * Depthwise 2-D convolution, input NHWC, filter HWC, output NHWC (Section 4.6.3, "(2-D)"):
+ *   O[n,h,w,c] (+)= sum_{kh,kw} I[n, h*sh + kh*dh, w*sw + kw*dw, c] * K[kh,kw,c]
+ * Iterators (n,h,w,c,kh,kw): the channel iterator is parallel, only the window is reduced.
+ * Same rules as the dense convolutions (no padding, filter not flipped, input large enough
+ * or SG_ERR_INVALID_ARG, strides in elements).  The op is bound by memory bandwidth and runs
+ * on the CUDA cores: four channels per thread when channels are contiguous in all three
+ * tensors, C is a multiple of 4 and pointers and pitches allow 16-byte (f32) / 8-byte (bf16)
+ * accesses; one element per thread otherwise.
+ *   I : N x H_in x W_in x C,    strides {n, h, w, c}
+ *   Kf: KH x KW x C,            strides {kh, kw, c}
+ *   O : N x H_out x W_out x C,  strides {n, h, w, c}   (f32)
+ */
+sg_status sg_depthwise_conv2d_nhwc_hwc(int64_t N, int64_t H_out, int64_t W_out, int64_t C, int64_t KH, int64_t KW,
+                                       int64_t H_in, int64_t W_in, int64_t stride_h, int64_t stride_w,
+                                       int64_t dilation_h, int64_t dilation_w,
+                                       const void *I, const int64_t i_strides[4],
+                                       const void *Kf, const int64_t k_strides[3],
+                                       float *O, const int64_t o_strides[4],
+                                       sg_dtype in_dtype, int mode, sg_stream_t stream);
+
+/*
+ * Depthwise 1-D convolution, input NWC, filter WC, output NWC (Section 4.6.3, "(1-D)"):
+ *   O[n,w,c] (+)= sum_kw I[n, w*sw + kw*dw, c] * K[kw,c]
+ * The 2-D op with H = KH = 1.   I strides {n, w, c}; Kf strides {kw, c}; O strides {n, w, c}.
+ */
+sg_status sg_depthwise_conv1d_nwc_wc(int64_t N, int64_t W_out, int64_t C, int64_t KW, int64_t W_in,
+                                     int64_t stride_w, int64_t dilation_w,
+                                     const void *I, const int64_t i_strides[3],
+                                     const void *Kf, const int64_t k_strides[2],
+                                     float *O, const int64_t o_strides[3],
+                                     sg_dtype in_dtype, int mode, sg_stream_t stream);
+
+/*
  * Synchronises `stream` and returns the current device's status word:
  * SG_OK, SG_ERR_DEVICE_TIMEOUT if any kernel since the last sg_check gave up
  * on a bounded wait (its output is then undefined), or SG_ERR_CUDA if the

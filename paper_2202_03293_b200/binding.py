@@ -22,7 +22,8 @@ SG_OVERWRITE, SG_ACCUMULATE = 0, 1
 SG_KERNEL_AUTO, SG_KERNEL_FFMA, SG_KERNEL_TENSOR, SG_KERNEL_CONV_STRIP = 0, 1, 2, 3
 
 EXPORTS = [
-    "sg_matmul", "sg_conv1d_nwc_wcf", "sg_conv2d_nhwc_hwcf", "sg_check", "sg_status_string",
+    "sg_matmul", "sg_conv1d_nwc_wcf", "sg_conv2d_nhwc_hwcf", "sg_depthwise_conv1d_nwc_wc",
+    "sg_depthwise_conv2d_nhwc_hwc", "sg_check", "sg_status_string",
     "sg_version", "sg_last_kernel", "sg_launch_count", "sg_set_kernel_override", "sg_set_tile_override",
     "sg_last_tile_choice", "sg_shutdown",
 ]
@@ -50,6 +51,10 @@ def lib() -> ctypes.CDLL:
         L.sg_conv1d_nwc_wcf.restype = ci
         L.sg_conv2d_nhwc_hwcf.argtypes = [i64] * 13 + [vp, p64, vp, p64, vp, p64, ci, ci, vp]
         L.sg_conv2d_nhwc_hwcf.restype = ci
+        L.sg_depthwise_conv2d_nhwc_hwc.argtypes = [i64] * 12 + [vp, p64, vp, p64, vp, p64, ci, ci, vp]
+        L.sg_depthwise_conv2d_nhwc_hwc.restype = ci
+        L.sg_depthwise_conv1d_nwc_wc.argtypes = [i64] * 7 + [vp, p64, vp, p64, vp, p64, ci, ci, vp]
+        L.sg_depthwise_conv1d_nwc_wc.restype = ci
         L.sg_check.argtypes = [vp]
         L.sg_check.restype = ci
         L.sg_status_string.argtypes = [ci]
@@ -143,6 +148,37 @@ def sg_conv2d_nhwc_hwcf(I: torch.Tensor, Kf: torch.Tensor, O: torch.Tensor, stri
                                    _arr(O.stride()), _dtype_code(I), mode, _stream(stream))
     if rc != SG_OK:
         raise SgError(rc, "sg_conv2d_nhwc_hwcf")
+    return O
+
+
+def sg_depthwise_conv2d_nhwc_hwc(I: torch.Tensor, Kf: torch.Tensor, O: torch.Tensor, stride=(1, 1), dilation=(1, 1),
+                                 mode: int = SG_OVERWRITE, stream=None) -> torch.Tensor:
+    """O[n,h,w,c] (+)= sum_{kh,kw} I[n, h*sh+kh*dh, w*sw+kw*dw, c] * Kf[kh,kw,c]."""
+    N, H_in, W_in, C = I.shape
+    KH, KW, C2 = Kf.shape
+    N2, H_out, W_out, C3 = O.shape
+    if C != C2 or C != C3 or N != N2 or O.dtype != torch.float32 or I.dtype != Kf.dtype:
+        raise ValueError("shape or dtype mismatch")
+    rc = lib().sg_depthwise_conv2d_nhwc_hwc(N, H_out, W_out, C, KH, KW, H_in, W_in, stride[0], stride[1], dilation[0],
+                                            dilation[1], _ptr(I), _arr(I.stride()), _ptr(Kf), _arr(Kf.stride()), _ptr(O),
+                                            _arr(O.stride()), _dtype_code(I), mode, _stream(stream))
+    if rc != SG_OK:
+        raise SgError(rc, "sg_depthwise_conv2d_nhwc_hwc")
+    return O
+
+
+def sg_depthwise_conv1d_nwc_wc(I: torch.Tensor, Kf: torch.Tensor, O: torch.Tensor, stride: int = 1, dilation: int = 1,
+                               mode: int = SG_OVERWRITE, stream=None) -> torch.Tensor:
+    """O[n,w,c] (+)= sum_kw I[n, w*sw+kw*dw, c] * Kf[kw,c]."""
+    N, W_in, C = I.shape
+    KW, C2 = Kf.shape
+    N2, W_out, C3 = O.shape
+    if C != C2 or C != C3 or N != N2 or O.dtype != torch.float32 or I.dtype != Kf.dtype:
+        raise ValueError("shape or dtype mismatch")
+    rc = lib().sg_depthwise_conv1d_nwc_wc(N, W_out, C, KW, W_in, stride, dilation, _ptr(I), _arr(I.stride()), _ptr(Kf),
+                                          _arr(Kf.stride()), _ptr(O), _arr(O.stride()), _dtype_code(I), mode, _stream(stream))
+    if rc != SG_OK:
+        raise SgError(rc, "sg_depthwise_conv1d_nwc_wc")
     return O
 
 

@@ -150,6 +150,53 @@ sg_status sg_conv2d_nhwc_hwcf(int64_t N, int64_t H_out, int64_t W_out, int64_t F
     return run(p, I, Kf, O, static_cast<cudaStream_t>(stream));
 }
 
+sg_status sg_depthwise_conv2d_nhwc_hwc(int64_t N, int64_t H_out, int64_t W_out, int64_t C, int64_t KH, int64_t KW,
+                                       int64_t H_in, int64_t W_in, int64_t stride_h, int64_t stride_w,
+                                       int64_t dilation_h, int64_t dilation_w, const void *I, const int64_t i_strides[4],
+                                       const void *Kf, const int64_t k_strides[3], float *O, const int64_t o_strides[4],
+                                       sg_dtype in_dtype, int mode, sg_stream_t stream) {
+    if (N < 0 || H_out < 0 || W_out < 0 || C < 0 || KH < 0 || KW < 0 || H_in < 0 || W_in < 0) return SG_ERR_INVALID_ARG;
+    if (stride_h < 1 || stride_w < 1 || dilation_h < 1 || dilation_w < 1) return SG_ERR_INVALID_ARG;
+    if (!i_strides || !k_strides || !o_strides) return SG_ERR_INVALID_ARG;
+    sg_status st = check_common(I, Kf, O, in_dtype, mode);
+    if (st != SG_OK) return st;
+    for (int i = 0; i < 4; ++i)
+        if (i_strides[i] < 0 || o_strides[i] < 0 || (i < 3 && k_strides[i] < 0)) return SG_ERR_INVALID_ARG;
+    if (!fits(N) || !fits(H_out) || !fits(W_out) || !fits(C) || !fits(KH) || !fits(KW) || !fits(H_in) || !fits(W_in) ||
+        !fits(stride_h) || !fits(stride_w) || !fits(dilation_h) || !fits(dilation_w)) return SG_ERR_UNSUPPORTED;
+    if (H_out > 0 && KH > 0 && H_in < (H_out - 1) * stride_h + (KH - 1) * dilation_h + 1) return SG_ERR_INVALID_ARG;
+    if (W_out > 0 && KW > 0 && W_in < (W_out - 1) * stride_w + (KW - 1) * dilation_w + 1) return SG_ERR_INVALID_ARG;
+    if (!fits(H_in * stride_h) || !fits(W_in * stride_w) || !fits(KH * KW)) return SG_ERR_UNSUPPORTED;
+    const bool has_out = N > 0 && H_out > 0 && W_out > 0 && C > 0;
+    if (!has_out) return SG_OK;
+    if (!O) return SG_ERR_INVALID_ARG;
+    if (KH * KW > 0 && (!I || !Kf)) return SG_ERR_INVALID_ARG;
+    if (KH * KW == 0 && mode == SG_ACCUMULATE) return SG_OK;      // empty window: the sum is 0
+    DepthwiseProblem p{};
+    p.N = (int)N; p.Ho = (int)H_out; p.Wo = (int)W_out; p.C = (int)C; p.KH = (int)KH; p.KW = (int)KW;
+    p.sh = (int)stride_h; p.sw = (int)stride_w; p.dh = (int)dilation_h; p.dw = (int)dilation_w;
+    p.i_n = i_strides[0]; p.i_h = i_strides[1]; p.i_w = i_strides[2]; p.i_c = i_strides[3];
+    p.k_kh = k_strides[0]; p.k_kw = k_strides[1]; p.k_c = k_strides[2];
+    p.o_n = o_strides[0]; p.o_h = o_strides[1]; p.o_w = o_strides[2]; p.o_c = o_strides[3];
+    p.in_bf16 = in_dtype == SG_BF16; p.accumulate = mode == SG_ACCUMULATE;
+    if (launch_depthwise(p, I, Kf, O, static_cast<cudaStream_t>(stream)) != cudaSuccess) return SG_ERR_CUDA;
+    t_last_kernel = SG_KERNEL_FFMA;     // a CUDA-core kernel
+    return SG_OK;
+}
+
+sg_status sg_depthwise_conv1d_nwc_wc(int64_t N, int64_t W_out, int64_t C, int64_t KW, int64_t W_in, int64_t stride_w,
+                                     int64_t dilation_w, const void *I, const int64_t i_strides[3], const void *Kf,
+                                     const int64_t k_strides[2], float *O, const int64_t o_strides[3], sg_dtype in_dtype,
+                                     int mode, sg_stream_t stream) {
+    if (!i_strides || !k_strides || !o_strides) return SG_ERR_INVALID_ARG;
+    // the 2-D op with H = KH = 1 (Section 4.6.3: "K_h and H are 1 in the 1-D case")
+    const int64_t is4[4] = {i_strides[0], 0, i_strides[1], i_strides[2]};
+    const int64_t ks3[3] = {0, k_strides[0], k_strides[1]};
+    const int64_t os4[4] = {o_strides[0], 0, o_strides[1], o_strides[2]};
+    return sg_depthwise_conv2d_nhwc_hwc(N, 1, W_out, C, 1, KW, 1, W_in, 1, stride_w, 1, dilation_w, I, is4, Kf, ks3, O, os4,
+                                        in_dtype, mode, stream);
+}
+
 sg_status sg_check(sg_stream_t stream) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaStreamSynchronize(s) != cudaSuccess) return SG_ERR_CUDA;

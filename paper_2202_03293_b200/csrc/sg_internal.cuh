@@ -58,6 +58,17 @@ void tensor_last_choice(int out[3]);
 // waits expire); the caller has already synchronised the stream.
 sg_status tensor_read_status(cudaStream_t stream);
 
+// Depthwise convolution (Section 4.6.3): O[n,h,w,c] (+)= sum_{kh,kw} I[n, h*sh+kh*dh, w*sw+kw*dw, c] * K[kh,kw,c].
+struct DepthwiseProblem {
+    int N, Ho, Wo, C, KH, KW;
+    int sh, sw, dh, dw;
+    int64_t i_n, i_h, i_w, i_c;
+    int64_t k_kh, k_kw, k_c;
+    int64_t o_n, o_h, o_w, o_c;
+    int in_bf16, accumulate;
+};
+cudaError_t launch_depthwise(const DepthwiseProblem &p, const void *I, const void *Kf, float *O, cudaStream_t stream);
+
 void count_launch(int n = 1);
 
 }  // namespace sg
