@@ -178,7 +178,20 @@ def op_specs(sg, seed):
                            torch.empty(Mx, Nx, device="cuda")),
                 lambda a, b, c: sg.sg_matmul(a, b, c))
 
+    def dw(Nx, Ho, Wo, Cx, KH, KW, st, dtype, label):
+        # bytes by the paper's model (Section 4.6.3): output + filter + input / prod gcd(stride, dilation)
+        es = 2 if dtype == "bf16" else 4
+        Hi, Wi = (Ho - 1) * st + KH, (Wo - 1) * st + KW
+        return (label, 2.0 * Nx * Ho * Wo * Cx * KH * KW, Nx * Ho * Wo * Cx * 4 + KH * KW * Cx * es + Nx * Hi * Wi * Cx * es, dtype,
+                lambda s: (gpu_operand((Nx, Hi, Wi, Cx), seed, 130 + s, "normal", dtype), gpu_operand((KH, KW, Cx), seed, 150, "normal", dtype),
+                           torch.empty(Nx, Ho, Wo, Cx, device="cuda")),
+                lambda i, k, o: sg.sg_depthwise_conv2d_nhwc_hwc(i, k, o, (st, st), (1, 1)))
+
     return {
+        "depthwise_112_f32": dw(1, 112, 112, 32, 3, 3, 1, "f32", "depthwise conv2d 1x114x114x32 * 3x3x32 f32 (MobileNet-like, batch 1)"),
+        "depthwise_batched_f32": dw(32, 112, 112, 64, 3, 3, 1, "f32", "depthwise conv2d 32x114x114x64 * 3x3x64 f32"),
+        "depthwise_batched_bf16": dw(32, 112, 112, 64, 3, 3, 1, "bf16", "depthwise conv2d 32x114x114x64 * 3x3x64 bf16"),
+        "depthwise_batched_s2_f32": dw(32, 56, 56, 128, 3, 3, 2, "f32", "depthwise conv2d 32x113x113x128 * 3x3x128 stride 2 f32"),
         "matmul128_f32": mm(128, 128, 128, "f32", "matmul 128^3 f32 (config 1)"),
         "matmul4096_bf16_atb": mm_t(4096, 4096, 4096, True, False, "matmul 4096^3 bf16, A stored transposed (A^T B)"),
         "matmul4096_bf16_abt": mm_t(4096, 4096, 4096, False, True, "matmul 4096^3 bf16, B stored transposed (A B^T)"),
