@@ -90,7 +90,7 @@ __device__ __forceinline__ void split4(const uint4 v, uint4 &h, uint4 &l) {
     }
 }
 
-template <int BN, int CG, bool F32, int KPS = 1>
+template <int BN, int CG, bool F32, int KPS = 1, bool TA = false>
 struct Cfg {
     // CG = 1: one CTA owns a 128 x BN tile.  CG = 2: a pair of CTAs (one cluster) owns a
     // 256 x BN tile; each CTA stages its own 128 input rows and its own BN/2 filter columns,
@@ -109,13 +109,20 @@ struct Cfg {
     // two slots holds what the converter warps make of them, [input hi | input lo | filter hi |
     // filter lo], the filter transposed to K-major on the way (kind::tf32 takes no N-major operand).
     static constexpr int SPLIT_SLOTS = F32 ? 2 : 0;
-    static constexpr int SPLIT_BYTES = 2 * STAGE_BYTES;
+    // TA (f32): the split input tile lives in tensor memory (the MMA reads its A operand there), which
+    // takes its writes and its three reads per k-step off the shared-memory pipe; a slot then holds
+    // [filter hi | filter lo] only.
+    static constexpr int SPLIT_BYTES = TA ? 2 * B_STAGE_BYTES : 2 * STAGE_BYTES;
     static constexpr int RING_BUDGET = 196608 - SPLIT_SLOTS * SPLIT_BYTES;
     static constexpr int STAGES = (RING_BUDGET / STAGE_BYTES) > 8 ? 8 : (RING_BUDGET / STAGE_BYTES);
     // warps: input producer, MMA, 4 epilogue (, 8 converter), filter producer
     static constexpr int THREADS = 192 + (F32 ? CONVERTER_THREADS : 0) + 32;
     static constexpr int FLT_WARP = THREADS / 32 - 1;
-    static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;      // two accumulator buffers
+    // two accumulator buffers (one when the split input's 2 slots x 64 columns would not fit beside two)
+    static constexpr int A_TMEM_COLS = TA ? 128 : 0;
+    static constexpr int ACC_BUFS = 2 * BN + A_TMEM_COLS > 512 ? 1 : 2;
+    static constexpr int USED_COLS = ACC_BUFS * BN + A_TMEM_COLS;
+    static constexpr int TMEM_COLS = USED_COLS <= 32 ? 32 : USED_COLS <= 64 ? 64 : USED_COLS <= 128 ? 128 : USED_COLS <= 256 ? 256 : 512;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SPLIT_SLOTS * SPLIT_BYTES + STAGING_BYTES +
                                       1024 /*alignment slack*/ + 256 /*barriers*/;
     static constexpr int B_KSTEP_DESC = 16 * ROW_BYTES / 16;   // bf16 filter tile, N-major: 16 k-rows per k-step
@@ -123,6 +130,7 @@ struct Cfg {
     static_assert(TMEM_COLS <= 512 && (TMEM_COLS & (TMEM_COLS - 1)) == 0, "TMEM columns");
     static_assert(STAGES >= 2 && STAGES <= 8, "ring depth");
     static_assert(KPS == 1 || (KPS == 2 && !F32), "k-blocks per stage");
+    static_assert(!TA || F32, "tensor-memory input operand: f32 path only");
 };
 
 // Static tile order: groups of 8 tile-rows, row index fastest inside a group, so that the
@@ -141,11 +149,12 @@ __device__ __forceinline__ void tile_coords(int t, int num_m_tiles, int num_n_ti
 // ([k][m], m contiguous: A^T B of Section 4.6.1) and consumed as an M-major operand; bit 1 = the
 // filter operand is stored transposed ([n][k], k contiguous: A B^T) and consumed K-major.
 template <int BN, int CG, bool F32, int KPS, int LAY>
-__global__ void __launch_bounds__(Cfg<BN, CG, F32, KPS>::THREADS, 1)
+__global__ void __launch_bounds__(Cfg<BN, CG, F32, KPS, (LAY & 4) != 0>::THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_flt,
                const __grid_constant__ CUtensorMap map_out, const TcParams p) {
-    using C = Cfg<BN, CG, F32, KPS>;
-    constexpr bool A_MN = (LAY & 1) != 0, B_KM = (LAY & 2) != 0;
+    constexpr bool A_MN = (LAY & 1) != 0, B_KM = (LAY & 2) != 0, TA = (LAY & 4) != 0;
+    using C = Cfg<BN, CG, F32, KPS, TA>;
+    static_assert(!TA || (F32 && !A_MN), "tensor-memory input operand: f32, input stored [m][k]");
     static_assert(LAY == 0 || KPS == 1, "transposed layouts: one k-block per stage");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -331,8 +340,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
             int it = 0, tl = 0;
             bool ok = true;
             for (int t = group_id; t < num_tiles && ok; t += num_groups, ++tl) {
-                const int buf = tl & 1;
-                if (!wait_all(mbar_wait(acc_empty_bar(buf), ((tl >> 1) & 1) ^ 1u, abort_flag))) { ok = false; break; }
+                const int buf = tl % C::ACC_BUFS;
+                if (!wait_all(mbar_wait(acc_empty_bar(buf), ((tl / C::ACC_BUFS) & 1) ^ 1u, abort_flag))) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 int tile, kb0, kb1;
@@ -342,6 +351,30 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                         const int s = it & 1;
                         if (!wait_all(mbar_wait<CG == 2>(split_full_bar(s), (it >> 1) & 1, abort_flag))) { ok = false; break; }
                         tc_fence_after();
+                        if constexpr (TA) {
+                            // filter hi | lo in the slot (K-major); input hi | lo in tensor memory, 32 columns
+                            // (k) each, lane = row: the MMA takes its A operand from there
+                            const uint32_t slot = split_addr + s * C::SPLIT_BYTES;
+                            const uint64_t bh = make_smem_desc(slot, 16, 1024);
+                            const uint64_t bl = make_smem_desc(slot + C::B_STAGE_BYTES, 16, 1024);
+                            const uint32_t a_hi = tmem_base + (uint32_t)(C::ACC_BUFS * BN + s * 64), a_lo = a_hi + 32;
+#pragma unroll
+                            for (int k = 0; k < K_STEPS; ++k) {
+                                const uint64_t o = (uint64_t)(k * 2);
+                                const uint32_t acc = (kb > kb0 || k > 0) ? 1u : 0u;
+                                if (issuer) {
+                                    if constexpr (CG == 1) {
+                                        umma_tf32_ts(d_tmem, a_lo + k * 8, bh + o, idesc, acc);   // small terms first
+                                        umma_tf32_ts(d_tmem, a_hi + k * 8, bl + o, idesc, 1u);
+                                        umma_tf32_ts(d_tmem, a_hi + k * 8, bh + o, idesc, 1u);
+                                    } else {
+                                        umma_tf32_ts_cg2(d_tmem, a_lo + k * 8, bh + o, idesc, acc);
+                                        umma_tf32_ts_cg2(d_tmem, a_hi + k * 8, bl + o, idesc, 1u);
+                                        umma_tf32_ts_cg2(d_tmem, a_hi + k * 8, bh + o, idesc, 1u);
+                                    }
+                                }
+                            }
+                        } else {
                         // slot: [input hi | input lo | filter hi | filter lo], all K-major: 8-row groups
                         // 1024 B apart, a k-step of 8 f32 is 32 B inside the swizzled 128-byte row
                         const uint32_t a_hi = split_addr + s * C::SPLIT_BYTES;
@@ -355,6 +388,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                             mma(d_tmem, al + o, bh + o, (kb > kb0 || k > 0) ? 1u : 0u);   // small terms first
                             mma(d_tmem, ah + o, bl + o, 1u);
                             mma(d_tmem, ah + o, bh + o, 1u);
+                        }
                         }
                         commit_all(split_empty_bar(s));
                     } else {
@@ -405,6 +439,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     const int r = it % C::STAGES, s = it & 1;
                     if (!mbar_wait(full_bar(r), (it / C::STAGES) & 1, abort_flag)) { ok = false; break; }
                     if (!mbar_wait<CG == 2>(split_empty_bar(s), ((it >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
+                    if constexpr (TA) tc_fence_after();     // the MMAs that read this slot's tensor-memory columns are done
                     const uint8_t *raw = smem_gen + r * C::STAGE_BYTES;
                     uint8_t *slot = smem_gen + C::STAGES * C::STAGE_BYTES + s * C::SPLIT_BYTES;
                     // An operand tile that arrives K-major (rows of 32 k, 128-byte swizzled by the TMA) is
@@ -457,14 +492,37 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     };
                     // input: K-major as stored, M-major when stored transposed; filter: N-major as stored,
                     // K-major when stored transposed.  kind::tf32 takes K-major operands only.
-                    if constexpr (A_MN) split_transpose(raw, slot, slot + A_STAGE_BYTES, std::integral_constant<int, BM>{});
-                    else split_elementwise(raw, slot, slot + A_STAGE_BYTES, std::integral_constant<int, A_STAGE_BYTES>{});
+                    uint8_t *b_slot = slot + (TA ? 0 : 2 * A_STAGE_BYTES);
+                    if constexpr (TA) {
+                        // input tile -> tensor memory: this warp may touch lane quarter (warp & 3); the two warps
+                        // of a quarter take 16 of the 32 k columns each.  Lane = row reads its 64 bytes of the
+                        // swizzled raw tile and stores 16 hi and 16 lo words.
+                        const int quarter = warp & 3, khalf = cw >> 2;
+                        const int row = quarter * 32 + lane;
+                        const uint8_t *rp = raw + row * 128;
+                        uint32_t hi[16], lo[16];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint4 v = *reinterpret_cast<const uint4 *>(rp + (((khalf * 4 + i) ^ (row & 7)) << 4));
+                            uint4 h, l;
+                            split4(v, h, l);
+                            hi[4 * i] = h.x; hi[4 * i + 1] = h.y; hi[4 * i + 2] = h.z; hi[4 * i + 3] = h.w;
+                            lo[4 * i] = l.x; lo[4 * i + 1] = l.y; lo[4 * i + 2] = l.z; lo[4 * i + 3] = l.w;
+                        }
+                        const uint32_t t_hi = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(C::ACC_BUFS * BN + s * 64 + khalf * 16);
+                        tmem_st_32x16(t_hi, hi);
+                        tmem_st_32x16(t_hi + 32, lo);
+                        tmem_st_wait();
+                        tc_fence_before();
+                    } else if constexpr (A_MN) {
+                        split_transpose(raw, slot, slot + A_STAGE_BYTES, std::integral_constant<int, BM>{});
+                    } else {
+                        split_elementwise(raw, slot, slot + A_STAGE_BYTES, std::integral_constant<int, A_STAGE_BYTES>{});
+                    }
                     if constexpr (B_KM)
-                        split_elementwise(raw + A_STAGE_BYTES, slot + 2 * A_STAGE_BYTES, slot + 2 * A_STAGE_BYTES + C::B_STAGE_BYTES,
-                                          std::integral_constant<int, C::B_STAGE_BYTES>{});
+                        split_elementwise(raw + A_STAGE_BYTES, b_slot, b_slot + C::B_STAGE_BYTES, std::integral_constant<int, C::B_STAGE_BYTES>{});
                     else
-                        split_transpose(raw + A_STAGE_BYTES, slot + 2 * A_STAGE_BYTES, slot + 2 * A_STAGE_BYTES + C::B_STAGE_BYTES,
-                                        std::integral_constant<int, C::B_COLS>{});
+                        split_transpose(raw + A_STAGE_BYTES, b_slot, b_slot + C::B_STAGE_BYTES, std::integral_constant<int, C::B_COLS>{});
                     fence_async_smem();     // generic-proxy writes -> visible to the tensor core's reads
                     __syncwarp();
                     if (lane == 0) {
@@ -490,10 +548,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
             int mt, nt;
             tile_coords(t / p.splits, p.num_m_tiles, p.num_n_tiles, mt, nt);
             const int m0 = (mt * CG + (int)cta_rank) * BM, n0 = nt * BN;
-            const int buf = tl & 1;
+            const int buf = tl % C::ACC_BUFS;
             // (the barrier's phase stays complete until these warps hand the buffer back, so the four
             // warps take the same way here and meet at every epi_sync below)
-            if (!mbar_wait(acc_full_bar(buf), (tl >> 1) & 1, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(acc_full_bar(buf), (tl / C::ACC_BUFS) & 1, abort_flag)) { ok = false; break; }
             tc_fence_after();
 #pragma unroll 1
             for (int j = 0; j < BN / 32; ++j, ++chunk_count) {
@@ -566,7 +624,7 @@ struct Driver {
     EncodeIm2colFn im2col = nullptr;
     int num_sms = 0;
     int device = -1;
-    bool attr_set[64] = {};
+    bool attr_set[96] = {};
     bool ok = false;
 };
 std::mutex g_mu;
@@ -575,6 +633,7 @@ int g_bn_override = -1;   // tile width forced by SG_TC_BN or sg_set_tile_overri
 int g_cg_override = 0;    // CTAs per tile (0: automatic)
 int g_split_override = 0; // k ranges per tile (0: automatic)
 int g_kps_override = 0;   // SG_TC_KPS=1 (testing): one k-block per stage everywhere
+int g_ta_override = -1;   // SG_TC_TA (testing): 0 never, 1 always keep the split f32 input tile in tensor memory
 int g_last_choice[3] = {0, 0, 0};
 
 bool init_driver() {
@@ -635,10 +694,11 @@ template <int BN, int CG, bool F32, int KPS, int LAY = 0>
 sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUtensorMap &mo, TcParams tp, int M, int N,
                          int slot, cudaStream_t stream) {
   if constexpr ((F32 && BN == 256 && CG == 1) || (KPS == 2 && (F32 || (BN == 256 && CG == 1))) ||
-                (LAY != 0 && (KPS != 1 || (BN == 256 && CG == 1) || (BN == 128 && CG == 2)))) {
+                ((LAY & 3) != 0 && (KPS != 1 || (BN == 256 && CG == 1) || (BN == 128 && CG == 2))) ||
+                ((LAY & 4) != 0 && (!F32 || (LAY & 3) != 0))) {
     return SG_ERR_INTERNAL;   // the split slots of a 128 x 256 f32 tile do not fit beside a TMA ring
   } else {
-    using C = Cfg<BN, CG, F32, KPS>;
+    using C = Cfg<BN, CG, F32, KPS, (LAY & 4) != 0>;
     if (!g_drv.attr_set[slot]) {
         if (cudaFuncSetAttribute(tc_gemm_kernel<BN, CG, F32, KPS, LAY>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
             return SG_ERR_CUDA;
@@ -707,6 +767,8 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         g_split_override = e ? atoi(e) : 0;
         e = getenv("SG_TC_KPS");
         g_kps_override = e ? atoi(e) : 0;
+        e = getenv("SG_TC_TA");
+        g_ta_override = e ? atoi(e) : -1;
     }
 
     alignas(64) CUtensorMap map_in, map_flt, map_out;
@@ -884,9 +946,14 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         tp.accumulate = 1;
     }
     g_last_choice[0] = kVariants[pick].bn; g_last_choice[1] = kVariants[pick].cg; g_last_choice[2] = splits;
-    const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0) + lay * 3 * kNumVariants;
+    // f32, plain layout: the split input tile goes to tensor memory unless that costs the second
+    // accumulator buffer (256 columns) on a reduction too short to pay for the lost overlap
+    const int lay_k = (f32 && lay == 0 && g_ta_override != 0 &&
+                       (kVariants[pick].bn < 256 || tp.kb_per_split >= 24 || g_ta_override == 1)) ? 4 : lay;
+    const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0) + lay_k * 3 * kNumVariants;
 #define SG_LAUNCH(BN_, CG_)                                                                                \
-    (f32 ? (lay == 0 ? launch_variant<BN_, CG_, true, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)         \
+    (f32 ? (lay_k == 4 ? launch_variant<BN_, CG_, true, 1, 4>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)     \
+            : lay == 0 ? launch_variant<BN_, CG_, true, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)         \
             : lay == 1 ? launch_variant<BN_, CG_, true, 1, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
             : lay == 2 ? launch_variant<BN_, CG_, true, 1, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
                        : launch_variant<BN_, CG_, true, 1, 3>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream))   \
