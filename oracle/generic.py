@@ -79,3 +79,46 @@ def depthwise_conv2d_maps(sh, sw, dh, dw):
     m_k = [[0, 0, 0, 0, 1, 0], [0, 0, 0, 0, 0, 1], [0, 0, 0, 1, 0, 0]]
     m_o = [[1, 0, 0, 0, 0, 0], [0, 1, 0, 0, 0, 0], [0, 0, 1, 0, 0, 0], [0, 0, 0, 1, 0, 0]]
     return m_in, m_k, m_o
+
+
+def evaluate_unary(domain, map_in, map_out, src, out_shape):
+    """out[map_out @ i] += src[map_in @ i] for every i in the domain (body: add, or a plain
+    assignment where every output index is reached once).  The memory-bound kernels of
+    Section 4.4 are this op with different maps.  Exact rational accumulation."""
+    domain = [int(d) for d in domain]
+    total = 1
+    for d in domain:
+        total *= d
+    acc = {}
+    for flat in range(total):
+        idx = []
+        rem = flat
+        for d in reversed(domain):
+            idx.append(rem % d)
+            rem //= d
+        idx.reverse()
+        k_in = tuple(sum(int(r[j]) * idx[j] for j in range(len(idx))) for r in map_in)
+        k_out = tuple(sum(int(r[j]) * idx[j] for j in range(len(idx))) for r in map_out)
+        acc[k_out] = acc.get(k_out, Fraction(0)) + Fraction(float(src[k_in]))
+    res = np.zeros(out_shape, np.float64)
+    for key, val in acc.items():
+        res[key] = float(val)
+    return res
+
+
+def copy2d_maps():
+    # iterators (i, j)
+    return [[1, 0], [0, 1]], [[1, 0], [0, 1]]
+
+
+def transpose2d_maps():
+    return [[1, 0], [0, 1]], [[0, 1], [1, 0]]
+
+
+def colred2d_maps():
+    # i is the reduction iterator: the output keeps j
+    return [[1, 0], [0, 1]], [[0, 1]]
+
+
+def rowred2d_maps():
+    return [[1, 0], [0, 1]], [[1, 0]]

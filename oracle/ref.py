@@ -194,3 +194,62 @@ def depthwise_conv1d_nwc_wc(I, Kf, stride=1, dilation=1, O_in=None, W_out=None, 
     out_hw = None if W_out is None else (1, W_out)
     O, S = depthwise_conv2d_nhwc_hwc(I[:, None], Kf[None], (1, stride), (1, dilation), O_in4, out_hw, threads)
     return O[:, 0], S[:, 0]
+
+
+def _elem_view(a):
+    """Bit-pattern view of a 2-D array of 2- or 4-byte elements (copy/transpose move bits)."""
+    a = np.asarray(a)
+    if a.ndim != 2 or a.itemsize not in (2, 4):
+        raise TypeError("expected a 2-D array of 2- or 4-byte elements")
+    return a.view(np.uint16 if a.itemsize == 2 else np.uint32)
+
+
+def copy2d(src):
+    """dst[i,j] = src[i,j] (Section 4.4, Copy2D); returns a dense array of src's dtype."""
+    v = _elem_view(src)
+    R, C = v.shape
+    dst = np.zeros((R, C), v.dtype)
+    ss = _estrides(v)
+    rc = lib().sg_ref_copy2d(_i64(R), _i64(C), _i64(v.itemsize), _ptr(v), _i64(ss[0]), _i64(ss[1]),
+                             _ptr(dst), _i64(C), _i64(1))
+    if rc:
+        raise ValueError("sg_ref_copy2d rejected its arguments")
+    return dst.view(np.asarray(src).dtype)
+
+
+def transpose2d(src):
+    """dst[j,i] = src[i,j] (Section 4.4, Transpose2D); returns a dense C x R array."""
+    v = _elem_view(src)
+    R, C = v.shape
+    dst = np.zeros((C, R), v.dtype)
+    ss = _estrides(v)
+    rc = lib().sg_ref_transpose2d(_i64(R), _i64(C), _i64(v.itemsize), _ptr(v), _i64(ss[0]), _i64(ss[1]),
+                                  _ptr(dst), _i64(R), _i64(1))
+    if rc:
+        raise ValueError("sg_ref_transpose2d rejected its arguments")
+    return dst.view(np.asarray(src).dtype)
+
+
+def _reduce2d(fn, A, n_out, out_in, threads):
+    A = _f32(A)
+    R, C = A.shape
+    mode = 0 if out_in is None else 1
+    out = np.zeros(n_out, np.float64) if out_in is None else np.array(out_in, dtype=np.float64, order="C")
+    assert out.shape == (n_out,)
+    S = np.zeros(n_out, np.float64)
+    sa = _estrides(A)
+    rc = fn(_i64(R), _i64(C), _ptr(A), _i64(sa[0]), _i64(sa[1]), _ptr(out), _ptr(S),
+            ctypes.c_int(mode), ctypes.c_int(threads))
+    if rc:
+        raise ValueError("the 2-D reduction rejected its arguments")
+    return out, S
+
+
+def colred2d(A, out_in=None, threads=0):
+    """out[j] = (out_in[j]) + sum_i A[i,j]: C outputs (Section 4.4, ColRed2D)."""
+    return _reduce2d(lib().sg_ref_colred2d, A, np.asarray(A).shape[1], out_in, threads)
+
+
+def rowred2d(A, out_in=None, threads=0):
+    """out[i] = (out_in[i]) + sum_j A[i,j]: R outputs (Section 4.4, RowRed2D)."""
+    return _reduce2d(lib().sg_ref_rowred2d, A, np.asarray(A).shape[0], out_in, threads)

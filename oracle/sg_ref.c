@@ -1,6 +1,6 @@
 /*
- * Reference (oracle) implementation of the structured contraction ops (and of the depthwise
- * convolutions, at the end of the file).
+ * Reference (oracle) implementation of the structured contraction ops (and, at the end of the
+ * file, of the depthwise convolutions and of the memory-bound 2-D kernels).
  *
  * THIS IS TEST INFRASTRUCTURE, NOT THE PRODUCT.  It is a deliberately plain,
  * slow CPU evaluation of each op's definition, used only to check the CUDA
@@ -261,6 +261,85 @@ int sg_ref_depthwise_conv2d_nhwc_hwc(int64_t N, int64_t Ho, int64_t Wo, int64_t 
                 }
             }
         }
+    }
+    return 0;
+}
+
+/*
+ * The memory-bound 2-D kernels (Section 4.4 "Benchmarks": Copy2D, Transpose2D, ColRed2D,
+ * RowRed2D; Section 4.5).  A is an R x C tensor read through its element strides.
+ *
+ *   Copy2D       dst[i,j] = src[i,j]                      iterators (i,j) parallel
+ *   Transpose2D  dst[j,i] = src[i,j]      (dst is C x R)  iterators (i,j) parallel
+ *   ColRed2D     out[j]   = sum_i A[i,j]  (out has C elements)   i is the reduction
+ *   RowRed2D     out[i]   = sum_j A[i,j]  (out has R elements)   j is the reduction
+ *
+ * Which reduction is which follows the caption of the L3 bandwidth figure: for a 250 x 960
+ * tensor the row reduction writes 250 values and the column reduction 960.  The reductions
+ * are sums (the paper ties them to matrix-vector products), accumulated in f64; `S` receives
+ * sum |a| per output element, `mode` 1 adds to the output (destination-passing).
+ * Copy and transpose move elements of `esize` bytes untouched, so they work on bit patterns.
+ */
+#include <string.h>
+
+int sg_ref_copy2d(int64_t R, int64_t C, int64_t esize, const void *src, int64_t ss0, int64_t ss1,
+                  void *dst, int64_t ds0, int64_t ds1)
+{
+    if (R < 0 || C < 0 || esize < 1) return 1;
+    for (int64_t i = 0; i < R; ++i)
+        for (int64_t j = 0; j < C; ++j)
+            memcpy((char *)dst + (i * ds0 + j * ds1) * esize,
+                   (const char *)src + (i * ss0 + j * ss1) * esize, (size_t)esize);
+    return 0;
+}
+
+int sg_ref_transpose2d(int64_t R, int64_t C, int64_t esize, const void *src, int64_t ss0, int64_t ss1,
+                       void *dst, int64_t ds0, int64_t ds1)
+{
+    if (R < 0 || C < 0 || esize < 1) return 1;
+    for (int64_t i = 0; i < R; ++i)
+        for (int64_t j = 0; j < C; ++j)
+            memcpy((char *)dst + (j * ds0 + i * ds1) * esize,
+                   (const char *)src + (i * ss0 + j * ss1) * esize, (size_t)esize);
+    return 0;
+}
+
+int sg_ref_colred2d(int64_t R, int64_t C, const float *A, int64_t as0, int64_t as1,
+                    double *out, double *S, int mode, int threads)
+{
+    if (R < 0 || C < 0) return 1;
+    int nt = use_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t j = 0; j < C; ++j) {
+        double acc = 0.0, sab = 0.0;
+        for (int64_t i = 0; i < R; ++i) {
+            double v = (double)A[i * as0 + j * as1];
+            acc += v;
+            sab += fabs(v);
+        }
+        out[j] = (mode ? out[j] : 0.0) + acc;
+        if (S) S[j] = sab;
+    }
+    return 0;
+}
+
+int sg_ref_rowred2d(int64_t R, int64_t C, const float *A, int64_t as0, int64_t as1,
+                    double *out, double *S, int mode, int threads)
+{
+    if (R < 0 || C < 0) return 1;
+    int nt = use_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t i = 0; i < R; ++i) {
+        double acc = 0.0, sab = 0.0;
+        for (int64_t j = 0; j < C; ++j) {
+            double v = (double)A[i * as0 + j * as1];
+            acc += v;
+            sab += fabs(v);
+        }
+        out[i] = (mode ? out[i] : 0.0) + acc;
+        if (S) S[i] = sab;
     }
     return 0;
 }
