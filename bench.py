@@ -46,6 +46,7 @@ NCU_TRAFFIC_BYTES = 25.5e6   # profiles/bench_sweep_launch_list.md: average over
 # tf32 : bf16 dense tensor throughput (nominal 1.1 : 2.25 PFLOP/s; the issue rate measured on
 # this chip is exactly half)
 TF32_OVER_BF16 = 0.5
+BW_ROWS, BW_COLS = 8192, 12288   # shape of the memory-bound 2-D kernels' rows in the per-op table
 
 
 def load_peaks():
@@ -187,7 +188,35 @@ def op_specs(sg, seed):
                            torch.empty(Nx, Ho, Wo, Cx, device="cuda")),
                 lambda i, k, o: sg.sg_depthwise_conv2d_nhwc_hwc(i, k, o, (st, st), (1, 1)))
 
+    bw_cache = {}
+
+    def bw_source(dtype):
+        # one seeded 8192 x 12288 tensor per dtype (403 / 201 MB, larger than L2); rotating sets are device copies
+        if dtype not in bw_cache:
+            bw_cache[dtype] = gpu_operand((BW_ROWS, BW_COLS), seed, 170, "uniform", dtype)
+        return bw_cache[dtype]
+
+    def bw(kind, dtype):
+        # the memory-bound 2-D kernels (Section 4.4); bytes = every input element read once, every output written once
+        es = 2 if dtype == "bf16" else 4
+        R, C = BW_ROWS, BW_COLS
+        tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+        if kind == "copy2d":
+            return (f"Copy2D {R}x{C} {dtype}", 0.0, 2 * R * C * es, dtype,
+                    lambda s: (bw_source(dtype).clone(), torch.empty(R, C, device="cuda", dtype=tdt)), lambda a, o: sg.sg_copy2d(a, o))
+        if kind == "transpose2d":
+            return (f"Transpose2D {R}x{C} {dtype}", 0.0, 2 * R * C * es, dtype,
+                    lambda s: (bw_source(dtype).clone(), torch.empty(C, R, device="cuda", dtype=tdt)), lambda a, o: sg.sg_transpose2d(a, o))
+        n_out = C if kind == "colred2d" else R
+        fn = sg.sg_colred2d if kind == "colred2d" else sg.sg_rowred2d
+        return (f"{'ColRed2D' if kind == 'colred2d' else 'RowRed2D'} {R}x{C} {dtype}", float(R * C), R * C * es + n_out * 4, dtype,
+                lambda s: (bw_source(dtype).clone(), torch.empty(n_out, device="cuda")), lambda a, o: fn(a, o))
+
     return {
+        "copy2d_f32": bw("copy2d", "f32"), "copy2d_bf16": bw("copy2d", "bf16"),
+        "transpose2d_f32": bw("transpose2d", "f32"), "transpose2d_bf16": bw("transpose2d", "bf16"),
+        "colred2d_f32": bw("colred2d", "f32"), "rowred2d_f32": bw("rowred2d", "f32"),
+        "colred2d_bf16": bw("colred2d", "bf16"), "rowred2d_bf16": bw("rowred2d", "bf16"),
         "depthwise_112_f32": dw(1, 112, 112, 32, 3, 3, 1, "f32", "depthwise conv2d 1x114x114x32 * 3x3x32 f32 (MobileNet-like, batch 1)"),
         "depthwise_batched_f32": dw(32, 112, 112, 64, 3, 3, 1, "f32", "depthwise conv2d 32x114x114x64 * 3x3x64 f32"),
         "depthwise_batched_bf16": dw(32, 112, 112, 64, 3, 3, 1, "bf16", "depthwise conv2d 32x114x114x64 * 3x3x64 bf16"),
@@ -239,7 +268,8 @@ def measure_op(sg, peaks, spec, reps=None):
     tf = flops / (ms * 1e-3) / 1e12
     tensor_peak = peaks["bf16_tflops"] * (TF32_OVER_BF16 if dtype == "f32" else 1.0)
     on_tensor = fam in (sg.SG_KERNEL_TENSOR, sg.SG_KERNEL_CONV_STRIP)
-    kernel_name = {sg.SG_KERNEL_TENSOR: "tensor", sg.SG_KERNEL_CONV_STRIP: "tensor (conv strip)"}.get(fam, "ffma")
+    kernel_name = {sg.SG_KERNEL_TENSOR: "tensor", sg.SG_KERNEL_CONV_STRIP: "tensor (conv strip)",
+                   sg.SG_KERNEL_TMA_MOVE: "tma move"}.get(fam, "cuda cores")
     t_compute = flops / ((tensor_peak if on_tensor else ffma_peak) * 1e12)
     t_bytes = bytes_ / (peaks["hbm_gbs"] * 1e9)
     bound = max(t_compute, t_bytes)

@@ -67,8 +67,9 @@ enum {
     SG_KERNEL_AUTO = 0,
     SG_KERNEL_FFMA = 1,        /* strided CUDA-core kernel, any layout                                   */
     SG_KERNEL_TENSOR = 2,      /* TMA + tcgen05 implicit GEMM (matmul; convolutions through TMA im2col)  */
-    SG_KERNEL_CONV_STRIP = 3   /* tcgen05 kernel for stride-1 bf16 convolutions: resident filter, each
+    SG_KERNEL_CONV_STRIP = 3,  /* tcgen05 kernel for stride-1 bf16 convolutions: resident filter, each
                                   input pixel fetched once per tile                                      */
+    SG_KERNEL_TMA_MOVE = 4     /* copy / transpose that move every tile with TMA loads and stores        */
 };
 
 /*
@@ -159,6 +160,40 @@ sg_status sg_depthwise_conv1d_nwc_wc(int64_t N, int64_t W_out, int64_t C, int64_
                                      sg_dtype in_dtype, int mode, sg_stream_t stream);
 
 /*
+ * The memory-bound 2-D kernels (Section 4.4, "Benchmarks": Copy2D, Transpose2D, ColRed2D,
+ * RowRed2D; measured in Section 4.5).  All operate on an R x C tensor whose element (i,j) is at
+ * base[i*stride_r + j*stride_c] (strides in elements, any non-negative values).
+ *
+ * Copy2D:       dst[i,j] = src[i,j]        dst is R x C
+ * Transpose2D:  dst[j,i] = src[i,j]        dst is C x R; dst_stride_r is the pitch of ITS rows
+ *                                          (index j), dst_stride_c the step along i
+ * Elements are moved as bit patterns of `dtype`'s size (4 bytes for SG_F32, 2 for SG_BF16);
+ * nothing is converted.  dst must not overlap src.  With unit column strides, 16-byte aligned
+ * bases and row pitches that are multiples of 16 bytes the call runs on TMA-only kernels
+ * (SG_KERNEL_TMA_MOVE); any other layout runs on a strided CUDA-core kernel.
+ */
+sg_status sg_copy2d(int64_t R, int64_t C, const void *src, int64_t src_stride_r, int64_t src_stride_c,
+                    void *dst, int64_t dst_stride_r, int64_t dst_stride_c, sg_dtype dtype, sg_stream_t stream);
+sg_status sg_transpose2d(int64_t R, int64_t C, const void *src, int64_t src_stride_r, int64_t src_stride_c,
+                         void *dst, int64_t dst_stride_r, int64_t dst_stride_c, sg_dtype dtype, sg_stream_t stream);
+
+/*
+ * ColRed2D:  out[j] (+)= sum_i A[i,j]   C outputs (the row index is reduced)
+ * RowRed2D:  out[i] (+)= sum_j A[i,j]   R outputs (the column index is reduced)
+ * The caption of the paper's L3 bandwidth figure fixes the naming: for a 250 x 960 tensor the
+ * row reduction writes 250 values, the column reduction 960.  A holds `in_dtype` elements, the
+ * sums are accumulated and written in f32 (bf16 inputs are widened exactly); out[k] is at
+ * out[k*out_stride].  mode as for the contractions; an empty reduction writes 0 (SG_OVERWRITE)
+ * or leaves out untouched (SG_ACCUMULATE).  When the shape has too few outputs to occupy the
+ * GPU the reduced index is split across thread blocks whose partial sums are added into `out`
+ * with float atomics, so the rounding of the last bits may differ from call to call.
+ */
+sg_status sg_colred2d(int64_t R, int64_t C, const void *A, int64_t a_stride_r, int64_t a_stride_c,
+                      float *out, int64_t out_stride, sg_dtype in_dtype, int mode, sg_stream_t stream);
+sg_status sg_rowred2d(int64_t R, int64_t C, const void *A, int64_t a_stride_r, int64_t a_stride_c,
+                      float *out, int64_t out_stride, sg_dtype in_dtype, int mode, sg_stream_t stream);
+
+/*
  * Synchronises `stream` and returns the current device's status word:
  * SG_OK, SG_ERR_DEVICE_TIMEOUT if any kernel since the last sg_check gave up
  * on a bounded wait (its output is then undefined), or SG_ERR_CUDA if the
@@ -174,7 +209,8 @@ int sg_version(void);
 
 /*
  * Which kernel family the most recent successful call on this host thread
- * selected: SG_KERNEL_FFMA, SG_KERNEL_TENSOR or SG_KERNEL_CONV_STRIP (0 before any call).
+ * selected: SG_KERNEL_FFMA (any CUDA-core kernel), SG_KERNEL_TENSOR, SG_KERNEL_CONV_STRIP or
+ * SG_KERNEL_TMA_MOVE (0 before any call).
  */
 int sg_last_kernel(void);
 
@@ -190,7 +226,8 @@ int64_t sg_launch_count(void);
  * convolution kernel where it applies, else the tensor-core GEMM, else the
  * CUDA-core kernel).  Forcing SG_KERNEL_TENSOR or SG_KERNEL_CONV_STRIP makes
  * calls that kernel cannot take return SG_ERR_UNSUPPORTED instead of falling
- * back.
+ * back.  For sg_copy2d / sg_transpose2d, SG_KERNEL_FFMA forces the strided kernel and
+ * SG_KERNEL_TMA_MOVE the TMA kernel (SG_ERR_UNSUPPORTED when the layout rules it out).
  */
 sg_status sg_set_kernel_override(int kernel_family);
 

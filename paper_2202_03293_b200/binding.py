@@ -19,11 +19,11 @@ _lib = None
 SG_OK = 0
 SG_F32, SG_BF16 = 0, 1
 SG_OVERWRITE, SG_ACCUMULATE = 0, 1
-SG_KERNEL_AUTO, SG_KERNEL_FFMA, SG_KERNEL_TENSOR, SG_KERNEL_CONV_STRIP = 0, 1, 2, 3
+SG_KERNEL_AUTO, SG_KERNEL_FFMA, SG_KERNEL_TENSOR, SG_KERNEL_CONV_STRIP, SG_KERNEL_TMA_MOVE = 0, 1, 2, 3, 4
 
 EXPORTS = [
     "sg_matmul", "sg_conv1d_nwc_wcf", "sg_conv2d_nhwc_hwcf", "sg_depthwise_conv1d_nwc_wc",
-    "sg_depthwise_conv2d_nhwc_hwc", "sg_check", "sg_status_string",
+    "sg_depthwise_conv2d_nhwc_hwc", "sg_copy2d", "sg_transpose2d", "sg_colred2d", "sg_rowred2d", "sg_check", "sg_status_string",
     "sg_version", "sg_last_kernel", "sg_launch_count", "sg_set_kernel_override", "sg_set_tile_override",
     "sg_last_tile_choice", "sg_shutdown",
 ]
@@ -55,6 +55,12 @@ def lib() -> ctypes.CDLL:
         L.sg_depthwise_conv2d_nhwc_hwc.restype = ci
         L.sg_depthwise_conv1d_nwc_wc.argtypes = [i64] * 7 + [vp, p64, vp, p64, vp, p64, ci, ci, vp]
         L.sg_depthwise_conv1d_nwc_wc.restype = ci
+        for fn in (L.sg_copy2d, L.sg_transpose2d):
+            fn.argtypes = [i64, i64, vp, i64, i64, vp, i64, i64, ci, vp]
+            fn.restype = ci
+        for fn in (L.sg_colred2d, L.sg_rowred2d):
+            fn.argtypes = [i64, i64, vp, i64, i64, vp, i64, ci, ci, vp]
+            fn.restype = ci
         L.sg_check.argtypes = [vp]
         L.sg_check.restype = ci
         L.sg_status_string.argtypes = [ci]
@@ -180,6 +186,47 @@ def sg_depthwise_conv1d_nwc_wc(I: torch.Tensor, Kf: torch.Tensor, O: torch.Tenso
     if rc != SG_OK:
         raise SgError(rc, "sg_depthwise_conv1d_nwc_wc")
     return O
+
+
+def _move2d(fn, name, src: torch.Tensor, dst: torch.Tensor, want_shape, stream):
+    if src.dim() != 2 or tuple(dst.shape) != tuple(want_shape) or src.dtype != dst.dtype:
+        raise ValueError(f"{name}: shape or dtype mismatch")
+    R, C = src.shape
+    rc = fn(R, C, _ptr(src), src.stride(0), src.stride(1), _ptr(dst), dst.stride(0), dst.stride(1), _dtype_code(src),
+            _stream(stream))
+    if rc != SG_OK:
+        raise SgError(rc, name)
+    return dst
+
+
+def sg_copy2d(src: torch.Tensor, dst: torch.Tensor, stream=None) -> torch.Tensor:
+    """dst[i,j] = src[i,j]."""
+    return _move2d(lib().sg_copy2d, "sg_copy2d", src, dst, src.shape, stream)
+
+
+def sg_transpose2d(src: torch.Tensor, dst: torch.Tensor, stream=None) -> torch.Tensor:
+    """dst[j,i] = src[i,j]; dst is C x R."""
+    return _move2d(lib().sg_transpose2d, "sg_transpose2d", src, dst, (src.shape[1], src.shape[0]), stream)
+
+
+def _reduce2d(fn, name, A: torch.Tensor, out: torch.Tensor, n_out, mode, stream):
+    if A.dim() != 2 or out.dim() != 1 or out.shape[0] != n_out or out.dtype != torch.float32:
+        raise ValueError(f"{name}: shape or dtype mismatch")
+    R, C = A.shape
+    rc = fn(R, C, _ptr(A), A.stride(0), A.stride(1), _ptr(out), out.stride(0), _dtype_code(A), int(mode), _stream(stream))
+    if rc != SG_OK:
+        raise SgError(rc, name)
+    return out
+
+
+def sg_colred2d(A: torch.Tensor, out: torch.Tensor, mode: int = SG_OVERWRITE, stream=None) -> torch.Tensor:
+    """out[j] (+)= sum_i A[i,j]."""
+    return _reduce2d(lib().sg_colred2d, "sg_colred2d", A, out, A.shape[1], mode, stream)
+
+
+def sg_rowred2d(A: torch.Tensor, out: torch.Tensor, mode: int = SG_OVERWRITE, stream=None) -> torch.Tensor:
+    """out[i] (+)= sum_j A[i,j]."""
+    return _reduce2d(lib().sg_rowred2d, "sg_rowred2d", A, out, A.shape[0], mode, stream)
 
 
 def sg_check(stream=None) -> None:

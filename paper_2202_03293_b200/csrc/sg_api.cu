@@ -197,6 +197,63 @@ sg_status sg_depthwise_conv1d_nwc_wc(int64_t N, int64_t W_out, int64_t C, int64_
                                         in_dtype, mode, stream);
 }
 
+namespace {
+sg_status move2d(bool transpose, int64_t R, int64_t C, const void *src, int64_t s_r, int64_t s_c, void *dst, int64_t d_r, int64_t d_c,
+                 sg_dtype dtype, sg_stream_t stream) {
+    using namespace sg;
+    if (dtype != SG_F32 && dtype != SG_BF16) return SG_ERR_UNSUPPORTED;
+    if (R < 0 || C < 0 || s_r < 0 || s_c < 0 || d_r < 0 || d_c < 0) return SG_ERR_INVALID_ARG;
+    if (!fits(R) || !fits(C)) return SG_ERR_UNSUPPORTED;
+    if (R == 0 || C == 0) return SG_OK;
+    if (!src || !dst) return SG_ERR_INVALID_ARG;
+    const int es = dtype == SG_BF16 ? 2 : 4;
+    if (reinterpret_cast<uintptr_t>(src) % es || reinterpret_cast<uintptr_t>(dst) % es) return SG_ERR_ALIGNMENT;
+    const int ov = g_override.load();
+    const int force = ov == SG_KERNEL_FFMA ? 1 : (ov == SG_KERNEL_TMA_MOVE ? 2 : 0);
+    int used_tma = 0;
+    const sg_status st = launch_move2d(transpose, R, C, src, s_r, s_c, dst, d_r, d_c, es, force, &used_tma, static_cast<cudaStream_t>(stream));
+    if (st == SG_OK) t_last_kernel = used_tma ? SG_KERNEL_TMA_MOVE : SG_KERNEL_FFMA;
+    return st;
+}
+
+sg_status reduce2d(bool colred, int64_t R, int64_t C, const void *A, int64_t a_r, int64_t a_c, float *out, int64_t out_stride,
+                   sg_dtype in_dtype, int mode, sg_stream_t stream) {
+    using namespace sg;
+    sg_status st = check_common(A, nullptr, out, in_dtype, mode);
+    if (st != SG_OK) return st;
+    if (R < 0 || C < 0 || a_r < 0 || a_c < 0 || out_stride < 0) return SG_ERR_INVALID_ARG;
+    if (!fits(R) || !fits(C)) return SG_ERR_UNSUPPORTED;
+    const int64_t n_out = colred ? C : R, n_red = colred ? R : C;
+    if (n_out == 0) return SG_OK;
+    if (!out || (n_red > 0 && !A)) return SG_ERR_INVALID_ARG;
+    if (n_red == 0 && mode == SG_ACCUMULATE) return SG_OK;
+    st = launch_reduce2d(colred, R, C, A, a_r, a_c, in_dtype == SG_BF16, out, out_stride, mode == SG_ACCUMULATE,
+                         static_cast<cudaStream_t>(stream));
+    if (st == SG_OK) t_last_kernel = SG_KERNEL_FFMA;     // CUDA-core kernels
+    return st;
+}
+}  // namespace
+
+sg_status sg_copy2d(int64_t R, int64_t C, const void *src, int64_t src_stride_r, int64_t src_stride_c, void *dst,
+                    int64_t dst_stride_r, int64_t dst_stride_c, sg_dtype dtype, sg_stream_t stream) {
+    return move2d(false, R, C, src, src_stride_r, src_stride_c, dst, dst_stride_r, dst_stride_c, dtype, stream);
+}
+
+sg_status sg_transpose2d(int64_t R, int64_t C, const void *src, int64_t src_stride_r, int64_t src_stride_c, void *dst,
+                         int64_t dst_stride_r, int64_t dst_stride_c, sg_dtype dtype, sg_stream_t stream) {
+    return move2d(true, R, C, src, src_stride_r, src_stride_c, dst, dst_stride_r, dst_stride_c, dtype, stream);
+}
+
+sg_status sg_colred2d(int64_t R, int64_t C, const void *A, int64_t a_stride_r, int64_t a_stride_c, float *out, int64_t out_stride,
+                      sg_dtype in_dtype, int mode, sg_stream_t stream) {
+    return reduce2d(true, R, C, A, a_stride_r, a_stride_c, out, out_stride, in_dtype, mode, stream);
+}
+
+sg_status sg_rowred2d(int64_t R, int64_t C, const void *A, int64_t a_stride_r, int64_t a_stride_c, float *out, int64_t out_stride,
+                      sg_dtype in_dtype, int mode, sg_stream_t stream) {
+    return reduce2d(false, R, C, A, a_stride_r, a_stride_c, out, out_stride, in_dtype, mode, stream);
+}
+
 sg_status sg_check(sg_stream_t stream) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaStreamSynchronize(s) != cudaSuccess) return SG_ERR_CUDA;
@@ -224,7 +281,7 @@ int64_t sg_launch_count(void) { return g_launches.load(); }
 
 sg_status sg_set_kernel_override(int kernel_family) {
     if (kernel_family != SG_KERNEL_AUTO && kernel_family != SG_KERNEL_FFMA && kernel_family != SG_KERNEL_TENSOR &&
-        kernel_family != SG_KERNEL_CONV_STRIP)
+        kernel_family != SG_KERNEL_CONV_STRIP && kernel_family != SG_KERNEL_TMA_MOVE)
         return SG_ERR_INVALID_ARG;
     g_override.store(kernel_family);
     return SG_OK;

@@ -1,0 +1,571 @@
+// The memory-bound 2-D kernels (Section 4.4: Copy2D, Transpose2D, ColRed2D, RowRed2D).
+//
+//   Copy2D       dst[i,j] = src[i,j]
+//   Transpose2D  dst[j,i] = src[i,j]
+//   ColRed2D     out[j] (+)= sum_i A[i,j]
+//   RowRed2D     out[i] (+)= sum_j A[i,j]
+//
+// All four are bound by HBM traffic; the kernels differ in how they keep enough bytes in flight.
+//   - Copy2D and Transpose2D, when the layout meets the TMA rules (unit column stride, 16-byte
+//     aligned bases and row pitches), move tiles with TMA only: a persistent CTA per SM slot runs
+//     a shared-memory ring that one thread fills with tensor loads and another drains with tensor
+//     stores.  The copy never touches the data with an ordinary instruction; the transpose has
+//     four warps turn each 128-row tile around in shared memory (16-byte reads of the 128-byte
+//     swizzled input tile, a register transpose of an E x E block, 16-byte writes into the
+//     swizzled output tile) between the load and the store.  Ragged edges cost nothing: loads
+//     read zeros beyond the tensor, stores are clipped.
+//   - The reductions use plain 16-byte loads with four in flight per thread at full occupancy,
+//     f32 accumulators, and a shared-memory / shuffle tree per CTA.  When the shape has too few
+//     independent outputs to fill the chip, the reduced index is split across CTAs and the
+//     partial sums meet in the output through float atomics (an overwriting call clears the
+//     output first); nothing but the operands is read or written.
+//   - Anything else (non-unit column strides, unaligned pitches) runs on strided 32 x 32 tile
+//     kernels.
+#include <algorithm>
+
+#include "sg_internal.cuh"
+#include "sg_tc_ptx.cuh"
+
+namespace sg {
+namespace {
+
+__device__ __forceinline__ void named_sync_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Bounded, flag-free wait used only while winding down after a time-out: lets copies that are
+// still in flight land before the CTA gives its shared memory back.
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+    for (int i = 0; i < (1 << 20); ++i)
+        if (mbar_try_wait(bar, parity)) return;
+}
+
+// ------------------------------------------------------------------------------ Copy2D (TMA)
+constexpr int CP_STAGES = 6;
+constexpr int CP_STORES_IN_FLIGHT = 2;
+constexpr int CP_STAGE_BYTES = 32768;
+
+// Tiles are dealt round-robin to the CTAs; warp 0 loads, warp 1 stores, one lane each.
+__global__ void __launch_bounds__(64) copy_tma_kernel(const __grid_constant__ CUtensorMap map_src,
+                                                       const __grid_constant__ CUtensorMap map_dst, int tiles_x, int num_tiles,
+                                                       int box_x, int box_y, uint32_t box_bytes) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[CP_STAGES], empty_bar[CP_STAGES];
+    __shared__ int abort_load, abort_store;
+    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < CP_STAGES; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        abort_load = 0; abort_store = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 0 && lane == 0) {
+        prefetch_tensormap(&map_src);
+        int k = 0;
+        for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++k) {
+            const int s = k % CP_STAGES;
+            const uint32_t ph = (uint32_t)(k / CP_STAGES) & 1u;
+            if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, &abort_load)) break;
+            mbar_expect_tx(smem_u32(&full_bar[s]), box_bytes);
+            tma_load_2d(ring + (uint32_t)s * CP_STAGE_BYTES, &map_src, smem_u32(&full_bar[s]), (t % tiles_x) * box_x, (t / tiles_x) * box_y);
+        }
+        if (abort_load)   // gave up: let the loads already issued land
+            for (int j = (k > CP_STAGES ? k - CP_STAGES : 0); j < k; ++j) mbar_drain(smem_u32(&full_bar[j % CP_STAGES]), (uint32_t)(j / CP_STAGES) & 1u);
+    } else if (warp == 1 && lane == 0) {
+        prefetch_tensormap(&map_dst);
+        int k = 0;
+        for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++k) {
+            const int s = k % CP_STAGES;
+            const uint32_t ph = (uint32_t)(k / CP_STAGES) & 1u;
+            if (!mbar_wait(smem_u32(&full_bar[s]), ph, &abort_store)) break;
+            tma_store_2d(&map_dst, ring + (uint32_t)s * CP_STAGE_BYTES, (t % tiles_x) * box_x, (t / tiles_x) * box_y);
+            bulk_commit();
+            if (k >= CP_STORES_IN_FLIGHT) {   // the store issued CP_STORES_IN_FLIGHT tiles ago has read its stage
+                bulk_wait_read<CP_STORES_IN_FLIGHT>();
+                mbar_arrive(smem_u32(&empty_bar[(k - CP_STORES_IN_FLIGHT) % CP_STAGES]));
+            }
+        }
+        bulk_wait_all();
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------- Transpose2D (TMA)
+// One tile = 128 input rows x 128 bytes (W = 128/ES columns).  Input stage: the tile as TMA wrote
+// it with the 128-byte swizzle (16-byte chunk index XOR row mod 8).  Output staging: the W x 128
+// transposed tile as 128/W blocks of [W rows][128 bytes], same swizzle, stored by four tensor
+// stores of 32 rows each (one per transposer warp).
+constexpr int TR_IN_STAGES = 4;
+constexpr int TR_TILE_BYTES = 16384;
+constexpr int TR_THREADS = 32 + 128;
+
+template <int ES>
+__device__ __forceinline__ void transpose_block(const uint4 (&v)[16 / ES], uint4 (&o)[16 / ES]) {
+    if constexpr (ES == 4) {
+        o[0] = make_uint4(v[0].x, v[1].x, v[2].x, v[3].x);
+        o[1] = make_uint4(v[0].y, v[1].y, v[2].y, v[3].y);
+        o[2] = make_uint4(v[0].z, v[1].z, v[2].z, v[3].z);
+        o[3] = make_uint4(v[0].w, v[1].w, v[2].w, v[3].w);
+    } else {
+        // 8 x 8 block of 2-byte elements: output row j gathers element j of every input row
+        uint32_t in[8][4], out[8][4];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) { in[r][0] = v[r].x; in[r][1] = v[r].y; in[r][2] = v[r].z; in[r][3] = v[r].w; }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+            for (int w = 0; w < 4; ++w)
+                out[j][w] = __byte_perm(in[2 * w][j >> 1], in[2 * w + 1][j >> 1], (j & 1) ? 0x7632 : 0x5410);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) o[j] = make_uint4(out[j][0], out[j][1], out[j][2], out[j][3]);
+    }
+}
+
+template <int ES>
+__global__ void __launch_bounds__(TR_THREADS) transpose_tma_kernel(const __grid_constant__ CUtensorMap map_src,
+                                                                    const __grid_constant__ CUtensorMap map_dst, int tiles_c,
+                                                                    int num_tiles, int dst_cols, int dst_rows) {
+    constexpr int E = 16 / ES;       // elements per 16-byte chunk = side of the register block
+    constexpr int W = 128 / ES;      // input columns per tile = output rows per tile
+    constexpr int P = 128 / E;       // row groups per tile
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[TR_IN_STAGES], empty_bar[TR_IN_STAGES];
+    __shared__ int abort_load, abort_turn;
+    const uint32_t in_ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t out_ring = in_ring + TR_IN_STAGES * TR_TILE_BYTES;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < TR_IN_STAGES; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 4); }
+        abort_load = 0; abort_turn = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 0) {
+        if (lane == 0) {
+            prefetch_tensormap(&map_src);
+            int k = 0;
+            for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++k) {
+                const int s = k % TR_IN_STAGES;
+                const uint32_t ph = (uint32_t)(k / TR_IN_STAGES) & 1u;
+                if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, &abort_load)) break;
+                mbar_expect_tx(smem_u32(&full_bar[s]), TR_TILE_BYTES);
+                tma_load_2d(in_ring + (uint32_t)s * TR_TILE_BYTES, &map_src, smem_u32(&full_bar[s]), (t % tiles_c) * W, (t / tiles_c) * 128);
+            }
+            if (abort_load)
+                for (int j = (k > TR_IN_STAGES ? k - TR_IN_STAGES : 0); j < k; ++j)
+                    mbar_drain(smem_u32(&full_bar[j % TR_IN_STAGES]), (uint32_t)(j / TR_IN_STAGES) & 1u);
+        }
+    } else {
+        const int w = warp - 1;
+        if (w == 0 && lane == 0) prefetch_tensormap(&map_dst);
+        // lanes of a quarter-warp take two row groups x four chunks: conflict-free 16-byte reads
+        const int q_lo = (lane & 3) | ((lane >> 1) & 4);
+        const int p_lo = ((lane >> 2) & 1) | ((lane >> 3) & 2);
+        int k = 0;
+        for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++k) {
+            const int s = k % TR_IN_STAGES;
+            const uint32_t ph = (uint32_t)(k / TR_IN_STAGES) & 1u;
+            mbar_wait(smem_u32(&full_bar[s]), ph, &abort_turn);       // a time-out sets abort_turn before the barrier below
+            if (lane == 0) bulk_wait_read<1>();                        // this warp's store from two tiles ago has read its staging
+            named_sync_128();
+            if (abort_turn) break;                                     // same answer in all 128 threads
+            const uint32_t in_tile = in_ring + (uint32_t)s * TR_TILE_BYTES;
+            const uint32_t out_tile = out_ring + (uint32_t)(k & 1) * TR_TILE_BYTES;
+#pragma unroll
+            for (int i = 0; i < P / 16; ++i) {
+                const int p = p_lo | (w << 2) | (i << 4);
+                const int q = q_lo;
+                uint4 v[E], o[E];
+#pragma unroll
+                for (int kk = 0; kk < E; ++kk) {
+                    const int row = E * p + kk;
+                    const uint32_t addr = in_tile + (uint32_t)row * 128u + (uint32_t)((q ^ (row & 7)) << 4);
+                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v[kk].x), "=r"(v[kk].y), "=r"(v[kk].z), "=r"(v[kk].w) : "r"(addr));
+                }
+                transpose_block<ES>(v, o);
+#pragma unroll
+                for (int j = 0; j < E; ++j) {
+                    const int c = E * q + j;                       // output row within the tile
+                    const uint32_t addr = out_tile + (uint32_t)(p >> 3) * (uint32_t)(W * 128) + (uint32_t)c * 128u +
+                                          (uint32_t)(((p & 7) ^ (c & 7)) << 4);
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(o[j].x), "r"(o[j].y), "r"(o[j].z), "r"(o[j].w) : "memory");
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&empty_bar[s]));       // the input stage may be refilled
+            fence_async_smem();                                        // staging writes -> visible to the tensor store
+            named_sync_128();
+            if (lane == 0) {
+                // store w: block w / (W/32) of the staging, rows (w % (W/32)) * 32 .. + 31; 4 KB each, back to back
+                const int b = w / (W / 32), h = w % (W / 32);
+                const int x = (t / tiles_c) * 128 + b * W, y = (t % tiles_c) * W + h * 32;
+                if (x < dst_cols && y < dst_rows) tma_store_2d(&map_dst, out_tile + (uint32_t)w * 4096u, x, y);
+                bulk_commit();
+            }
+        }
+        if (lane == 0) bulk_wait_all();
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------ strided 32 x 32 tile kernel
+// dst[i*d_i + j*d_j] = src[i*s_i + j*s_j]; a transpose is the same call with the destination
+// strides exchanged.  WRITE_BY_I: consecutive threads write consecutive i (the destination is
+// contiguous along i), else consecutive j.
+template <typename U, bool WRITE_BY_I>
+__global__ void __launch_bounds__(256) tile_move_kernel(const U *__restrict__ src, int64_t s_i, int64_t s_j, U *__restrict__ dst,
+                                                         int64_t d_i, int64_t d_j, int R, int C, int tiles_j, int64_t num_tiles) {
+    __shared__ U tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int64_t t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+        const int i0 = (int)(t / tiles_j) * 32, j0 = (int)(t % tiles_j) * 32;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int i = i0 + ty + 8 * k, j = j0 + tx;
+            if (i < R && j < C) tile[ty + 8 * k][tx] = src[(int64_t)i * s_i + (int64_t)j * s_j];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if constexpr (WRITE_BY_I) {
+                const int i = i0 + tx, j = j0 + ty + 8 * k;
+                if (i < R && j < C) dst[(int64_t)i * d_i + (int64_t)j * d_j] = tile[tx][ty + 8 * k];
+            } else {
+                const int i = i0 + ty + 8 * k, j = j0 + tx;
+                if (i < R && j < C) dst[(int64_t)i * d_i + (int64_t)j * d_j] = tile[ty + 8 * k][tx];
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// --------------------------------------------------------------------------------- reductions
+template <typename T, int VEC>
+struct Chunk {
+    float f[VEC];
+};
+
+__device__ __forceinline__ float widen(float x) { return x; }
+__device__ __forceinline__ float widen(uint16_t bits) { return __uint_as_float((uint32_t)bits << 16); }
+
+// Adds up to VEC consecutive elements starting at `ptr` (element stride `sc`) into acc.
+// `nvalid` == VEC takes the 16-byte path (VEC > 1 implies sc == 1 and an aligned address).
+template <typename T, int VEC>
+__device__ __forceinline__ void add_chunk(float (&acc)[VEC], const T *ptr, int64_t sc, int nvalid) {
+    if constexpr (VEC > 1) {
+        if (nvalid == VEC) {
+            const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(ptr));
+            if constexpr (sizeof(T) == 4) {
+                acc[0] += __uint_as_float(raw.x); acc[1] += __uint_as_float(raw.y);
+                acc[2] += __uint_as_float(raw.z); acc[3] += __uint_as_float(raw.w);
+            } else {
+                const uint32_t wds[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    acc[2 * w] += __uint_as_float(wds[w] << 16);
+                    acc[2 * w + 1] += __uint_as_float(wds[w] & 0xFFFF0000u);
+                }
+            }
+            return;
+        }
+    }
+#pragma unroll
+    for (int v = 0; v < VEC; ++v)
+        if (v < nvalid) acc[v] += widen(__ldg(ptr + (int64_t)v * sc));
+}
+
+// ColRed2D.  A CTA owns `cw` chunks of VEC columns and the rows [r0, r1) of its split;
+// thread (g, cc) = (t / cw, t % cw) walks rows r0+g, r0+g+rp, ... of chunk cc.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) colred_kernel(const T *__restrict__ A, int64_t ld, int64_t sc, int R, int C,
+                                                      float *__restrict__ out, int64_t os, int cw, int rp, int rows_per_split,
+                                                      int use_atomic, int accumulate) {
+    __shared__ float red[256][VEC + 1];
+    const int t = threadIdx.x, g = t / cw, cc = t - g * cw;
+    const int64_t col0 = ((int64_t)blockIdx.x * cw + cc) * VEC;
+    const int r0 = blockIdx.y * rows_per_split;
+    const int r1 = min(R, r0 + rows_per_split);
+    float acc[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
+    const bool active = g < rp && col0 < C;
+    const int nvalid = active ? (int)min((int64_t)VEC, (int64_t)C - col0) : 0;
+    if (active) {
+        const T *base = A + col0 * sc;
+        int64_t r = r0 + g;
+        for (; r + 3 * rp < r1; r += 4 * rp) {
+            float a0[VEC], a1[VEC], a2[VEC], a3[VEC];
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) a0[v] = a1[v] = a2[v] = a3[v] = 0.f;
+            add_chunk<T, VEC>(a0, base + r * ld, sc, nvalid);
+            add_chunk<T, VEC>(a1, base + (r + rp) * ld, sc, nvalid);
+            add_chunk<T, VEC>(a2, base + (r + 2 * rp) * ld, sc, nvalid);
+            add_chunk<T, VEC>(a3, base + (r + 3 * rp) * ld, sc, nvalid);
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[v] += (a0[v] + a1[v]) + (a2[v] + a3[v]);
+        }
+        for (; r < r1; r += rp) add_chunk<T, VEC>(acc, base + r * ld, sc, nvalid);
+    }
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) red[t][v] = acc[v];
+    __syncthreads();
+    if (g == 0 && col0 < C) {
+        for (int gg = 1; gg < rp; ++gg)
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[v] += red[gg * cw + cc][v];
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) {
+            if (v < nvalid) {
+                float *o = out + (col0 + v) * os;
+                if (use_atomic) atomicAdd(o, acc[v]);
+                else *o = (accumulate ? *o : 0.f) + acc[v];
+            }
+        }
+    }
+}
+
+// RowRed2D.  `lanes` (a power of two <= 32) lanes share a row; a warp holds 32/lanes rows.
+// blockIdx.y selects the column range [c0, c1) of a split (whole chunks except at the end).
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) rowred_kernel(const T *__restrict__ A, int64_t ld, int64_t sc, int R, int C,
+                                                      float *__restrict__ out, int64_t os, int lanes, int cols_per_split,
+                                                      int use_atomic, int accumulate) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int rows_per_warp = 32 / lanes;
+    const int64_t row = ((int64_t)blockIdx.x * 8 + warp) * rows_per_warp + lane / lanes;
+    const int sub = lane % lanes;
+    const int c0 = blockIdx.y * cols_per_split;
+    const int c1 = min(C, c0 + cols_per_split);
+    float acc[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) acc[v] = 0.f;
+    if (row < R && c0 < c1) {
+        const T *base = A + row * ld;
+        const int full_end = c0 + (c1 - c0) / VEC * VEC;      // whole chunks
+        int64_t c = c0 + sub * VEC;
+        const int64_t step = lanes * VEC;
+        for (; c + 3 * step < full_end; c += 4 * step) {
+            float a0[VEC], a1[VEC], a2[VEC], a3[VEC];
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) a0[v] = a1[v] = a2[v] = a3[v] = 0.f;
+            add_chunk<T, VEC>(a0, base + c * sc, sc, VEC);
+            add_chunk<T, VEC>(a1, base + (c + step) * sc, sc, VEC);
+            add_chunk<T, VEC>(a2, base + (c + 2 * step) * sc, sc, VEC);
+            add_chunk<T, VEC>(a3, base + (c + 3 * step) * sc, sc, VEC);
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[v] += (a0[v] + a1[v]) + (a2[v] + a3[v]);
+        }
+        for (; c < full_end; c += step) add_chunk<T, VEC>(acc, base + c * sc, sc, VEC);
+        if (VEC > 1 && sub == 0 && full_end < c1) {            // the ragged end of the range, element by element
+            float tail = 0.f;
+            for (int cc = full_end; cc < c1; ++cc) tail += widen(__ldg(base + (int64_t)cc * sc));
+            acc[0] += tail;
+        }
+    }
+    float sum = acc[0];
+#pragma unroll
+    for (int v = 1; v < VEC; ++v) sum += acc[v];
+    for (int off = lanes >> 1; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    if (sub == 0 && row < R && (c0 < c1 || blockIdx.y == 0)) {
+        float *o = out + row * os;
+        if (use_atomic) atomicAdd(o, sum);
+        else *o = (accumulate ? *o : 0.f) + sum;
+    }
+}
+
+__global__ void zero_vector_kernel(float *__restrict__ out, int64_t n, int64_t os) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) out[i * os] = 0.f;
+}
+
+inline bool aligned16(const void *p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
+
+template <typename T, int VEC>
+cudaError_t launch_reduce_typed(bool colred, const T *A, int64_t ld, int64_t sc, int R, int C, float *out, int64_t os,
+                                int accumulate, int num_sms, cudaStream_t stream) {
+    const int target_ctas = num_sms * 8;
+    if (!colred) {
+        // RowRed2D: one output per row
+        const int chunks = (C + VEC - 1) / VEC;
+        int lanes = 1;
+        while (lanes < 32 && lanes < chunks) lanes <<= 1;
+        const int rows_per_cta = 8 * (32 / lanes);
+        const int64_t row_ctas = ((int64_t)R + rows_per_cta - 1) / rows_per_cta;
+        int splits = 1;
+        const int min_chunks_per_split = lanes * 16;
+        if (row_ctas < target_ctas && chunks > min_chunks_per_split)
+            splits = (int)std::min<int64_t>((target_ctas + row_ctas - 1) / row_ctas, (chunks + min_chunks_per_split - 1) / min_chunks_per_split);
+        int chunks_per_split = (chunks + splits - 1) / splits;
+        chunks_per_split = (chunks_per_split + lanes - 1) / lanes * lanes;
+        splits = (chunks + chunks_per_split - 1) / chunks_per_split;
+        const int use_atomic = splits > 1;
+        if (use_atomic && !accumulate) {
+            zero_vector_kernel<<<(int)std::min<int64_t>(((int64_t)R + 255) / 256, 1184), 256, 0, stream>>>(out, R, os);
+            count_launch();
+        }
+        rowred_kernel<T, VEC><<<dim3((unsigned)row_ctas, (unsigned)splits), 256, 0, stream>>>(A, ld, sc, R, C, out, os, lanes,
+                                                                                              chunks_per_split * VEC, use_atomic, accumulate);
+    } else {
+        // ColRed2D: one output per column
+        const int64_t chunks = ((int64_t)C + VEC - 1) / VEC;
+        const int cw = (int)std::min<int64_t>(chunks, 256);
+        const int rp = 256 / cw;
+        const int64_t col_blocks = (chunks + cw - 1) / cw;
+        int splits = 1;
+        const int min_rows_per_split = rp * 16;
+        if (col_blocks < target_ctas && R > min_rows_per_split)
+            splits = (int)std::min<int64_t>((target_ctas + col_blocks - 1) / col_blocks, ((int64_t)R + min_rows_per_split - 1) / min_rows_per_split);
+        int rows_per_split = (R + splits - 1) / splits;
+        rows_per_split = (rows_per_split + rp - 1) / rp * rp;
+        splits = (R + rows_per_split - 1) / rows_per_split;
+        const int use_atomic = splits > 1;
+        if (use_atomic && !accumulate) {
+            zero_vector_kernel<<<(int)std::min<int64_t>(((int64_t)C + 255) / 256, 1184), 256, 0, stream>>>(out, C, os);
+            count_launch();
+        }
+        colred_kernel<T, VEC><<<dim3((unsigned)col_blocks, (unsigned)splits), 256, 0, stream>>>(A, ld, sc, R, C, out, os, cw, rp,
+                                                                                                rows_per_split, use_atomic, accumulate);
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+template <typename U>
+cudaError_t launch_tile_move(const U *src, int64_t s_i, int64_t s_j, U *dst, int64_t d_i, int64_t d_j, int R, int C, int num_sms,
+                             cudaStream_t stream) {
+    const int tiles_j = (C + 31) / 32;
+    const int64_t num_tiles = (int64_t)((R + 31) / 32) * tiles_j;
+    const int grid = (int)std::min<int64_t>(num_tiles, (int64_t)num_sms * 8);
+    // write along whichever destination index is closer to contiguous
+    if (d_i < d_j) tile_move_kernel<U, true><<<grid, 256, 0, stream>>>(src, s_i, s_j, dst, d_i, d_j, R, C, tiles_j, num_tiles);
+    else tile_move_kernel<U, false><<<grid, 256, 0, stream>>>(src, s_i, s_j, dst, d_i, d_j, R, C, tiles_j, num_tiles);
+    count_launch();
+    return cudaGetLastError();
+}
+
+bool g_attr_copy = false, g_attr_tr4 = false, g_attr_tr2 = false;
+
+}  // namespace
+
+sg_status launch_move2d(bool transpose, int64_t R, int64_t C, const void *src, int64_t s_r, int64_t s_c, void *dst, int64_t d_r,
+                        int64_t d_c, int esize, int force, int *used_tma, cudaStream_t stream) {
+    *used_tma = 0;
+    int num_sms = 0;
+    if (!tensor_driver_ready(&num_sms)) return SG_ERR_CUDA;
+    const bool tma_ok = force != 1 && s_c == 1 && d_c == 1 && aligned16(src) && aligned16(dst) && (s_r * esize) % 16 == 0 &&
+                        (d_r * esize) % 16 == 0 && s_r * esize < ((int64_t)1 << 40) && d_r * esize < ((int64_t)1 << 40) &&
+                        (R == 1 || s_r >= C) && ((transpose ? C : R) == 1 || d_r >= (transpose ? R : C));
+    const CUtensorMapDataType type = esize == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32 : CU_TENSOR_MAP_DATA_TYPE_UINT16;
+    // TMA checks the bounds of the contiguous dimension in 16-byte units, so a store would write the rest of the unit
+    // in which a row of the destination ends: the TMA kernels take the part whose destination rows are whole units
+    // (`body`), the strided kernel the last few columns of the destination.
+    const int vec = 16 / esize;
+    const int64_t inner = transpose ? R : C;             // extent of the destination's contiguous dimension
+    const int64_t body = inner - inner % vec, tail = inner - body;
+    if (tma_ok && body > 0 && (tail == 0 || force != 2)) {
+        const int64_t Rb = transpose ? body : R, Cb = transpose ? C : body;      // the source part the TMA kernel moves
+        bool launched = false;
+        CUtensorMap map_src, map_dst;
+        cuuint64_t st_src[1] = {(cuuint64_t)(s_r * esize)}, st_dst[1] = {(cuuint64_t)(d_r * esize)};
+        if (!transpose) {
+            // box: up to 256 elements wide, as many rows as fit a 32 KB stage
+            const int box_x = (int)std::min<int64_t>(256, Cb);
+            const int box_y = (int)std::min<int64_t>(std::min<int64_t>(256, CP_STAGE_BYTES / (box_x * esize)), Rb);
+            cuuint64_t dims[2] = {(cuuint64_t)Cb, (cuuint64_t)Rb};
+            cuuint32_t box[2] = {(cuuint32_t)box_x, (cuuint32_t)box_y};
+            const int64_t tiles_x = (Cb + box_x - 1) / box_x, tiles_y = (Rb + box_y - 1) / box_y;
+            if (tiles_x * tiles_y < ((int64_t)1 << 31) &&
+                tensor_encode_tiled(&map_src, type, 2, const_cast<void *>(src), dims, st_src, box, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B) &&
+                tensor_encode_tiled(&map_dst, type, 2, dst, dims, st_dst, box, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B)) {
+                const int smem = CP_STAGES * CP_STAGE_BYTES + 1024;
+                if (!g_attr_copy) {
+                    if (cudaFuncSetAttribute(copy_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SG_ERR_CUDA;
+                    g_attr_copy = true;
+                }
+                const int num_tiles = (int)(tiles_x * tiles_y);
+                copy_tma_kernel<<<std::min(num_tiles, num_sms), 64, smem, stream>>>(map_src, map_dst, (int)tiles_x, num_tiles, box_x, box_y,
+                                                                                    (uint32_t)(box_x * box_y * esize));
+                launched = true;
+            }
+        } else {
+            const int W = 128 / esize;
+            cuuint64_t dims_s[2] = {(cuuint64_t)Cb, (cuuint64_t)Rb}, dims_d[2] = {(cuuint64_t)Rb, (cuuint64_t)Cb};
+            cuuint32_t box_s[2] = {(cuuint32_t)W, 128}, box_d[2] = {(cuuint32_t)W, 32};
+            const int64_t tiles_c = (Cb + W - 1) / W, tiles_r = (Rb + 127) / 128;
+            if (tiles_c * tiles_r < ((int64_t)1 << 31) &&
+                tensor_encode_tiled(&map_src, type, 2, const_cast<void *>(src), dims_s, st_src, box_s, CU_TENSOR_MAP_SWIZZLE_128B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B) &&
+                tensor_encode_tiled(&map_dst, type, 2, dst, dims_d, st_dst, box_d, CU_TENSOR_MAP_SWIZZLE_128B,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B)) {
+                const int smem = (TR_IN_STAGES + 2) * TR_TILE_BYTES + 1024;
+                bool &attr = esize == 4 ? g_attr_tr4 : g_attr_tr2;
+                if (!attr) {
+                    const cudaError_t e = esize == 4
+                        ? cudaFuncSetAttribute(transpose_tma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
+                        : cudaFuncSetAttribute(transpose_tma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+                    if (e != cudaSuccess) return SG_ERR_CUDA;
+                    attr = true;
+                }
+                const int num_tiles = (int)(tiles_c * tiles_r);
+                const int grid = std::min(num_tiles, 2 * num_sms);
+                if (esize == 4) transpose_tma_kernel<4><<<grid, TR_THREADS, smem, stream>>>(map_src, map_dst, (int)tiles_c, num_tiles, (int)Rb, (int)Cb);
+                else transpose_tma_kernel<2><<<grid, TR_THREADS, smem, stream>>>(map_src, map_dst, (int)tiles_c, num_tiles, (int)Rb, (int)Cb);
+                launched = true;
+            }
+        }
+        if (launched) {
+            count_launch();
+            *used_tma = 1;
+            if (cudaGetLastError() != cudaSuccess) return SG_ERR_CUDA;
+            if (tail == 0) return SG_OK;
+            // the last `tail` columns of the destination: source rows [body, R) of a transpose, columns [body, C) of a copy
+            const char *s_tail = static_cast<const char *>(src) + (transpose ? body * s_r : body * s_c) * esize;
+            char *d_tail = static_cast<char *>(dst) + body * d_c * esize;
+            const int64_t Rt = transpose ? tail : R, Ct = transpose ? C : tail;
+            const int64_t di = transpose ? d_c : d_r, dj = transpose ? d_r : d_c;
+            const cudaError_t e = esize == 4
+                ? launch_tile_move(reinterpret_cast<const uint32_t *>(s_tail), s_r, s_c, reinterpret_cast<uint32_t *>(d_tail), di, dj, (int)Rt, (int)Ct, num_sms, stream)
+                : launch_tile_move(reinterpret_cast<const uint16_t *>(s_tail), s_r, s_c, reinterpret_cast<uint16_t *>(d_tail), di, dj, (int)Rt, (int)Ct, num_sms, stream);
+            return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
+        }
+    }
+    if (force == 2) return SG_ERR_UNSUPPORTED;
+    // strided path: destination index pair (i, j) of the source element; a transpose exchanges the strides
+    const int64_t di = transpose ? d_c : d_r, dj = transpose ? d_r : d_c;
+    const cudaError_t e = esize == 4
+        ? launch_tile_move(static_cast<const uint32_t *>(src), s_r, s_c, static_cast<uint32_t *>(dst), di, dj, (int)R, (int)C, num_sms, stream)
+        : launch_tile_move(static_cast<const uint16_t *>(src), s_r, s_c, static_cast<uint16_t *>(dst), di, dj, (int)R, (int)C, num_sms, stream);
+    return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
+}
+
+sg_status launch_reduce2d(bool colred, int64_t R, int64_t C, const void *A, int64_t a_r, int64_t a_c, int in_bf16, float *out,
+                          int64_t os, int accumulate, cudaStream_t stream) {
+    int num_sms = 0;
+    if (!tensor_driver_ready(&num_sms)) return SG_ERR_CUDA;
+    const int64_t n_out = colred ? C : R, n_red = colred ? R : C;
+    if (n_red == 0) {      // empty sum: the neutral value
+        if (!accumulate) {
+            zero_vector_kernel<<<(int)std::min<int64_t>((n_out + 255) / 256, 1184), 256, 0, stream>>>(out, n_out, os);
+            count_launch();
+            if (cudaGetLastError() != cudaSuccess) return SG_ERR_CUDA;
+        }
+        return SG_OK;
+    }
+    const int es = in_bf16 ? 2 : 4;
+    const bool vec_ok = a_c == 1 && aligned16(A) && (a_r * es) % 16 == 0;
+    cudaError_t e;
+    if (in_bf16) {
+        const uint16_t *p = static_cast<const uint16_t *>(A);
+        e = vec_ok ? launch_reduce_typed<uint16_t, 8>(colred, p, a_r, a_c, (int)R, (int)C, out, os, accumulate, num_sms, stream)
+                   : launch_reduce_typed<uint16_t, 1>(colred, p, a_r, a_c, (int)R, (int)C, out, os, accumulate, num_sms, stream);
+    } else {
+        const float *p = static_cast<const float *>(A);
+        e = vec_ok ? launch_reduce_typed<float, 4>(colred, p, a_r, a_c, (int)R, (int)C, out, os, accumulate, num_sms, stream)
+                   : launch_reduce_typed<float, 1>(colred, p, a_r, a_c, (int)R, (int)C, out, os, accumulate, num_sms, stream);
+    }
+    return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
+}
+
+sg_status bandwidth_read_status(cudaStream_t stream) { return read_status_word(stream); }
+
+}  // namespace sg

@@ -345,6 +345,7 @@ sg_status launch_conv_strip(const Problem &p, const void *In, const void *Flt, f
     if (reinterpret_cast<uintptr_t>(In) % 16 || reinterpret_cast<uintptr_t>(Flt) % 16 || reinterpret_cast<uintptr_t>(O) % 16)
         return SG_ERR_UNSUPPORTED;
     if (!mult(p.i_w * es, 16) || !mult(p.k_c * es, 16)) return SG_ERR_UNSUPPORTED;
+    if (!mult((int64_t)p.C * es, 16) || !mult((int64_t)p.N * es, 16)) return SG_ERR_UNSUPPORTED;   // TMA bounds work in 16-byte units
     if (p.KW > 1 && !mult(p.k_kw * es, 16)) return SG_ERR_UNSUPPORTED;
     if (p.KH > 1 && !mult(p.k_kh * es, 16)) return SG_ERR_UNSUPPORTED;
     if (!mult(p.o_w, 4) || (p.Ho > 1 && !mult(p.o_h, 4)) || (p.batch > 1 && !mult(p.o_n, 4)) || !mult(p.N, 4)) return SG_ERR_UNSUPPORTED;

@@ -69,6 +69,16 @@ struct DepthwiseProblem {
 };
 cudaError_t launch_depthwise(const DepthwiseProblem &p, const void *I, const void *Kf, float *O, cudaStream_t stream);
 
+// The memory-bound 2-D kernels (Section 4.4).  launch_move2d: dst[i,j] = src[i,j], or dst[j,i] = src[i,j] when
+// `transpose`; elements of `esize` (2 or 4) bytes, strides in elements; `force` 0 picks, 1 = strided kernel only, 2 = TMA
+// kernel or SG_ERR_UNSUPPORTED; *used_tma reports whether the TMA kernels ran.
+// launch_reduce2d: out[j] (+)= sum_i A[i,j] when `colred`, else out[i] (+)= sum_j A[i,j].
+sg_status launch_move2d(bool transpose, int64_t R, int64_t C, const void *src, int64_t s_r, int64_t s_c, void *dst, int64_t d_r,
+                        int64_t d_c, int esize, int force, int *used_tma, cudaStream_t stream);
+sg_status launch_reduce2d(bool colred, int64_t R, int64_t C, const void *A, int64_t a_r, int64_t a_c, int in_bf16, float *out,
+                          int64_t os, int accumulate, cudaStream_t stream);
+sg_status bandwidth_read_status(cudaStream_t stream);
+
 void count_launch(int n = 1);
 
 }  // namespace sg

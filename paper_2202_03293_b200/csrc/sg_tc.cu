@@ -746,6 +746,10 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         reinterpret_cast<uintptr_t>(O) % 16) return SG_ERR_UNSUPPORTED;
     const int64_t a_pitch = a_mn ? p.i_c : p.i_w, b_pitch = b_km ? p.k_f : p.k_c;     // elements between rows as stored
     if (!mult(a_pitch * es, 16) || !mult(b_pitch * es, 16) || !mult(p.o_w * 4, 16)) return SG_ERR_UNSUPPORTED;
+    // TMA checks the bounds of the contiguous dimension in 16-byte units: an extent that ends inside a unit would
+    // let loads read, and stores write, the rest of that unit (row padding), so such extents are left to the CUDA-core kernel
+    if (!mult((a_mn ? (int64_t)p.M : (int64_t)p.C) * es, 16) || !mult((b_km ? (int64_t)p.K : (int64_t)p.N) * es, 16) ||
+        !mult((int64_t)p.N * 4, 16)) return SG_ERR_UNSUPPORTED;
     if (a_mn && (p.M % BK != 0 || a_pitch < p.M)) return SG_ERR_UNSUPPORTED;   // whole sub-tile blocks of m (64 bf16 / 32 f32 rows)
     if (b_km && b_pitch < p.K) return SG_ERR_UNSUPPORTED;
     if (p.Ho > 1 && p.o_h != (int64_t)p.Wo * p.o_w) return SG_ERR_UNSUPPORTED;
@@ -975,7 +979,8 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
 sg_status tensor_read_status(cudaStream_t stream) {
     const sg_status a = read_status_word(stream);
     const sg_status b = conv_read_status(stream);
-    return a != SG_OK ? a : b;
+    const sg_status c = bandwidth_read_status(stream);
+    return a != SG_OK ? a : (b != SG_OK ? b : c);
 }
 
 bool tensor_driver_ready(int *num_sms) {

@@ -242,6 +242,24 @@ def test_matmul_padded_rows_and_offsets():
     assert torch.all(Cbig[:, :4] == 0)
 
 
+def test_padded_rows_whose_extent_ends_inside_a_16_byte_unit():
+    # aligned pitches, but K and N end inside a 16-byte unit: TMA would read and write the rest of that unit (the row
+    # padding, NaN here), so the call must not take the tensor path; nothing outside the views may change
+    M, N, K = 130, 57, 43
+    for dtype in ("bf16", "f32"):
+        Abig, a = operand((M, 48), SEED, 60, "uniform", dtype)
+        Bbig, b = operand((K, 64), SEED, 61, "uniform", dtype)
+        Abig[:, K:] = float("nan")
+        Bbig[:, N:] = float("nan")
+        Cbig = torch.full((M, 64), float("nan"), device="cuda")
+        sg.sg_matmul(Abig[:, :K], Bbig[:, :N], Cbig[:, :N])
+        torch.cuda.synchronize()
+        assert sg.sg_last_kernel() == FFMA
+        want, S = ref.matmul(a[:, :K], b[:, :N])
+        assert_within_bound(Cbig[:, :N], want, S, "ragged extents, padded pitches")
+        assert torch.all(torch.isnan(Cbig[:, N:]))
+
+
 def test_degenerate_sizes():
     A = torch.ones(8, 0, device="cuda", dtype=torch.bfloat16)
     B = torch.ones(0, 8, device="cuda", dtype=torch.bfloat16)
