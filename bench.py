@@ -46,7 +46,7 @@ NCU_TRAFFIC_BYTES = 25.5e6   # profiles/bench_sweep_launch_list.md: average over
 # tf32 : bf16 dense tensor throughput (nominal 1.1 : 2.25 PFLOP/s; the issue rate measured on
 # this chip is exactly half)
 TF32_OVER_BF16 = 0.5
-BW_ROWS, BW_COLS = 8192, 12288   # shape of the memory-bound 2-D kernels' rows in the per-op table
+BW_ROWS, BW_COLS = 16384, 12288   # shape of the memory-bound 2-D kernels' rows in the per-op table (805 MB of f32)
 
 
 def load_peaks():
@@ -191,7 +191,7 @@ def op_specs(sg, seed):
     bw_cache = {}
 
     def bw_source(dtype):
-        # one seeded 8192 x 12288 tensor per dtype (403 / 201 MB, larger than L2); rotating sets are device copies
+        # one seeded tensor per dtype, several times the size of L2; rotating sets are device copies
         if dtype not in bw_cache:
             bw_cache[dtype] = gpu_operand((BW_ROWS, BW_COLS), seed, 170, "uniform", dtype)
         return bw_cache[dtype]

@@ -29,8 +29,6 @@
 namespace sg {
 namespace {
 
-__device__ __forceinline__ void named_sync_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
 // Bounded, flag-free wait used only while winding down after a time-out: lets copies that are
 // still in flight land before the CTA gives its shared memory back.
 __device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
@@ -39,9 +37,26 @@ __device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
 }
 
 // ------------------------------------------------------------------------------ Copy2D (TMA)
-constexpr int CP_STAGES = 6;
-constexpr int CP_STORES_IN_FLIGHT = 2;
-constexpr int CP_STAGE_BYTES = 32768;
+#ifndef SG_CP_STAGES
+#define SG_CP_STAGES 6
+#endif
+#ifndef SG_CP_STORES_IN_FLIGHT
+#define SG_CP_STORES_IN_FLIGHT 2
+#endif
+#ifndef SG_CP_STAGE_BYTES
+#define SG_CP_STAGE_BYTES 32768
+#endif
+#ifndef SG_CP_CTAS_PER_SM
+#define SG_CP_CTAS_PER_SM 1
+#endif
+#ifndef SG_CP_BOX_X
+#define SG_CP_BOX_X 256
+#endif
+constexpr int CP_STAGES = SG_CP_STAGES;                         // ring depth
+constexpr int CP_STORES_IN_FLIGHT = SG_CP_STORES_IN_FLIGHT;     // stores whose shared-memory reads may be pending
+constexpr int CP_STAGE_BYTES = SG_CP_STAGE_BYTES;
+constexpr int CP_CTAS_PER_SM = SG_CP_CTAS_PER_SM;
+static_assert(CP_STAGES > CP_STORES_IN_FLIGHT + 1, "the ring must leave room for loads");
 
 // Tiles are dealt round-robin to the CTAs; warp 0 loads, warp 1 stores, one lane each.
 __global__ void __launch_bounds__(64) copy_tma_kernel(const __grid_constant__ CUtensorMap map_src,
@@ -93,7 +108,11 @@ __global__ void __launch_bounds__(64) copy_tma_kernel(const __grid_constant__ CU
 // One tile = 128 input rows x 128 bytes (W = 128/ES columns).  Input stage: the tile as TMA wrote
 // it with the 128-byte swizzle (16-byte chunk index XOR row mod 8).  Output staging: the W x 128
 // transposed tile as 128/W blocks of [W rows][128 bytes], same swizzle, stored by four tensor
-// stores of 32 rows each (one per transposer warp).
+// stores of 32 rows each (one per transposer warp, which also produces exactly those rows).
+#ifndef SG_TR_PANEL
+#define SG_TR_PANEL 8
+#endif
+constexpr int TR_PANEL = SG_TR_PANEL;     // tile columns per panel of the tile order
 constexpr int TR_IN_STAGES = 4;
 constexpr int TR_TILE_BYTES = 16384;
 constexpr int TR_THREADS = 32 + 128;
@@ -120,10 +139,22 @@ __device__ __forceinline__ void transpose_block(const uint4 (&v)[16 / ES], uint4
     }
 }
 
+// Tile order: panels of `panel` tile columns, walked row by row inside a panel.  The tiles in flight at one time then
+// cover a block of the matrix rather than a thin strip of it, so that both the reads (128 bytes per row and tile) and the
+// writes (128 input rows = one run of an output row per tile) fall on runs of memory that neighbouring tiles extend.
+__device__ __forceinline__ void tile_coords(int t, int tiles_c, int tiles_r, int panel, int &tr, int &tc) {
+    const int per_panel = panel * tiles_r;
+    const int pi = t / per_panel, within = t - pi * per_panel;
+    const int start = pi * panel, width = min(panel, tiles_c - start);
+    tr = within / width;
+    tc = start + within - tr * width;
+}
+
 template <int ES>
 __global__ void __launch_bounds__(TR_THREADS) transpose_tma_kernel(const __grid_constant__ CUtensorMap map_src,
                                                                     const __grid_constant__ CUtensorMap map_dst, int tiles_c,
-                                                                    int num_tiles, int dst_cols, int dst_rows) {
+                                                                    int tiles_r, int panel, int dst_cols, int dst_rows) {
+    const int num_tiles = tiles_c * tiles_r;
     constexpr int E = 16 / ES;       // elements per 16-byte chunk = side of the register block
     constexpr int W = 128 / ES;      // input columns per tile = output rows per tile
     constexpr int P = 128 / E;       // row groups per tile
@@ -148,32 +179,38 @@ __global__ void __launch_bounds__(TR_THREADS) transpose_tma_kernel(const __grid_
                 const uint32_t ph = (uint32_t)(k / TR_IN_STAGES) & 1u;
                 if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, &abort_load)) break;
                 mbar_expect_tx(smem_u32(&full_bar[s]), TR_TILE_BYTES);
-                tma_load_2d(in_ring + (uint32_t)s * TR_TILE_BYTES, &map_src, smem_u32(&full_bar[s]), (t % tiles_c) * W, (t / tiles_c) * 128);
+                int tr, tc;
+                tile_coords(t, tiles_c, tiles_r, panel, tr, tc);
+                tma_load_2d(in_ring + (uint32_t)s * TR_TILE_BYTES, &map_src, smem_u32(&full_bar[s]), tc * W, tr * 128);
             }
             if (abort_load)
                 for (int j = (k > TR_IN_STAGES ? k - TR_IN_STAGES : 0); j < k; ++j)
                     mbar_drain(smem_u32(&full_bar[j % TR_IN_STAGES]), (uint32_t)(j / TR_IN_STAGES) & 1u);
         }
     } else {
+        // Warp w owns store w of every tile: the 32 output rows x 128 bytes that sit at staging offset w * 4 KB.  What it
+        // reads for them (f32: input rows 32w .. 32w+31, all 32 columns; 2-byte elements: rows 64(w/2) .. +63, columns
+        // 32(w%2) .. +31) nobody else reads, so the four warps never wait for one another.
         const int w = warp - 1;
-        if (w == 0 && lane == 0) prefetch_tensormap(&map_dst);
-        // lanes of a quarter-warp take two row groups x four chunks: conflict-free 16-byte reads
-        const int q_lo = (lane & 3) | ((lane >> 1) & 4);
-        const int p_lo = ((lane >> 2) & 1) | ((lane >> 3) & 2);
+        if (lane == 0) prefetch_tensormap(&map_dst);
+        // each lane turns E x E blocks (row group p, 16-byte chunk q); a quarter-warp covers two row groups x four chunks
+        const int q = ES == 4 ? ((lane & 3) | ((lane >> 1) & 4)) : (4 * (w & 1) + (lane & 3));
+        const int p0 = ES == 4 ? (8 * w + ((lane >> 2) & 1) + 2 * ((lane >> 4) & 1)) : (8 * (w >> 1) + (lane >> 2));
+        constexpr int BLOCKS_PER_LANE = ES == 4 ? 2 : 1;
+        const int b = w / (W / 32), h = w % (W / 32);
         int k = 0;
         for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++k) {
             const int s = k % TR_IN_STAGES;
             const uint32_t ph = (uint32_t)(k / TR_IN_STAGES) & 1u;
-            mbar_wait(smem_u32(&full_bar[s]), ph, &abort_turn);       // a time-out sets abort_turn before the barrier below
+            const bool ok = mbar_wait(smem_u32(&full_bar[s]), ph, &abort_turn);
+            if (!__all_sync(0xffffffffu, ok)) break;
             if (lane == 0) bulk_wait_read<1>();                        // this warp's store from two tiles ago has read its staging
-            named_sync_128();
-            if (abort_turn) break;                                     // same answer in all 128 threads
+            __syncwarp();
             const uint32_t in_tile = in_ring + (uint32_t)s * TR_TILE_BYTES;
             const uint32_t out_tile = out_ring + (uint32_t)(k & 1) * TR_TILE_BYTES;
 #pragma unroll
-            for (int i = 0; i < P / 16; ++i) {
-                const int p = p_lo | (w << 2) | (i << 4);
-                const int q = q_lo;
+            for (int i = 0; i < BLOCKS_PER_LANE; ++i) {
+                const int p = p0 + 4 * i;
                 uint4 v[E], o[E];
 #pragma unroll
                 for (int kk = 0; kk < E; ++kk) {
@@ -190,14 +227,13 @@ __global__ void __launch_bounds__(TR_THREADS) transpose_tma_kernel(const __grid_
                     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(o[j].x), "r"(o[j].y), "r"(o[j].z), "r"(o[j].w) : "memory");
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&empty_bar[s]));       // the input stage may be refilled
             fence_async_smem();                                        // staging writes -> visible to the tensor store
-            named_sync_128();
+            __syncwarp();
             if (lane == 0) {
-                // store w: block w / (W/32) of the staging, rows (w % (W/32)) * 32 .. + 31; 4 KB each, back to back
-                const int b = w / (W / 32), h = w % (W / 32);
-                const int x = (t / tiles_c) * 128 + b * W, y = (t % tiles_c) * W + h * 32;
+                mbar_arrive(smem_u32(&empty_bar[s]));                  // this warp is done with the input stage
+                int tr, tc;
+                tile_coords(t, tiles_c, tiles_r, panel, tr, tc);
+                const int x = tr * 128 + b * W, y = tc * W + h * 32;
                 if (x < dst_cols && y < dst_rows) tma_store_2d(&map_dst, out_tile + (uint32_t)w * 4096u, x, y);
                 bulk_commit();
             }
@@ -249,28 +285,65 @@ __device__ __forceinline__ float widen(uint16_t bits) { return __uint_as_float((
 
 // Adds up to VEC consecutive elements starting at `ptr` (element stride `sc`) into acc.
 // `nvalid` == VEC takes the 16-byte path (VEC > 1 implies sc == 1 and an aligned address).
+// One whole chunk (VEC > 1: 16 bytes at an aligned address), added element-wise into acc.
+template <typename T, int VEC>
+__device__ __forceinline__ void accumulate_raw(float (&acc)[VEC], const uint4 &raw) {
+    if constexpr (VEC == 4) {
+        acc[0] += __uint_as_float(raw.x); acc[1] += __uint_as_float(raw.y);
+        acc[2] += __uint_as_float(raw.z); acc[3] += __uint_as_float(raw.w);
+    } else if constexpr (VEC == 8) {
+        const uint32_t wds[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            acc[2 * w] += __uint_as_float(wds[w] << 16);
+            acc[2 * w + 1] += __uint_as_float(wds[w] & 0xFFFF0000u);
+        }
+    }
+}
+
 template <typename T, int VEC>
 __device__ __forceinline__ void add_chunk(float (&acc)[VEC], const T *ptr, int64_t sc, int nvalid) {
     if constexpr (VEC > 1) {
         if (nvalid == VEC) {
-            const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(ptr));
-            if constexpr (sizeof(T) == 4) {
-                acc[0] += __uint_as_float(raw.x); acc[1] += __uint_as_float(raw.y);
-                acc[2] += __uint_as_float(raw.z); acc[3] += __uint_as_float(raw.w);
-            } else {
-                const uint32_t wds[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    acc[2 * w] += __uint_as_float(wds[w] << 16);
-                    acc[2 * w + 1] += __uint_as_float(wds[w] & 0xFFFF0000u);
-                }
-            }
+            accumulate_raw<T, VEC>(acc, __ldg(reinterpret_cast<const uint4 *>(ptr)));
             return;
         }
     }
 #pragma unroll
     for (int v = 0; v < VEC; ++v)
         if (v < nvalid) acc[v] += widen(__ldg(ptr + (int64_t)v * sc));
+}
+
+// Rows r, r+rp, ... < r1 of one chunk, eight loads in flight.  FULL: the chunk has all VEC columns (16-byte loads).
+template <typename T, int VEC, bool FULL>
+__device__ __forceinline__ void colred_walk(float (&acc)[VEC], const T *base, int64_t ld, int64_t sc, int64_t r, int64_t r1, int rp,
+                                            int nvalid) {
+    constexpr int U = 8;
+    if constexpr (FULL && VEC > 1) {
+        // all eight 16-byte loads are issued before the first is consumed
+        for (; r + (U - 1) * rp < r1; r += U * rp) {
+            uint4 raw[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) raw[u] = __ldg(reinterpret_cast<const uint4 *>(base + (r + u * rp) * ld));
+#pragma unroll
+            for (int u = 0; u < U; ++u) accumulate_raw<T, VEC>(acc, raw[u]);
+        }
+    } else {
+        for (; r + (U - 1) * rp < r1; r += U * rp) {
+            float part[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) part[u] = 0.f;
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) {
+                if (v < nvalid) {
+#pragma unroll
+                    for (int u = 0; u < U; ++u) part[u] = widen(__ldg(base + (r + u * rp) * ld + (int64_t)v * sc));
+                    acc[v] += ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
+                }
+            }
+        }
+    }
+    for (; r < r1; r += rp) add_chunk<T, VEC>(acc, base + r * ld, sc, FULL ? VEC : nvalid);
 }
 
 // ColRed2D.  A CTA owns `cw` chunks of VEC columns and the rows [r0, r1) of its split;
@@ -291,19 +364,8 @@ __global__ void __launch_bounds__(256) colred_kernel(const T *__restrict__ A, in
     const int nvalid = active ? (int)min((int64_t)VEC, (int64_t)C - col0) : 0;
     if (active) {
         const T *base = A + col0 * sc;
-        int64_t r = r0 + g;
-        for (; r + 3 * rp < r1; r += 4 * rp) {
-            float a0[VEC], a1[VEC], a2[VEC], a3[VEC];
-#pragma unroll
-            for (int v = 0; v < VEC; ++v) a0[v] = a1[v] = a2[v] = a3[v] = 0.f;
-            add_chunk<T, VEC>(a0, base + r * ld, sc, nvalid);
-            add_chunk<T, VEC>(a1, base + (r + rp) * ld, sc, nvalid);
-            add_chunk<T, VEC>(a2, base + (r + 2 * rp) * ld, sc, nvalid);
-            add_chunk<T, VEC>(a3, base + (r + 3 * rp) * ld, sc, nvalid);
-#pragma unroll
-            for (int v = 0; v < VEC; ++v) acc[v] += (a0[v] + a1[v]) + (a2[v] + a3[v]);
-        }
-        for (; r < r1; r += rp) add_chunk<T, VEC>(acc, base + r * ld, sc, nvalid);
+        if (nvalid == VEC) colred_walk<T, VEC, true>(acc, base, ld, sc, r0 + g, r1, rp, VEC);
+        else colred_walk<T, VEC, false>(acc, base, ld, sc, r0 + g, r1, rp, nvalid);
     }
 #pragma unroll
     for (int v = 0; v < VEC; ++v) red[t][v] = acc[v];
@@ -343,16 +405,21 @@ __global__ void __launch_bounds__(256) rowred_kernel(const T *__restrict__ A, in
         const int full_end = c0 + (c1 - c0) / VEC * VEC;      // whole chunks
         int64_t c = c0 + sub * VEC;
         const int64_t step = lanes * VEC;
-        for (; c + 3 * step < full_end; c += 4 * step) {
-            float a0[VEC], a1[VEC], a2[VEC], a3[VEC];
+        if constexpr (VEC > 1) {
+            for (; c + 7 * step < full_end; c += 8 * step) {      // eight 16-byte loads in flight
+                uint4 raw[8];
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) a0[v] = a1[v] = a2[v] = a3[v] = 0.f;
-            add_chunk<T, VEC>(a0, base + c * sc, sc, VEC);
-            add_chunk<T, VEC>(a1, base + (c + step) * sc, sc, VEC);
-            add_chunk<T, VEC>(a2, base + (c + 2 * step) * sc, sc, VEC);
-            add_chunk<T, VEC>(a3, base + (c + 3 * step) * sc, sc, VEC);
+                for (int u = 0; u < 8; ++u) raw[u] = __ldg(reinterpret_cast<const uint4 *>(base + c + u * step));
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) acc[v] += (a0[v] + a1[v]) + (a2[v] + a3[v]);
+                for (int u = 0; u < 8; ++u) accumulate_raw<T, VEC>(acc, raw[u]);
+            }
+        } else {
+            for (; c + 7 * step < full_end; c += 8 * step) {
+                float part[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) part[u] = widen(__ldg(base + (c + u * step) * sc));
+                acc[0] += ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
+            }
         }
         for (; c < full_end; c += step) add_chunk<T, VEC>(acc, base + c * sc, sc, VEC);
         if (VEC > 1 && sub == 0 && full_end < c1) {            // the ragged end of the range, element by element
@@ -409,10 +476,18 @@ cudaError_t launch_reduce_typed(bool colred, const T *A, int64_t ld, int64_t sc,
         const int cw = (int)std::min<int64_t>(chunks, 256);
         const int rp = 256 / cw;
         const int64_t col_blocks = (chunks + cw - 1) / cw;
+        // row ranges: as many as give every SM its full set of resident thread blocks, in one wave
+        static int resident = 0;
+        if (resident == 0) {
+            int n = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, colred_kernel<T, VEC>, 256, 0) != cudaSuccess || n < 1) n = 2;
+            resident = n;
+        }
         int splits = 1;
         const int min_rows_per_split = rp * 16;
-        if (col_blocks < target_ctas && R > min_rows_per_split)
-            splits = (int)std::min<int64_t>((target_ctas + col_blocks - 1) / col_blocks, ((int64_t)R + min_rows_per_split - 1) / min_rows_per_split);
+        const int64_t wave = (int64_t)num_sms * resident;
+        if (col_blocks < wave && R > min_rows_per_split)
+            splits = (int)std::min<int64_t>(wave / col_blocks, ((int64_t)R + min_rows_per_split - 1) / min_rows_per_split);
         int rows_per_split = (R + splits - 1) / splits;
         rows_per_split = (rows_per_split + rp - 1) / rp * rp;
         splits = (R + rows_per_split - 1) / rows_per_split;
@@ -467,7 +542,7 @@ sg_status launch_move2d(bool transpose, int64_t R, int64_t C, const void *src, i
         cuuint64_t st_src[1] = {(cuuint64_t)(s_r * esize)}, st_dst[1] = {(cuuint64_t)(d_r * esize)};
         if (!transpose) {
             // box: up to 256 elements wide, as many rows as fit a 32 KB stage
-            const int box_x = (int)std::min<int64_t>(256, Cb);
+            const int box_x = (int)std::min<int64_t>(SG_CP_BOX_X, Cb);
             const int box_y = (int)std::min<int64_t>(std::min<int64_t>(256, CP_STAGE_BYTES / (box_x * esize)), Rb);
             cuuint64_t dims[2] = {(cuuint64_t)Cb, (cuuint64_t)Rb};
             cuuint32_t box[2] = {(cuuint32_t)box_x, (cuuint32_t)box_y};
@@ -483,7 +558,7 @@ sg_status launch_move2d(bool transpose, int64_t R, int64_t C, const void *src, i
                     g_attr_copy = true;
                 }
                 const int num_tiles = (int)(tiles_x * tiles_y);
-                copy_tma_kernel<<<std::min(num_tiles, num_sms), 64, smem, stream>>>(map_src, map_dst, (int)tiles_x, num_tiles, box_x, box_y,
+                copy_tma_kernel<<<std::min(num_tiles, CP_CTAS_PER_SM * num_sms), 64, smem, stream>>>(map_src, map_dst, (int)tiles_x, num_tiles, box_x, box_y,
                                                                                     (uint32_t)(box_x * box_y * esize));
                 launched = true;
             }
@@ -508,8 +583,9 @@ sg_status launch_move2d(bool transpose, int64_t R, int64_t C, const void *src, i
                 }
                 const int num_tiles = (int)(tiles_c * tiles_r);
                 const int grid = std::min(num_tiles, 2 * num_sms);
-                if (esize == 4) transpose_tma_kernel<4><<<grid, TR_THREADS, smem, stream>>>(map_src, map_dst, (int)tiles_c, num_tiles, (int)Rb, (int)Cb);
-                else transpose_tma_kernel<2><<<grid, TR_THREADS, smem, stream>>>(map_src, map_dst, (int)tiles_c, num_tiles, (int)Rb, (int)Cb);
+                const int panel = (int)std::min<int64_t>(tiles_c, TR_PANEL);
+                if (esize == 4) transpose_tma_kernel<4><<<grid, TR_THREADS, smem, stream>>>(map_src, map_dst, (int)tiles_c, (int)tiles_r, panel, (int)Rb, (int)Cb);
+                else transpose_tma_kernel<2><<<grid, TR_THREADS, smem, stream>>>(map_src, map_dst, (int)tiles_c, (int)tiles_r, panel, (int)Rb, (int)Cb);
                 launched = true;
             }
         }
