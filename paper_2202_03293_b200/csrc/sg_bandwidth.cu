@@ -275,6 +275,8 @@ __global__ void __launch_bounds__(256) tile_move_kernel(const U *__restrict__ sr
 }
 
 // --------------------------------------------------------------------------------- reductions
+inline bool aligned16(const void *p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
+
 template <typename T, int VEC>
 struct Chunk {
     float f[VEC];
@@ -374,6 +376,14 @@ __global__ void __launch_bounds__(256) colred_kernel(const T *__restrict__ A, in
         for (int gg = 1; gg < rp; ++gg)
 #pragma unroll
             for (int v = 0; v < VEC; ++v) acc[v] += red[gg * cw + cc][v];
+        if (VEC >= 4 && use_atomic == 2 && nvalid == VEC) {
+            // dense, 16-byte aligned output: four sums per atomic
+#pragma unroll
+            for (int v = 0; v < VEC; v += 4)
+                asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(out + col0 + v), "f"(acc[v]), "f"(acc[(v + 1) % VEC]),
+                             "f"(acc[(v + 2) % VEC]), "f"(acc[(v + 3) % VEC]) : "memory");
+            return;
+        }
 #pragma unroll
         for (int v = 0; v < VEC; ++v) {
             if (v < nvalid) {
@@ -443,8 +453,6 @@ __global__ void zero_vector_kernel(float *__restrict__ out, int64_t n, int64_t o
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) out[i * os] = 0.f;
 }
 
-inline bool aligned16(const void *p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
-
 template <typename T, int VEC>
 cudaError_t launch_reduce_typed(bool colred, const T *A, int64_t ld, int64_t sc, int R, int C, float *out, int64_t os,
                                 int accumulate, int num_sms, cudaStream_t stream) {
@@ -491,7 +499,8 @@ cudaError_t launch_reduce_typed(bool colred, const T *A, int64_t ld, int64_t sc,
         int rows_per_split = (R + splits - 1) / splits;
         rows_per_split = (rows_per_split + rp - 1) / rp * rp;
         splits = (R + rows_per_split - 1) / rows_per_split;
-        const int use_atomic = splits > 1;
+        // 2: the output is dense and 16-byte aligned, so whole chunks may use vector atomics
+        const int use_atomic = splits > 1 ? ((os == 1 && aligned16(out)) ? 2 : 1) : 0;
         if (use_atomic && !accumulate) {
             zero_vector_kernel<<<(int)std::min<int64_t>(((int64_t)C + 255) / 256, 1184), 256, 0, stream>>>(out, C, os);
             count_launch();
