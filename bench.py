@@ -159,7 +159,7 @@ def time_graph(calls, reps, warmup=3):
     return e0.elapsed_time(e1) / reps / len(calls)
 
 
-def op_specs(sg, seed):
+def op_specs(sg, seed, bw_rows=None):
     """The other configured ops: name -> (label, flops, compulsory bytes, dtype, make(set) -> buffers, call)."""
     import torch
 
@@ -193,13 +193,13 @@ def op_specs(sg, seed):
     def bw_source(dtype):
         # one seeded tensor per dtype, several times the size of L2; rotating sets are device copies
         if dtype not in bw_cache:
-            bw_cache[dtype] = gpu_operand((BW_ROWS, BW_COLS), seed, 170, "uniform", dtype)
+            bw_cache[dtype] = gpu_operand((bw_rows or BW_ROWS, BW_COLS), seed, 170, "uniform", dtype)
         return bw_cache[dtype]
 
     def bw(kind, dtype):
         # the memory-bound 2-D kernels (Section 4.4); bytes = every input element read once, every output written once
         es = 2 if dtype == "bf16" else 4
-        R, C = BW_ROWS, BW_COLS
+        R, C = bw_rows or BW_ROWS, BW_COLS
         tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
         if kind == "copy2d":
             return (f"Copy2D {R}x{C} {dtype}", 0.0, 2 * R * C * es, dtype,
@@ -385,6 +385,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--streams", type=int, default=4, help="parallel branches of the step's CUDA graphs")
     ap.add_argument("--op", default=None, help="time only this op of the per-op table (used for profiler captures)")
+    ap.add_argument("--bw-rows", type=int, default=None,
+                    help="with --op: rows of the memory-bound 2-D kernels' tensor (a smaller case for profiler captures)")
     ap.add_argument("--sweep-table", default=None, help="also time every shape of the sweep on its own and write the table to this JSON file")
     args = ap.parse_args()
 
@@ -413,7 +415,7 @@ def main():
     warmup = max(args.warmup, 3)
 
     if args.op is not None:
-        specs = op_specs(sg, seed)
+        specs = op_specs(sg, seed, args.bw_rows)
         if args.op not in specs:
             raise SystemExit(f"--op must be one of {sorted(specs)}")
         print(json.dumps(measure_op(sg, peaks, specs[args.op], reps=max(1, min(args.steps, 5)))), flush=True)
