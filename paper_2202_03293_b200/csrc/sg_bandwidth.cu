@@ -208,23 +208,44 @@ __global__ void __launch_bounds__(TR_THREADS) transpose_tma_kernel(const __grid_
             __syncwarp();
             const uint32_t in_tile = in_ring + (uint32_t)s * TR_TILE_BYTES;
             const uint32_t out_tile = out_ring + (uint32_t)(k & 1) * TR_TILE_BYTES;
+            if constexpr (ES == 2) {
+                // 2-byte elements: the matrix load/store instructions do the turn.  Instruction i handles input rows
+                // 8p .. 8p+7 (p = 8b + i) of the warp's four chunks: ldmatrix.trans hands every lane two consecutive
+                // elements of a transposed 8 x 8 block per chunk, stmatrix writes those blocks as 16-byte rows.  In both,
+                // the eight row addresses of a block fall on eight different swizzled chunks: no bank conflicts.
+                const int m = lane >> 3, rr = lane & 7;           // this lane addresses row rr of block m
+                const int qm = 4 * h + m;                         // chunk of block m
+                const int c = 8 * qm + rr;                        // output row this lane addresses
 #pragma unroll
-            for (int i = 0; i < BLOCKS_PER_LANE; ++i) {
-                const int p = p0 + 4 * i;
-                uint4 v[E], o[E];
-#pragma unroll
-                for (int kk = 0; kk < E; ++kk) {
-                    const int row = E * p + kk;
-                    const uint32_t addr = in_tile + (uint32_t)row * 128u + (uint32_t)((q ^ (row & 7)) << 4);
-                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v[kk].x), "=r"(v[kk].y), "=r"(v[kk].z), "=r"(v[kk].w) : "r"(addr));
+                for (int i = 0; i < 8; ++i) {
+                    const int row = 8 * (8 * b + i) + rr;
+                    const uint32_t src_addr = in_tile + (uint32_t)row * 128u + (uint32_t)((qm ^ rr) << 4);
+                    uint32_t r0, r1, r2, r3;
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(src_addr));
+                    const uint32_t dst_addr = out_tile + (uint32_t)b * (uint32_t)(W * 128) + (uint32_t)c * 128u + (uint32_t)((i ^ (c & 7)) << 4);
+                    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};"
+                                 ::"r"(dst_addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
                 }
-                transpose_block<ES>(v, o);
+            } else {
 #pragma unroll
-                for (int j = 0; j < E; ++j) {
-                    const int c = E * q + j;                       // output row within the tile
-                    const uint32_t addr = out_tile + (uint32_t)(p >> 3) * (uint32_t)(W * 128) + (uint32_t)c * 128u +
-                                          (uint32_t)(((p & 7) ^ (c & 7)) << 4);
-                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(o[j].x), "r"(o[j].y), "r"(o[j].z), "r"(o[j].w) : "memory");
+                for (int i = 0; i < BLOCKS_PER_LANE; ++i) {
+                    const int p = p0 + 4 * i;
+                    uint4 v[E], o[E];
+#pragma unroll
+                    for (int kk = 0; kk < E; ++kk) {
+                        const int row = E * p + kk;
+                        const uint32_t addr = in_tile + (uint32_t)row * 128u + (uint32_t)((q ^ (row & 7)) << 4);
+                        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v[kk].x), "=r"(v[kk].y), "=r"(v[kk].z), "=r"(v[kk].w) : "r"(addr));
+                    }
+                    transpose_block<ES>(v, o);
+#pragma unroll
+                    for (int j = 0; j < E; ++j) {
+                        const int c = E * q + j;                       // output row within the tile
+                        const uint32_t addr = out_tile + (uint32_t)(p >> 3) * (uint32_t)(W * 128) + (uint32_t)c * 128u +
+                                              (uint32_t)(((p & 7) ^ (c & 7)) << 4);
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(o[j].x), "r"(o[j].y), "r"(o[j].z), "r"(o[j].w) : "memory");
+                    }
                 }
             }
             fence_async_smem();                                        // staging writes -> visible to the tensor store
