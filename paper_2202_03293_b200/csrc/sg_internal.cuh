@@ -68,6 +68,7 @@ struct DepthwiseProblem {
     int in_bf16, accumulate;
 };
 cudaError_t launch_depthwise(const DepthwiseProblem &p, const void *I, const void *Kf, float *O, cudaStream_t stream);
+sg_status depthwise_read_status(cudaStream_t stream);
 
 // The memory-bound 2-D kernels (Section 4.4).  launch_move2d: dst[i,j] = src[i,j], or dst[j,i] = src[i,j] when
 // `transpose`; elements of `esize` (2 or 4) bytes, strides in elements; `force` 0 picks, 1 = strided kernel only, 2 = TMA

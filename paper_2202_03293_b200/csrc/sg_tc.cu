@@ -980,7 +980,8 @@ sg_status tensor_read_status(cudaStream_t stream) {
     const sg_status a = read_status_word(stream);
     const sg_status b = conv_read_status(stream);
     const sg_status c = bandwidth_read_status(stream);
-    return a != SG_OK ? a : (b != SG_OK ? b : c);
+    const sg_status d = depthwise_read_status(stream);
+    return a != SG_OK ? a : (b != SG_OK ? b : (c != SG_OK ? c : d));
 }
 
 bool tensor_driver_ready(int *num_sms) {

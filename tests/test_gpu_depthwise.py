@@ -102,3 +102,34 @@ def test_depthwise_closed_forms_exactness_and_rejections():
     sg.sg_depthwise_conv2d_nhwc_hwc(torch.zeros(1, 4, 4, 8, device="cuda"), torch.zeros(0, 3, 8, device="cuda"), E)
     torch.cuda.synchronize()
     assert torch.all(E == 0.0)
+
+
+# 3 x 3, unit strides, enough tiles to fill the GPU: the kernels that stage whole input tiles (TMA) or walk down the rows
+# with a rolling register window.  Ragged tile edges in h, w and the channel blocks, batch 1 and batched, 32- and
+# 64-channel blocks, integer data (exact), accumulate mode.
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("N,Ho,Wo,C", [(8, 56, 56, 64), (5, 37, 45, 96), (16, 30, 70, 32), (1, 200, 210, 128), (3, 61, 33, 200),
+                                       (2, 100, 100, 40), (16, 200, 203, 16)])
+def test_depthwise_conv2d_tiled_kernels(dtype, N, Ho, Wo, C):
+    O, want, S = run2d(N, Ho, Wo, C, 3, 3, (1, 1), (1, 1), dtype)
+    assert_within_bound(O, want, S, "depthwise conv2d, tiled")
+    O, want, S = run2d(N, Ho, Wo, C, 3, 3, (1, 1), (1, 1), dtype, dist="ints")
+    assert np.array_equal(O.cpu().numpy().astype(np.float64), want)
+    O, want, S = run2d(N, Ho, Wo, C, 3, 3, (1, 1), (1, 1), dtype, accumulate=True, extra=(1, 2))
+    assert_within_bound(O, want, S, "depthwise conv2d, tiled, accumulate")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_depthwise_conv2d_tiled_channel_slice(dtype):
+    # a 64-channel slice of an 80-channel tensor (pixel pitch != C) into a slice of a wider output; NaN around the slice
+    # of the output must survive, and the channels outside the input slice must not leak in
+    N, Ho, Wo, C = 6, 40, 48, 64
+    Ibig, i = operand((N, Ho + 2, Wo + 2, 80), SEED, 20, "normal", dtype)
+    K, k = operand((3, 3, C), SEED, 21, "normal", dtype)
+    Obig = torch.full((N, Ho, Wo, 72), float("nan"), device="cuda")
+    sg.sg_depthwise_conv2d_nhwc_hwc(Ibig[..., 8:72], K, Obig[..., 4:68])
+    torch.cuda.synchronize()
+    sg.sg_check()
+    want, S = ref.depthwise_conv2d_nhwc_hwc(np.ascontiguousarray(i[..., 8:72]), k)
+    assert_within_bound(Obig[..., 4:68], want, S, "channel slice, tiled")
+    assert torch.all(torch.isnan(Obig[..., :4])) and torch.all(torch.isnan(Obig[..., 68:]))
