@@ -217,14 +217,15 @@ depthwise_roll_kernel(const DepthwiseProblem p, const T *__restrict__ I, const T
 // walks down the DT_ROWS output rows of its column with the 3 x 3 window of float4 in registers (three new
 // shared-memory reads per output, conflict-free: a warp reads whole contiguous pixels) and stores its outputs
 // straight from registers (a warp writes whole pixels).  Warp 8 is the producer.
-constexpr int DT_ROWS = 8;
 constexpr int DT_THREADS = 256 + 32;
 
-template <typename T, int CB>
+// S: stride along h and w (1 or 2).  A tile is ROWS output rows x TWB output columns x CB channels.
+template <typename T, int CB, int S>
 struct DtCfg {
     static constexpr int CG = CB / 4;                 // channel groups (threads) per pixel
     static constexpr int TWB = 256 / CG;              // output columns per tile
-    static constexpr int IN_W = TWB + 2, IN_H = DT_ROWS + 2;
+    static constexpr int ROWS = S == 1 ? 8 : 2;       // output rows per tile
+    static constexpr int IN_W = (TWB - 1) * S + 3, IN_H = (ROWS - 1) * S + 3;
     static constexpr int PIXEL_BYTES = CB * (int)sizeof(T);
     static constexpr int BOX_BYTES = PIXEL_BYTES * IN_W * IN_H;
     static constexpr int STAGE_BYTES = (BOX_BYTES + 127) / 128 * 128;
@@ -241,11 +242,13 @@ __device__ __forceinline__ float4 lds4(uint32_t addr, __nv_bfloat16) {
     return make_float4(__uint_as_float(a << 16), __uint_as_float(a & 0xFFFF0000u), __uint_as_float(b << 16), __uint_as_float(b & 0xFFFF0000u));
 }
 
-template <typename T, int CB>
+// The grid is a multiple of c_blocks (or smaller than it never), so a CTA keeps one channel block
+// for all its tiles and a thread loads its nine filter values once.
+template <typename T, int CB, int S>
 __global__ void __launch_bounds__(DT_THREADS)
 depthwise_tma_kernel(const __grid_constant__ CUtensorMap map_in, const DepthwiseProblem p, const T *__restrict__ Kf,
                      float *__restrict__ O, int tiles_w, int tiles_h, int c_blocks, int num_tiles) {
-    using C = DtCfg<T, CB>;
+    using C = DtCfg<T, CB, S>;
     extern __shared__ uint8_t dt_smem[];
     __shared__ uint64_t full_bar[2], empty_bar[2];
     __shared__ int abort_load, abort_compute;
@@ -270,7 +273,7 @@ depthwise_tma_kernel(const __grid_constant__ CUtensorMap map_in, const Depthwise
                 const int wt = r % tiles_w; r /= tiles_w;
                 const int ht = r % tiles_h, n = r / tiles_h;
                 mbar_expect_tx(smem_u32(&full_bar[s]), C::BOX_BYTES);
-                tma_load_4d(ring + (uint32_t)s * C::STAGE_BYTES, &map_in, smem_u32(&full_bar[s]), cb * CB, wt * C::TWB, ht * DT_ROWS, n);
+                tma_load_4d(ring + (uint32_t)s * C::STAGE_BYTES, &map_in, smem_u32(&full_bar[s]), cb * CB, wt * C::TWB * S, ht * C::ROWS * S, n);
             }
             if (abort_load)      // gave up: let the loads already issued land before the shared memory goes away
                 for (int j = (k > 2 ? k - 2 : 0); j < k; ++j)
@@ -278,43 +281,45 @@ depthwise_tma_kernel(const __grid_constant__ CUtensorMap map_in, const Depthwise
         }
     } else {
         const int cg = threadIdx.x % C::CG, wl = threadIdx.x / C::CG;
+        const int c = (int)(blockIdx.x % c_blocks) * CB + cg * 4;      // the same for every tile of this CTA
+        float4 flt[3][3];
+#pragma unroll
+        for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+            for (int kw = 0; kw < 3; ++kw)
+                flt[kh][kw] = c < p.C ? load4(Kf + (int64_t)kh * p.k_kh + (int64_t)kw * p.k_kw + c) : make_float4(0.f, 0.f, 0.f, 0.f);
         int k = 0;
         for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++k) {
             const int s = k & 1;
             const uint32_t ph = (uint32_t)(k >> 1) & 1u;
-            int r = t;
-            const int cb = r % c_blocks; r /= c_blocks;
+            int r = t / c_blocks;
             const int wt = r % tiles_w; r /= tiles_w;
             const int ht = r % tiles_h, n = r / tiles_h;
-            const int c = cb * CB + cg * 4, w = wt * C::TWB + wl, h0 = ht * DT_ROWS;
+            const int w = wt * C::TWB + wl, h0 = ht * C::ROWS;
             const bool live = c < p.C && w < p.Wo;
-            float4 flt[3][3];
-#pragma unroll
-            for (int kh = 0; kh < 3; ++kh)
-#pragma unroll
-                for (int kw = 0; kw < 3; ++kw)
-                    flt[kh][kw] = live ? load4(Kf + (int64_t)kh * p.k_kh + (int64_t)kw * p.k_kw + c) : make_float4(0.f, 0.f, 0.f, 0.f);
             const bool ok = mbar_wait(smem_u32(&full_bar[s]), ph, &abort_compute);
             if (!__all_sync(0xffffffffu, ok)) break;
-            // this thread's column of the tile: pixel (row r, column wl + kw) of the stage
-            const uint32_t col_base = ring + (uint32_t)s * C::STAGE_BYTES + (uint32_t)(wl * CB + cg * 4) * (uint32_t)sizeof(T);
+            // this thread's columns of the tile: pixel (row r, column S*wl + kw) of the stage; tile row r lives in win[r % 3]
+            const uint32_t col_base = ring + (uint32_t)s * C::STAGE_BYTES + (uint32_t)(wl * S * CB + cg * 4) * (uint32_t)sizeof(T);
             float4 win[3][3];
 #pragma unroll
-            for (int rr = 0; rr < 2; ++rr)
+            for (int rr = 0; rr < 3 - S; ++rr)
 #pragma unroll
                 for (int kw = 0; kw < 3; ++kw) win[rr][kw] = lds4(col_base + (uint32_t)((rr * C::IN_W + kw) * C::PIXEL_BYTES), T());
             float *out = O + (int64_t)n * p.o_n + (int64_t)w * p.o_w + c;
 #pragma unroll
-            for (int hh = 0; hh < DT_ROWS; ++hh) {
-                // rows hh, hh+1 sit in win[hh % 3], win[(hh+1) % 3]; row hh+2 goes to win[(hh+2) % 3]
+            for (int hh = 0; hh < C::ROWS; ++hh) {
+                // the window of output row hh is tile rows S*hh .. S*hh+2; the first 3-S of them are already held
 #pragma unroll
-                for (int kw = 0; kw < 3; ++kw)
-                    win[(hh + 2) % 3][kw] = lds4(col_base + (uint32_t)(((hh + 2) * C::IN_W + kw) * C::PIXEL_BYTES), T());
+                for (int rr = S * hh + 3 - S; rr <= S * hh + 2; ++rr)
+#pragma unroll
+                    for (int kw = 0; kw < 3; ++kw)
+                        win[rr % 3][kw] = lds4(col_base + (uint32_t)((rr * C::IN_W + kw) * C::PIXEL_BYTES), T());
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                 for (int kh = 0; kh < 3; ++kh)
 #pragma unroll
-                    for (int kw = 0; kw < 3; ++kw) fma4(acc, win[(hh + kh) % 3][kw], flt[kh][kw]);
+                    for (int kw = 0; kw < 3; ++kw) fma4(acc, win[(S * hh + kh) % 3][kw], flt[kh][kw]);
                 if (live && h0 + hh < p.Ho) {
                     float4 *o = reinterpret_cast<float4 *>(out + (int64_t)(h0 + hh) * p.o_h);
                     if (p.accumulate) {
@@ -354,16 +359,17 @@ depthwise_generic_kernel(const DepthwiseProblem p, const T *__restrict__ I, cons
     }
 }
 
-template <typename T, int CB>
+template <typename T, int CB, int S>
 bool try_launch_tma(const DepthwiseProblem &p, const T *I, const T *Kf, float *O, int num_sms, cudaStream_t stream, cudaError_t *err) {
-    using C = DtCfg<T, CB>;
+    using C = DtCfg<T, CB, S>;
     const int64_t es = sizeof(T);
-    const int tiles_w = (p.Wo + C::TWB - 1) / C::TWB, tiles_h = (p.Ho + DT_ROWS - 1) / DT_ROWS, c_blocks = (p.C + CB - 1) / CB;
+    const int tiles_w = (p.Wo + C::TWB - 1) / C::TWB, tiles_h = (p.Ho + C::ROWS - 1) / C::ROWS, c_blocks = (p.C + CB - 1) / CB;
     const int64_t tiles = (int64_t)p.N * tiles_h * tiles_w * c_blocks;
-    if (tiles < num_sms || tiles >= ((int64_t)1 << 31)) return false;
-    // the part of the input that is read: (Ho+2) x (Wo+2) pixels per image
-    const int64_t s_n = p.N > 1 ? p.i_n : (int64_t)(p.Ho + 2) * p.i_h;
-    cuuint64_t dims[4] = {(cuuint64_t)p.C, (cuuint64_t)(p.Wo + 2), (cuuint64_t)(p.Ho + 2), (cuuint64_t)p.N};
+    if (tiles < num_sms || tiles >= ((int64_t)1 << 31) || c_blocks > num_sms) return false;
+    // the part of the input that is read: ((Ho-1)*S+3) x ((Wo-1)*S+3) pixels per image
+    const int64_t h_ext = (int64_t)(p.Ho - 1) * S + 3, w_ext = (int64_t)(p.Wo - 1) * S + 3;
+    const int64_t s_n = p.N > 1 ? p.i_n : h_ext * p.i_h;
+    cuuint64_t dims[4] = {(cuuint64_t)p.C, (cuuint64_t)w_ext, (cuuint64_t)h_ext, (cuuint64_t)p.N};
     cuuint64_t strides[3] = {(cuuint64_t)(p.i_w * es), (cuuint64_t)(p.i_h * es), (cuuint64_t)(s_n * es)};
     cuuint32_t box[4] = {(cuuint32_t)CB, (cuuint32_t)C::IN_W, (cuuint32_t)C::IN_H, 1};
     for (int i = 0; i < 3; ++i)
@@ -375,11 +381,13 @@ bool try_launch_tma(const DepthwiseProblem &p, const T *I, const T *Kf, float *O
     const int smem = 2 * C::STAGE_BYTES + 128;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(depthwise_tma_kernel<T, CB>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+        if (cudaFuncSetAttribute(depthwise_tma_kernel<T, CB, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
         attr_set = true;
     }
-    const int grid = (int)std::min<int64_t>(tiles, 2 * (int64_t)num_sms);
-    depthwise_tma_kernel<T, CB><<<grid, DT_THREADS, smem, stream>>>(map_in, p, Kf, O, tiles_w, tiles_h, c_blocks, (int)tiles);
+    // two CTAs per SM, rounded down to a multiple of the channel blocks: tile t has block t % c_blocks, so every CTA keeps one
+    int64_t grid = std::min<int64_t>(tiles, 2 * (int64_t)num_sms);
+    grid -= grid % c_blocks;
+    depthwise_tma_kernel<T, CB, S><<<(int)grid, DT_THREADS, smem, stream>>>(map_in, p, Kf, O, tiles_w, tiles_h, c_blocks, (int)tiles);
     count_launch();
     *err = cudaGetLastError();
     return true;
@@ -400,13 +408,16 @@ cudaError_t launch_typed(const DepthwiseProblem &p, const T *I, const T *Kf, flo
     const unsigned blocks = (unsigned)blocks64;
     const bool small = work < ((int64_t)1 << 32) - 256;
     const bool unit3 = p.sw == 1 && p.dw == 1 && p.KW == 3 && p.KH == 3;
-    if (vec && unit3 && p.sh == 1 && p.dh == 1 && reinterpret_cast<uintptr_t>(I) % 16 == 0 && (p.C * (int64_t)sizeof(T)) % 16 == 0) {
+    const bool win3 = p.KW == 3 && p.KH == 3 && p.dw == 1 && p.dh == 1;
+    if (vec && win3 && p.sh == p.sw && p.sh <= 2 && reinterpret_cast<uintptr_t>(I) % 16 == 0 &&
+        (p.C * (int64_t)sizeof(T)) % 16 == 0) {
         // TMA-staged tiles (TMA checks the channel bound in 16-byte units, hence the condition on C)
         int num_sms = 0;
         cudaError_t err = cudaSuccess;
-        if (tensor_driver_ready(&num_sms)) {
-            const bool done = p.C >= 64 ? try_launch_tma<T, 64>(p, I, Kf, O, num_sms, stream, &err)
-                                        : (p.C >= 32 ? try_launch_tma<T, 32>(p, I, Kf, O, num_sms, stream, &err) : false);
+        if (tensor_driver_ready(&num_sms) && p.C >= 32) {
+            bool done;
+            if (p.sh == 1) done = p.C >= 64 ? try_launch_tma<T, 64, 1>(p, I, Kf, O, num_sms, stream, &err) : try_launch_tma<T, 32, 1>(p, I, Kf, O, num_sms, stream, &err);
+            else done = p.C >= 64 ? try_launch_tma<T, 64, 2>(p, I, Kf, O, num_sms, stream, &err) : try_launch_tma<T, 32, 2>(p, I, Kf, O, num_sms, stream, &err);
             if (done) return err;
         }
     }

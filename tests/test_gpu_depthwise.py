@@ -108,14 +108,16 @@ def test_depthwise_closed_forms_exactness_and_rejections():
 # with a rolling register window.  Ragged tile edges in h, w and the channel blocks, batch 1 and batched, 32- and
 # 64-channel blocks, integer data (exact), accumulate mode.
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("stride", [1, 2])
 @pytest.mark.parametrize("N,Ho,Wo,C", [(8, 56, 56, 64), (5, 37, 45, 96), (16, 30, 70, 32), (1, 200, 210, 128), (3, 61, 33, 200),
                                        (2, 100, 100, 40), (16, 200, 203, 16)])
-def test_depthwise_conv2d_tiled_kernels(dtype, N, Ho, Wo, C):
-    O, want, S = run2d(N, Ho, Wo, C, 3, 3, (1, 1), (1, 1), dtype)
+def test_depthwise_conv2d_tiled_kernels(dtype, stride, N, Ho, Wo, C):
+    st = (stride, stride)
+    O, want, S = run2d(N, Ho, Wo, C, 3, 3, st, (1, 1), dtype)
     assert_within_bound(O, want, S, "depthwise conv2d, tiled")
-    O, want, S = run2d(N, Ho, Wo, C, 3, 3, (1, 1), (1, 1), dtype, dist="ints")
+    O, want, S = run2d(N, Ho, Wo, C, 3, 3, st, (1, 1), dtype, dist="ints")
     assert np.array_equal(O.cpu().numpy().astype(np.float64), want)
-    O, want, S = run2d(N, Ho, Wo, C, 3, 3, (1, 1), (1, 1), dtype, accumulate=True, extra=(1, 2))
+    O, want, S = run2d(N, Ho, Wo, C, 3, 3, st, (1, 1), dtype, accumulate=True, extra=(1, 2))
     assert_within_bound(O, want, S, "depthwise conv2d, tiled, accumulate")
 
 
