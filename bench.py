@@ -196,27 +196,32 @@ def op_specs(sg, seed, bw_rows=None):
             bw_cache[dtype] = gpu_operand((bw_rows or BW_ROWS, BW_COLS), seed, 170, "uniform", dtype)
         return bw_cache[dtype]
 
-    def bw(kind, dtype):
-        # the memory-bound 2-D kernels (Section 4.4); bytes = every input element read once, every output written once
+    def bw(kind, dtype, shape=None):
+        # the memory-bound 2-D kernels (Section 4.4); bytes = every input element read once, every output written once.
+        # shape None: the large tensor above; else a small seeded tensor of its own (the paper's cache-resident sizes)
         es = 2 if dtype == "bf16" else 4
-        R, C = bw_rows or BW_ROWS, BW_COLS
+        R, C = shape or (bw_rows or BW_ROWS, BW_COLS)
         tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+        src = (lambda s: gpu_operand((R, C), seed, 171 + s, "uniform", dtype)) if shape else (lambda s: bw_source(dtype).clone())
         if kind == "copy2d":
             return (f"Copy2D {R}x{C} {dtype}", 0.0, 2 * R * C * es, dtype,
-                    lambda s: (bw_source(dtype).clone(), torch.empty(R, C, device="cuda", dtype=tdt)), lambda a, o: sg.sg_copy2d(a, o))
+                    lambda s: (src(s), torch.empty(R, C, device="cuda", dtype=tdt)), lambda a, o: sg.sg_copy2d(a, o))
         if kind == "transpose2d":
             return (f"Transpose2D {R}x{C} {dtype}", 0.0, 2 * R * C * es, dtype,
-                    lambda s: (bw_source(dtype).clone(), torch.empty(C, R, device="cuda", dtype=tdt)), lambda a, o: sg.sg_transpose2d(a, o))
+                    lambda s: (src(s), torch.empty(C, R, device="cuda", dtype=tdt)), lambda a, o: sg.sg_transpose2d(a, o))
         n_out = C if kind == "colred2d" else R
         fn = sg.sg_colred2d if kind == "colred2d" else sg.sg_rowred2d
         return (f"{'ColRed2D' if kind == 'colred2d' else 'RowRed2D'} {R}x{C} {dtype}", float(R * C), R * C * es + n_out * 4, dtype,
-                lambda s: (bw_source(dtype).clone(), torch.empty(n_out, device="cuda")), lambda a, o: fn(a, o))
+                lambda s: (src(s), torch.empty(n_out, device="cuda")), lambda a, o: fn(a, o))
 
+    paper_shape = (250, 960)      # the one size the paper names for these kernels (caption of its L3 bandwidth figure)
     return {
         "copy2d_f32": bw("copy2d", "f32"), "copy2d_bf16": bw("copy2d", "bf16"),
         "transpose2d_f32": bw("transpose2d", "f32"), "transpose2d_bf16": bw("transpose2d", "bf16"),
         "colred2d_f32": bw("colred2d", "f32"), "rowred2d_f32": bw("rowred2d", "f32"),
         "colred2d_bf16": bw("colred2d", "bf16"), "rowred2d_bf16": bw("rowred2d", "bf16"),
+        "copy2d_250x960_f32": bw("copy2d", "f32", paper_shape), "transpose2d_250x960_f32": bw("transpose2d", "f32", paper_shape),
+        "colred2d_250x960_f32": bw("colred2d", "f32", paper_shape), "rowred2d_250x960_f32": bw("rowred2d", "f32", paper_shape),
         "depthwise_112_f32": dw(1, 112, 112, 32, 3, 3, 1, "f32", "depthwise conv2d 1x114x114x32 * 3x3x32 f32 (MobileNet-like, batch 1)"),
         "depthwise_batched_f32": dw(32, 112, 112, 64, 3, 3, 1, "f32", "depthwise conv2d 32x114x114x64 * 3x3x64 f32"),
         "depthwise_batched_bf16": dw(32, 112, 112, 64, 3, 3, 1, "bf16", "depthwise conv2d 32x114x114x64 * 3x3x64 bf16"),

@@ -1,14 +1,20 @@
 /*
  * sg.h: C ABI of the structured contraction library for NVIDIA B200 (sm_100a).
  *
- * Three ops, each defined by a rectangular iteration domain and one indexing
- * map per operand, evaluated on the GPU by hand-written CUDA kernels:
+ * Three contractions, each defined by a rectangular iteration domain and one
+ * indexing map per operand, evaluated on the GPU by hand-written CUDA kernels:
  *
  *   sg_matmul             C[m,n]     (+)= sum_k         A[m,k] * B[k,n]
  *   sg_conv1d_nwc_wcf     O[n,w,f]   (+)= sum_{kw,c}    I[n, w*sw + kw*dw, c] * K[kw,c,f]
  *   sg_conv2d_nhwc_hwcf   O[n,h,w,f] (+)= sum_{kh,kw,c} I[n, h*sh + kh*dh, w*sw + kw*dw, c] * K[kh,kw,c,f]
  *
- * Conventions common to all entry points
+ * and, declared further down, the memory-bound ops of the same paper: the
+ * depthwise convolutions (sg_depthwise_conv1d_nwc_wc, sg_depthwise_conv2d_nhwc_hwc)
+ * and the 2-D copy, transpose and row / column reductions (sg_copy2d,
+ * sg_transpose2d, sg_colred2d, sg_rowred2d).
+ *
+ * Conventions common to all entry points (the contraction-specific ones apply
+ * to the three ops above)
  *   - Every data pointer is a DEVICE pointer owned by the caller.  Inputs are
  *     read only; the output is written (SG_OVERWRITE) or read and written
  *     (SG_ACCUMULATE).  The output must not overlap an input.
