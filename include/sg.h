@@ -168,7 +168,8 @@ sg_status sg_depthwise_conv1d_nwc_wc(int64_t N, int64_t W_out, int64_t C, int64_
 /*
  * The memory-bound 2-D kernels (Section 4.4, "Benchmarks": Copy2D, Transpose2D, ColRed2D,
  * RowRed2D; measured in Section 4.5).  All operate on an R x C tensor whose element (i,j) is at
- * base[i*stride_r + j*stride_c] (strides in elements, any non-negative values).
+ * base[i*stride_r + j*stride_c] (strides in elements, any non-negative values); R and C up to
+ * 2^31 - 2^20 (SG_ERR_UNSUPPORTED beyond).
  *
  * Copy2D:       dst[i,j] = src[i,j]        dst is R x C
  * Transpose2D:  dst[j,i] = src[i,j]        dst is C x R; dst_stride_r is the pitch of ITS rows

@@ -14,6 +14,7 @@ thread_local int t_last_kernel = 0;
 constexpr int64_t kMaxDim = std::numeric_limits<int32_t>::max();
 
 inline bool fits(int64_t v) { return v >= 0 && v <= kMaxDim; }
+constexpr int64_t kTileSlack = 1 << 20;   // head room for extents rounded up to tiles or split ranges
 
 sg_status run(const Problem &p, const void *In, const void *Flt, float *O, cudaStream_t stream) {
     if (p.M == 0 || p.N == 0) return SG_OK;                       // nothing to write
@@ -203,7 +204,7 @@ sg_status move2d(bool transpose, int64_t R, int64_t C, const void *src, int64_t 
     using namespace sg;
     if (dtype != SG_F32 && dtype != SG_BF16) return SG_ERR_UNSUPPORTED;
     if (R < 0 || C < 0 || s_r < 0 || s_c < 0 || d_r < 0 || d_c < 0) return SG_ERR_INVALID_ARG;
-    if (!fits(R) || !fits(C)) return SG_ERR_UNSUPPORTED;
+    if (!fits(R + kTileSlack) || !fits(C + kTileSlack)) return SG_ERR_UNSUPPORTED;   // tile coordinates stay in int32
     if (R == 0 || C == 0) return SG_OK;
     if (!src || !dst) return SG_ERR_INVALID_ARG;
     const int es = dtype == SG_BF16 ? 2 : 4;
@@ -222,7 +223,7 @@ sg_status reduce2d(bool colred, int64_t R, int64_t C, const void *A, int64_t a_r
     sg_status st = check_common(A, nullptr, out, in_dtype, mode);
     if (st != SG_OK) return st;
     if (R < 0 || C < 0 || a_r < 0 || a_c < 0 || out_stride < 0) return SG_ERR_INVALID_ARG;
-    if (!fits(R) || !fits(C)) return SG_ERR_UNSUPPORTED;
+    if (!fits(R + kTileSlack) || !fits(C + kTileSlack)) return SG_ERR_UNSUPPORTED;   // rounded-up split ranges stay in int32
     const int64_t n_out = colred ? C : R, n_red = colred ? R : C;
     if (n_out == 0) return SG_OK;
     if (!out || (n_red > 0 && !A)) return SG_ERR_INVALID_ARG;
