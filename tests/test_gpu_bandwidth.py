@@ -200,11 +200,11 @@ def test_reductions_empty():
 
 
 def test_full_size_moves_sampled():
-    """The bench shapes (larger than L2): rows and columns sampled against the oracle."""
-    R, C = 8192, 12288
+    """The shape bench.py times (805 MB of f32, larger than L2): rows and columns sampled against the oracle."""
+    R, C = 16384, 12288
     bits = random_bits((R, C), 4, 20)
     src = to_dev(bits)
-    rows = np.array([0, 1, 127, 128, 4095, 8190, 8191])
+    rows = np.array([0, 1, 127, 128, 4095, 8190, 8191, 8192, 16383])
     cols = np.array([0, 31, 32, 6143, 12287])
     dst = torch.empty_like(src)
     sg.sg_copy2d(src, dst)
@@ -227,7 +227,7 @@ def test_full_size_moves_sampled():
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_full_size_reductions(dtype):
-    R, C = 8192, 12288
+    R, C = 16384, 12288        # the shape bench.py times
     A, a = operand((R, C), SEED, 21, "uniform", dtype)
     for op, fn, oracle, n_out in (("col", sg.sg_colred2d, ref.colred2d, C), ("row", sg.sg_rowred2d, ref.rowred2d, R)):
         out = torch.full((n_out,), float("nan"), device="cuda")

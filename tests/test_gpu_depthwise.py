@@ -110,7 +110,7 @@ def test_depthwise_closed_forms_exactness_and_rejections():
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("stride", [1, 2])
 @pytest.mark.parametrize("N,Ho,Wo,C", [(8, 56, 56, 64), (5, 37, 45, 96), (16, 30, 70, 32), (1, 200, 210, 128), (3, 61, 33, 200),
-                                       (2, 100, 100, 40), (16, 200, 203, 16)])
+                                       (2, 100, 100, 40), (16, 200, 203, 16), (32, 112, 112, 64)])   # the last: bench.py's layer
 def test_depthwise_conv2d_tiled_kernels(dtype, stride, N, Ho, Wo, C):
     st = (stride, stride)
     O, want, S = run2d(N, Ho, Wo, C, 3, 3, st, (1, 1), dtype)
