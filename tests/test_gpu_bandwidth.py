@@ -236,3 +236,24 @@ def test_full_size_reductions(dtype):
         sg.sg_check()
         want, S = oracle(a)
         assert assert_within_bound(out, want, S, f"{op}red full size {dtype}") < 1e-5
+
+
+def test_random_shapes_and_pitches():
+    """Seeded sweep over small shapes, pitches (aligned and not), dtypes and modes: every kernel path and every
+    hand-over between the TMA body and the strided tail gets hit many times."""
+    rng = np.random.default_rng(SEED)
+    for case in range(60):
+        R, C = int(rng.integers(1, 420)), int(rng.integers(1, 420))
+        esize = int(rng.choice([2, 4]))
+        op = str(rng.choice(["copy", "transpose"]))
+        dst_cols = R if op == "transpose" else C
+        aligned = bool(rng.integers(0, 2))
+        sp = (up8(C) + 8 * int(rng.integers(0, 3))) if aligned else C + int(rng.integers(0, 7))
+        dp = (up8(dst_cols) + 8 * int(rng.integers(0, 3))) if aligned else dst_cols + int(rng.integers(0, 7))
+        check_move(op, R, C, esize, sp, dp)
+    for case in range(60):
+        R, C = int(rng.integers(1, 700)), int(rng.integers(1, 700))
+        dtype = str(rng.choice(["f32", "bf16"]))
+        op = str(rng.choice(["col", "row"]))
+        pitch = up8(C) if rng.integers(0, 2) else C + int(rng.integers(0, 5))
+        run_reduce(op, R, C, dtype, accumulate=bool(rng.integers(0, 2)), pitch=pitch)
