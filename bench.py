@@ -524,13 +524,35 @@ def main():
         h2d = sum(a.numel() * a.element_size() + b.numel() * b.element_size() for a, b, _ in host.values())
         d2h = sum(c.numel() * 4 for _, _, c in host.values())
 
+        # The calls of a step are independent, so the user-side pipeline is three streams: inputs go up on one,
+        # sg_matmul runs on the current one, results come down on a third; events order each shape's copy-in ->
+        # matmul -> copy-out, and the next step's reuse of the same device buffers.
+        cur = torch.cuda.current_stream()
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        ev_in = {key: torch.cuda.Event() for key in bufs}
+        ev_mm = {key: torch.cuda.Event() for key in bufs}
+        ev_out = {key: torch.cuda.Event() for key in bufs}
+        e2e_order = [(dt, m, n, k) for dt in ("f32", "bf16") for (m, n, k) in order]
+
         def e2e_step():
-            for key, (a, b, c) in bufs.items():
+            for key in e2e_order:
+                a, b, c = bufs[key]
                 ah, bh, ch = host[key]
-                a.copy_(ah, non_blocking=True)
-                b.copy_(bh, non_blocking=True)
+                with torch.cuda.stream(s_in):
+                    s_in.wait_event(ev_mm[key])          # the previous step's matmul has read a and b
+                    a.copy_(ah, non_blocking=True)
+                    b.copy_(bh, non_blocking=True)
+                    ev_in[key].record(s_in)
+                cur.wait_event(ev_in[key])
+                cur.wait_event(ev_out[key])              # the previous step's copy-out has read c
                 sg.sg_matmul(a, b, c)
-                ch.copy_(c, non_blocking=True)
+                ev_mm[key].record(cur)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev_mm[key])
+                    ch.copy_(c, non_blocking=True)
+                    ev_out[key].record(s_out)
+            cur.wait_stream(s_in)
+            cur.wait_stream(s_out)                       # the step ends when its last result is on the host
 
         e2e_step()
         barrier()
