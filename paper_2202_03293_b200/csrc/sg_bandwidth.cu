@@ -546,7 +546,9 @@ cudaError_t launch_tile_move(const U *src, int64_t s_i, int64_t s_j, U *dst, int
     return cudaGetLastError();
 }
 
-bool g_attr_copy = false, g_attr_tr4 = false, g_attr_tr2 = false;
+// device on which each kernel's shared-memory limit was last raised (the attribute is per device)
+int g_attr_copy = -1, g_attr_tr4 = -1, g_attr_tr2 = -1;
+inline int current_device() { int d = 0; cudaGetDevice(&d); return d; }
 
 }  // namespace
 
@@ -583,9 +585,10 @@ sg_status launch_move2d(bool transpose, int64_t R, int64_t C, const void *src, i
                 tensor_encode_tiled(&map_dst, type, 2, dst, dims, st_dst, box, CU_TENSOR_MAP_SWIZZLE_NONE,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B)) {
                 const int smem = CP_STAGES * CP_STAGE_BYTES + 1024;
-                if (!g_attr_copy) {
+                const int dev = current_device();
+                if (g_attr_copy != dev) {
                     if (cudaFuncSetAttribute(copy_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SG_ERR_CUDA;
-                    g_attr_copy = true;
+                    g_attr_copy = dev;
                 }
                 const int num_tiles = (int)(tiles_x * tiles_y);
                 copy_tma_kernel<<<std::min(num_tiles, CP_CTAS_PER_SM * num_sms), 64, smem, stream>>>(map_src, map_dst, (int)tiles_x, num_tiles, box_x, box_y,
@@ -603,13 +606,14 @@ sg_status launch_move2d(bool transpose, int64_t R, int64_t C, const void *src, i
                 tensor_encode_tiled(&map_dst, type, 2, dst, dims_d, st_dst, box_d, CU_TENSOR_MAP_SWIZZLE_128B,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B)) {
                 const int smem = (TR_IN_STAGES + 2) * TR_TILE_BYTES + 1024;
-                bool &attr = esize == 4 ? g_attr_tr4 : g_attr_tr2;
-                if (!attr) {
+                int &attr = esize == 4 ? g_attr_tr4 : g_attr_tr2;
+                const int dev = current_device();
+                if (attr != dev) {
                     const cudaError_t e = esize == 4
                         ? cudaFuncSetAttribute(transpose_tma_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
                         : cudaFuncSetAttribute(transpose_tma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
                     if (e != cudaSuccess) return SG_ERR_CUDA;
-                    attr = true;
+                    attr = dev;
                 }
                 const int num_tiles = (int)(tiles_c * tiles_r);
                 const int grid = std::min(num_tiles, 2 * num_sms);

@@ -379,10 +379,12 @@ bool try_launch_tma(const DepthwiseProblem &p, const T *I, const T *Kf, float *O
                              const_cast<T *>(I), dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
         return false;
     const int smem = 2 * C::STAGE_BYTES + 128;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static int attr_device = -1;      // the attribute is per device
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (attr_device != dev) {
         if (cudaFuncSetAttribute(depthwise_tma_kernel<T, CB, S>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
-        attr_set = true;
+        attr_device = dev;
     }
     // two CTAs per SM, rounded down to a multiple of the channel blocks: tile t has block t % c_blocks, so every CTA keeps one
     int64_t grid = std::min<int64_t>(tiles, 2 * (int64_t)num_sms);
