@@ -47,7 +47,8 @@ constexpr int BM = 128;           // rows of an output tile = lanes of TMEM = M 
 constexpr int ROW_BYTES = 128;    // one k-block = one 128-byte swizzle row: 64 bf16 or 32 f32
 constexpr int K_STEPS = 4;        // tcgen05.mma per k-block and product: 32 bytes of k each
 constexpr int A_STAGE_BYTES = BM * ROW_BYTES;
-constexpr int CONVERTER_THREADS = 256;        // f32 path: 8 warps splitting tiles into hi and lo
+constexpr int CONVERTER_THREADS = 512;        // f32 path: 16 warps splitting tiles into hi and lo (one k-block is a serial
+                                              // chain of ~200 instructions per warp with 8 warps: longer than its MMAs take)
 constexpr int STAGING_BYTES = 2 * 16384;      // epilogue: 2 staging tiles of 128 rows x 128 B
 
 
@@ -465,55 +466,43 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     // An operand tile that arrives MN-major (sub-tiles of [32 k][32 rows-or-columns], 128-byte
                     // rows, not swizzled) is transposed while it is split: the split tiles are K-major,
                     // [row][32 k] rows of 128 B in 8-row groups with the 128-byte swizzle (16-byte chunk c of
-                    // row f sits at chunk c ^ (f & 7)).  A unit is a quarter of a sub-tile (8 k); lane = f
-                    // reads a column (one 128-byte row per load across the warp) and writes 2 chunks of its row.
+                    // row f sits at chunk c ^ (f & 7)).  A unit is an eighth of a sub-tile (4 k); lane = f
+                    // reads a column (one 128-byte row per load across the warp) and writes one chunk of its row.
                     auto split_transpose = [&](const uint8_t *src_tile, uint8_t *hi_tile, uint8_t *lo_tile, auto cols_tag) {
                         constexpr int COLS = decltype(cols_tag)::value;
                         const float *braw = reinterpret_cast<const float *>(src_tile);
-                        constexpr int UNITS = 4 * COLS / 32;
+                        constexpr int UNITS = 8 * COLS / 32;
 #pragma unroll
                         for (int u = cw; u < UNITS; u += CONVERTER_THREADS / 32) {
-                            const int j = u >> 2, quarter = u & 3;
-                            const float *col = braw + j * (C::SUB_BYTES / 4) + quarter * 8 * 32 + lane;
-                            uint32_t x[8];
+                            const int j = u >> 3, eighth = u & 7;
+                            const float *col = braw + j * (C::SUB_BYTES / 4) + eighth * 4 * 32 + lane;
+                            uint32_t x[4];
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) x[k] = __float_as_uint(col[k * 32]);
+                            for (int k = 0; k < 4; ++k) x[k] = __float_as_uint(col[k * 32]);
                             const int f = j * 32 + lane;
-                            const int row_off = (f >> 3) * 1024 + (f & 7) * 128;
-#pragma unroll
-                            for (int c = 0; c < 2; ++c) {
-                                uint4 h, l;
-                                split4(make_uint4(x[4 * c], x[4 * c + 1], x[4 * c + 2], x[4 * c + 3]), h, l);
-                                const int off = row_off + (((quarter * 2 + c) ^ (f & 7)) << 4);
-                                *reinterpret_cast<uint4 *>(hi_tile + off) = h;
-                                *reinterpret_cast<uint4 *>(lo_tile + off) = l;
-                            }
+                            const int off = (f >> 3) * 1024 + (f & 7) * 128 + ((eighth ^ (f & 7)) << 4);
+                            uint4 h, l;
+                            split4(make_uint4(x[0], x[1], x[2], x[3]), h, l);
+                            *reinterpret_cast<uint4 *>(hi_tile + off) = h;
+                            *reinterpret_cast<uint4 *>(lo_tile + off) = l;
                         }
                     };
                     // input: K-major as stored, M-major when stored transposed; filter: N-major as stored,
                     // K-major when stored transposed.  kind::tf32 takes K-major operands only.
                     uint8_t *b_slot = slot + (TA ? 0 : 2 * A_STAGE_BYTES);
+                    // Order within a k-block: the input rows are read first, the filter part (shared memory to shared
+                    // memory) runs while those loads are in flight, then the input part goes to tensor memory and the
+                    // proxy fence for the filter writes overlaps the tensor-memory stores; one wait at the end.
+                    uint4 a_raw[2];
                     if constexpr (TA) {
-                        // input tile -> tensor memory: this warp may touch lane quarter (warp & 3); the two warps
-                        // of a quarter take 16 of the 32 k columns each.  Lane = row reads its 64 bytes of the
-                        // swizzled raw tile and stores 16 hi and 16 lo words.
-                        const int quarter = warp & 3, khalf = cw >> 2;
-                        const int row = quarter * 32 + lane;
+                        // input tile -> tensor memory: this warp may touch lane quarter (warp & 3); the four warps
+                        // of a quarter take 8 of the 32 k columns each.  Lane = row reads its 32 bytes of the
+                        // swizzled raw tile and stores 8 hi and 8 lo words.
+                        const int row = (warp & 3) * 32 + lane;
                         const uint8_t *rp = raw + row * 128;
-                        uint32_t hi[16], lo[16];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint4 v = *reinterpret_cast<const uint4 *>(rp + (((khalf * 4 + i) ^ (row & 7)) << 4));
-                            uint4 h, l;
-                            split4(v, h, l);
-                            hi[4 * i] = h.x; hi[4 * i + 1] = h.y; hi[4 * i + 2] = h.z; hi[4 * i + 3] = h.w;
-                            lo[4 * i] = l.x; lo[4 * i + 1] = l.y; lo[4 * i + 2] = l.z; lo[4 * i + 3] = l.w;
-                        }
-                        const uint32_t t_hi = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(C::ACC_BUFS * BN + s * 64 + khalf * 16);
-                        tmem_st_32x16(t_hi, hi);
-                        tmem_st_32x16(t_hi + 32, lo);
-                        tmem_st_wait();
-                        tc_fence_before();
+                        for (int i = 0; i < 2; ++i)
+                            a_raw[i] = *reinterpret_cast<const uint4 *>(rp + ((((cw >> 2) * 2 + i) ^ (row & 7)) << 4));
                     } else if constexpr (A_MN) {
                         split_transpose(raw, slot, slot + A_STAGE_BYTES, std::integral_constant<int, BM>{});
                     } else {
@@ -523,7 +512,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                         split_elementwise(raw + A_STAGE_BYTES, b_slot, b_slot + C::B_STAGE_BYTES, std::integral_constant<int, C::B_STAGE_BYTES>{});
                     else
                         split_transpose(raw + A_STAGE_BYTES, b_slot, b_slot + C::B_STAGE_BYTES, std::integral_constant<int, C::B_COLS>{});
+                    if constexpr (TA) {
+                        const int quarter = warp & 3, kpart = cw >> 2;
+                        uint32_t hi[8], lo[8];
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {
+                            uint4 h, l;
+                            split4(a_raw[i], h, l);
+                            hi[4 * i] = h.x; hi[4 * i + 1] = h.y; hi[4 * i + 2] = h.z; hi[4 * i + 3] = h.w;
+                            lo[4 * i] = l.x; lo[4 * i + 1] = l.y; lo[4 * i + 2] = l.z; lo[4 * i + 3] = l.w;
+                        }
+                        const uint32_t t_hi = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(C::ACC_BUFS * BN + s * 64 + kpart * 8);
+                        tmem_st_32x8(t_hi, hi);
+                        tmem_st_32x8(t_hi + 32, lo);
+                    }
                     fence_async_smem();     // generic-proxy writes -> visible to the tensor core's reads
+                    if constexpr (TA) {
+                        tmem_st_wait();
+                        tc_fence_before();
+                    }
                     __syncwarp();
                     if (lane == 0) {
                         mbar_arrive(empty_bar(r));          // the raw stage may be refilled
