@@ -42,7 +42,7 @@ FLOPS_PER_STEP = 2 * FLOPS_PER_DTYPE
 
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture; None when the
 # kernel changed after the capture was taken.
-NCU_TRAFFIC_BYTES = 25.5e6   # profiles/bench_sweep_launch_list.md: average over the 125 f32 launches of a step
+NCU_TRAFFIC_BYTES = 25.4e6   # profiles/bench_sweep_launch_list.md: average over the 125 f32 launches of a step
 # tf32 : bf16 dense tensor throughput (nominal 1.1 : 2.25 PFLOP/s; the issue rate measured on
 # this chip is exactly half)
 TF32_OVER_BF16 = 0.5
@@ -585,7 +585,7 @@ def main():
                 "kernel": "tc_gemm_kernel<BN, CG, f32> (125 launches per step, %.0f%% of the step)" % (100 * share_f32),
                 "peak_source": f"{peaks['source']} {peak_kind} x {TF32_OVER_BF16} (tf32 : bf16 tensor rate); timed region {timed_seconds:.2f} s",
                 "algorithmic_flops_per_step": FLOPS_PER_DTYPE, "avg_launch_us": round(ms_per_step * share_f32 * 1e3 / len(SHAPES), 2),
-                "note": "f32 accuracy costs three tf32 products per term, so this kernel's own ceiling is frac = 0.333",
+                "note": "f32 accuracy costs three tf32 products per term, so this kernel's own ceiling is about frac = 0.333 (the peak is a measured cuBLAS rate, not a hard limit)",
                 "frac_of_3xtf32_ceiling": round(3 * f32_tf / tf32_peak, 4),
                 "bf16_half": {"achieved": round(bf16_tf, 1), "peak": peaks[peak_kind], "frac": round(bf16_tf / peaks[peak_kind], 4),
                               "share_of_step": round(1 - share_f32, 4)}}
