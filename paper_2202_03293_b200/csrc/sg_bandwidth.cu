@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(64) copy_tma_kernel(const __grid_constant__ CU
                 mbar_arrive(smem_u32(&empty_bar[(k - CP_STORES_IN_FLIGHT) % CP_STAGES]));
             }
         }
-        bulk_wait_all();
+        bulk_wait_read<0>();      // the ring must stay until the last stores have read it; the grid's end completes the writes
     }
     __syncthreads();
 }
@@ -259,7 +259,7 @@ __global__ void __launch_bounds__(TR_THREADS) transpose_tma_kernel(const __grid_
                 bulk_commit();
             }
         }
-        if (lane == 0) bulk_wait_all();
+        if (lane == 0) bulk_wait_read<0>();
     }
     __syncthreads();
 }

@@ -595,7 +595,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                 else mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));
             }
         }
-        if (lane == 0) bulk_wait_all();
+        // the staging tiles must stay until the last stores have read them; the writes themselves are complete
+        // when the grid is
+        if (lane == 0) bulk_wait_read<0>();
     }
 
     // ---------------------------------------------------------------- teardown
