@@ -633,7 +633,7 @@ struct Driver {
     EncodeIm2colFn im2col = nullptr;
     int num_sms = 0;
     int device = -1;
-    bool attr_set[96] = {};
+    bool attr_set[128] = {};
     bool ok = false;
 };
 std::mutex g_mu;
@@ -704,7 +704,7 @@ sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUt
                          int slot, cudaStream_t stream) {
   if constexpr ((F32 && BN == 256 && CG == 1) || (KPS == 2 && (F32 || (BN == 256 && CG == 1))) ||
                 ((LAY & 3) != 0 && (KPS != 1 || (BN == 256 && CG == 1) || (BN == 128 && CG == 2))) ||
-                ((LAY & 4) != 0 && (!F32 || (LAY & 3) != 0))) {
+                ((LAY & 4) != 0 && (!F32 || (LAY & 1) != 0))) {
     return SG_ERR_INTERNAL;   // the split slots of a 128 x 256 f32 tile do not fit beside a TMA ring
   } else {
     using C = Cfg<BN, CG, F32, KPS, (LAY & 4) != 0>;
@@ -959,13 +959,14 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         tp.accumulate = 1;
     }
     g_last_choice[0] = kVariants[pick].bn; g_last_choice[1] = kVariants[pick].cg; g_last_choice[2] = splits;
-    // f32, plain layout: the split input tile goes to tensor memory unless that costs the second
+    // f32, input stored [m][k] (the filter may be stored either way): the split input tile goes to tensor memory unless that costs the second
     // accumulator buffer (256 columns) on a reduction too short to pay for the lost overlap
-    const int lay_k = (f32 && lay == 0 && g_ta_override != 0 &&
-                       (kVariants[pick].bn < 256 || tp.kb_per_split >= 24 || g_ta_override == 1)) ? 4 : lay;
+    const int lay_k = (f32 && (lay & 1) == 0 && g_ta_override != 0 &&
+                       (kVariants[pick].bn < 256 || tp.kb_per_split >= 24 || g_ta_override == 1)) ? (lay | 4) : lay;
     const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0) + lay_k * 3 * kNumVariants;
 #define SG_LAUNCH(BN_, CG_)                                                                                \
     (f32 ? (lay_k == 4 ? launch_variant<BN_, CG_, true, 1, 4>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)     \
+            : lay_k == 6 ? launch_variant<BN_, CG_, true, 1, 6>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)   \
             : lay == 0 ? launch_variant<BN_, CG_, true, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)         \
             : lay == 1 ? launch_variant<BN_, CG_, true, 1, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
             : lay == 2 ? launch_variant<BN_, CG_, true, 1, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
