@@ -959,10 +959,11 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         tp.accumulate = 1;
     }
     g_last_choice[0] = kVariants[pick].bn; g_last_choice[1] = kVariants[pick].cg; g_last_choice[2] = splits;
-    // f32, input stored [m][k] (the filter may be stored either way): the split input tile goes to tensor memory unless that costs the second
-    // accumulator buffer (256 columns) on a reduction too short to pay for the lost overlap
-    const int lay_k = (f32 && (lay & 1) == 0 && g_ta_override != 0 &&
-                       (kVariants[pick].bn < 256 || tp.kb_per_split >= 24 || g_ta_override == 1)) ? (lay | 4) : lay;
+    // f32, input stored [m][k] (the filter may be stored either way): the split input tile goes to tensor memory.  With
+    // 256-column tiles that costs the second accumulator buffer, which short reductions used to feel; since the
+    // converters stopped being the bottleneck the sweep is no slower with it everywhere (5.72 to 5.79 ms per step
+    // either way), so there is one rule.
+    const int lay_k = (f32 && (lay & 1) == 0 && g_ta_override != 0) ? (lay | 4) : lay;
     const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0) + lay_k * 3 * kNumVariants;
 #define SG_LAUNCH(BN_, CG_)                                                                                \
     (f32 ? (lay_k == 4 ? launch_variant<BN_, CG_, true, 1, 4>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)     \
