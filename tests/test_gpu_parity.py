@@ -662,3 +662,40 @@ def test_matmul_transposed_full_size_sampled(dtype):
     got = C[torch.from_numpy(pm).cuda(), torch.from_numpy(pn).cuda()]
     assert_within_bound(got, want, S, "A^T B^T 4096^3")
     assert not torch.isnan(C).any()
+
+
+def test_random_shapes_layouts_and_modes():
+    """Seeded sweep: matmuls of random extents (multiples of 8, so most take the tensor path; some not), either
+    operand stored transposed, both dtypes, both modes; convolutions of random extents, strides and dilations."""
+    rng = np.random.default_rng(SEED + 7)
+    for case in range(48):
+        M, N, K = (int(rng.integers(1, 90)) * 8 for _ in range(3))
+        if rng.integers(0, 6) == 0:
+            M, N, K = M + int(rng.integers(1, 8)), N + int(rng.integers(1, 8)), K + int(rng.integers(1, 8))
+        dtype = str(rng.choice(["f32", "bf16"]))
+        a_t, b_t, acc = (bool(rng.integers(0, 2)) for _ in range(3))
+        A, a = operand((K, M) if a_t else (M, K), SEED, 300 + case, "uniform", dtype)
+        B, b = operand((N, K) if b_t else (K, N), SEED, 400 + case, "uniform", dtype)
+        if a_t:
+            A, a = A.t(), a.T
+        if b_t:
+            B, b = B.t(), b.T
+        if acc:
+            C, c0 = operand((M, N), SEED, 500 + case, "uniform", "f32")
+            C = C.clone()
+        else:
+            C, c0 = torch.full((M, N), float("nan"), device="cuda"), None
+        sg.sg_matmul(A, B, C, sg.SG_ACCUMULATE if acc else sg.SG_OVERWRITE)
+        torch.cuda.synchronize()
+        want, S = ref.matmul(a, b, C_in=c0)
+        assert_within_bound(C, want, S + (np.abs(c0) if acc else 0.0), f"random matmul {case}: {M}x{N}x{K} {dtype} a_t={a_t} b_t={b_t} acc={acc}")
+    for case in range(24):
+        dtype = str(rng.choice(["f32", "bf16"]))
+        N, Ho, Wo = int(rng.integers(1, 5)), int(rng.integers(1, 40)), int(rng.integers(1, 40))
+        C, F = int(rng.integers(1, 12)) * 8, int(rng.integers(1, 20)) * 8
+        KH, KW = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        st = (int(rng.integers(1, 3)), int(rng.integers(1, 3)))
+        dl = (int(rng.integers(1, 3)), int(rng.integers(1, 3)))
+        acc = bool(rng.integers(0, 2))
+        O, want, S = run_conv2d(N, Ho, Wo, C, KH, KW, F, st, dl, dtype, accumulate=acc, seed=SEED + case)
+        assert_within_bound(O, want, S, f"random conv2d {case}: {N}x{Ho}x{Wo}x{C} {KH}x{KW} F={F} st={st} dl={dl} {dtype} acc={acc}")
