@@ -427,7 +427,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
             }
         }
     } else if (warp >= 6) {
-        // ------------------------------------------------------------ converter (f32 only; warps 6 to 13)
+        // ------------------------------------------------------------ converter (f32 only; warps 6 to 21)
         if constexpr (F32) {
             const int cw = warp - 6;                       // converter warp
             const int ct = (int)threadIdx.x - 192;         // converter thread
