@@ -22,9 +22,10 @@
 //                          an MN-major operand instead of being transposed.
 //
 // f32 inputs run on the same pipeline as three tf32 products per k-step ("3xTF32"): the TMA
-// writes the raw f32 tiles into its ring, four converter warps split every element x into two
+// writes the raw f32 tiles into its ring, sixteen converter warps split every element x into two
 // values hi = x rounded to tf32 and lo = x - hi and write them to a second ring of two slots
-// (transposing the filter tile to K-major on the way, which kind::tf32 needs), and the MMA
+// (transposing the filter tile to K-major on the way, which kind::tf32 needs; the input tile's
+// hi and lo go to tensor memory when it is stored [m][k]), and the MMA
 // thread accumulates lo*hi + hi*lo + hi*hi in f32: the dropped terms are below 2^-21 |a*b|, so
 // f32 accuracy is kept.  Raw tiles are 128 rows x 32 f32 (input) and 32 k-rows x 32 f32
 // sub-tiles (filter), again 128 bytes per row.
