@@ -194,6 +194,7 @@ sg_status sg_transpose2d(int64_t R, int64_t C, const void *src, int64_t src_stri
  * or leaves out untouched (SG_ACCUMULATE).  When the shape has too few outputs to occupy the
  * GPU the reduced index is split across thread blocks whose partial sums are added into `out`
  * with float atomics, so the rounding of the last bits may differ from call to call.
+ * `out` must not overlap A.
  */
 sg_status sg_colred2d(int64_t R, int64_t C, const void *A, int64_t a_stride_r, int64_t a_stride_c,
                       float *out, int64_t out_stride, sg_dtype in_dtype, int mode, sg_stream_t stream);
