@@ -10,9 +10,10 @@
 //     aligned bases and row pitches), move tiles with TMA only: a persistent CTA per SM slot runs
 //     a shared-memory ring that one thread fills with tensor loads and another drains with tensor
 //     stores.  The copy never touches the data with an ordinary instruction; the transpose has
-//     four warps turn each 128-row tile around in shared memory (16-byte reads of the 128-byte
-//     swizzled input tile, a register transpose of an E x E block, 16-byte writes into the
-//     swizzled output tile) between the load and the store.  Ragged edges cost nothing: loads
+//     four warps turn each 128-row tile around in shared memory between the load and the store
+//     (4-byte elements: 16-byte reads of the 128-byte swizzled input tile, a register transpose
+//     of a 4 x 4 block, 16-byte writes into the swizzled output tile; 2-byte elements: 8 x 8
+//     blocks through ldmatrix.trans and stmatrix).  Ragged edges cost nothing: loads
 //     read zeros beyond the tensor, stores are clipped.
 //   - The reductions use plain 16-byte loads with four in flight per thread at full occupancy,
 //     f32 accumulators, and a shared-memory / shuffle tree per CTA.  When the shape has too few
@@ -117,26 +118,12 @@ constexpr int TR_IN_STAGES = 4;
 constexpr int TR_TILE_BYTES = 16384;
 constexpr int TR_THREADS = 32 + 128;
 
-template <int ES>
-__device__ __forceinline__ void transpose_block(const uint4 (&v)[16 / ES], uint4 (&o)[16 / ES]) {
-    if constexpr (ES == 4) {
-        o[0] = make_uint4(v[0].x, v[1].x, v[2].x, v[3].x);
-        o[1] = make_uint4(v[0].y, v[1].y, v[2].y, v[3].y);
-        o[2] = make_uint4(v[0].z, v[1].z, v[2].z, v[3].z);
-        o[3] = make_uint4(v[0].w, v[1].w, v[2].w, v[3].w);
-    } else {
-        // 8 x 8 block of 2-byte elements: output row j gathers element j of every input row
-        uint32_t in[8][4], out[8][4];
-#pragma unroll
-        for (int r = 0; r < 8; ++r) { in[r][0] = v[r].x; in[r][1] = v[r].y; in[r][2] = v[r].z; in[r][3] = v[r].w; }
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-#pragma unroll
-            for (int w = 0; w < 4; ++w)
-                out[j][w] = __byte_perm(in[2 * w][j >> 1], in[2 * w + 1][j >> 1], (j & 1) ? 0x7632 : 0x5410);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) o[j] = make_uint4(out[j][0], out[j][1], out[j][2], out[j][3]);
-    }
+// 4 x 4 block of 4-byte elements held as four 16-byte rows: the transpose is a renaming of registers.
+__device__ __forceinline__ void transpose_block(const uint4 (&v)[4], uint4 (&o)[4]) {
+    o[0] = make_uint4(v[0].x, v[1].x, v[2].x, v[3].x);
+    o[1] = make_uint4(v[0].y, v[1].y, v[2].y, v[3].y);
+    o[2] = make_uint4(v[0].z, v[1].z, v[2].z, v[3].z);
+    o[3] = make_uint4(v[0].w, v[1].w, v[2].w, v[3].w);
 }
 
 // Tile order: panels of `panel` tile columns, walked row by row inside a panel.  The tiles in flight at one time then
@@ -238,7 +225,7 @@ __global__ void __launch_bounds__(TR_THREADS) transpose_tma_kernel(const __grid_
                         const uint32_t addr = in_tile + (uint32_t)row * 128u + (uint32_t)((q ^ (row & 7)) << 4);
                         asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v[kk].x), "=r"(v[kk].y), "=r"(v[kk].z), "=r"(v[kk].w) : "r"(addr));
                     }
-                    transpose_block<ES>(v, o);
+                    transpose_block(v, o);
 #pragma unroll
                     for (int j = 0; j < E; ++j) {
                         const int c = E * q + j;                       // output row within the tile
