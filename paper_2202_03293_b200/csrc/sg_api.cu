@@ -274,7 +274,7 @@ const char *sg_status_string(sg_status status) {
     return "unknown status";
 }
 
-int sg_version(void) { return 100; }
+int sg_version(void) { return 200; }   // 0.2.0: depthwise convolutions and the memory-bound 2-D kernels joined the three contractions
 
 int sg_last_kernel(void) { return t_last_kernel; }
 
