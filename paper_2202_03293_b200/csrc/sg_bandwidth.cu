@@ -380,6 +380,8 @@ __global__ void __launch_bounds__(256) colred_kernel(const T *__restrict__ A, in
 #pragma unroll
     for (int v = 0; v < VEC; ++v) red[t][v] = acc[v];
     __syncthreads();
+    // (after the clearing kernel of an overwriting split reduction; this grid may have started beside it)
+    if (use_atomic) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (g == 0 && col0 < C) {
         for (int gg = 1; gg < rp; ++gg)
 #pragma unroll
@@ -450,6 +452,7 @@ __global__ void __launch_bounds__(256) rowred_kernel(const T *__restrict__ A, in
 #pragma unroll
     for (int v = 1; v < VEC; ++v) sum += acc[v];
     for (int off = lanes >> 1; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    if (use_atomic) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (sub == 0 && row < R && (c0 < c1 || blockIdx.y == 0)) {
         float *o = out + row * os;
         if (use_atomic) atomicAdd(o, sum);
@@ -458,7 +461,24 @@ __global__ void __launch_bounds__(256) rowred_kernel(const T *__restrict__ A, in
 }
 
 __global__ void zero_vector_kernel(float *__restrict__ out, int64_t n, int64_t os) {
+    asm volatile("griddepcontrol.launch_dependents;");   // the reduction behind it may start; it waits before its atomics
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) out[i * os] = 0.f;
+}
+
+// Launches `kernel`; `after_clear`: a clearing kernel was just enqueued ahead of it and the launch may overlap it
+// (programmatic dependent launch; the kernel waits for the clearing grid before its first atomic).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_reduction(void (*kernel)(KArgs...), dim3 grid, bool after_clear, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_clear ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 template <typename T, int VEC>
@@ -484,8 +504,10 @@ cudaError_t launch_reduce_typed(bool colred, const T *A, int64_t ld, int64_t sc,
             zero_vector_kernel<<<(int)std::min<int64_t>(((int64_t)R + 255) / 256, 1184), 256, 0, stream>>>(out, R, os);
             count_launch();
         }
-        rowred_kernel<T, VEC><<<dim3((unsigned)row_ctas, (unsigned)splits), 256, 0, stream>>>(A, ld, sc, R, C, out, os, lanes,
-                                                                                              chunks_per_split * VEC, use_atomic, accumulate);
+        const cudaError_t e = launch_reduction(rowred_kernel<T, VEC>, dim3((unsigned)row_ctas, (unsigned)splits), use_atomic && !accumulate, stream,
+                                               A, ld, sc, R, C, out, os, lanes, chunks_per_split * VEC, use_atomic, accumulate);
+        count_launch();
+        return e;
     } else {
         // ColRed2D: one output per column
         const int64_t chunks = ((int64_t)C + VEC - 1) / VEC;
@@ -513,11 +535,11 @@ cudaError_t launch_reduce_typed(bool colred, const T *A, int64_t ld, int64_t sc,
             zero_vector_kernel<<<(int)std::min<int64_t>(((int64_t)C + 255) / 256, 1184), 256, 0, stream>>>(out, C, os);
             count_launch();
         }
-        colred_kernel<T, VEC><<<dim3((unsigned)col_blocks, (unsigned)splits), 256, 0, stream>>>(A, ld, sc, R, C, out, os, cw, rp,
-                                                                                                rows_per_split, use_atomic, accumulate);
+        const cudaError_t e = launch_reduction(colred_kernel<T, VEC>, dim3((unsigned)col_blocks, (unsigned)splits), use_atomic && !accumulate, stream,
+                                               A, ld, sc, R, C, out, os, cw, rp, rows_per_split, use_atomic, accumulate);
+        count_launch();
+        return e;
     }
-    count_launch();
-    return cudaGetLastError();
 }
 
 template <typename U>

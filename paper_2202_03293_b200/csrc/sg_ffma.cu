@@ -208,6 +208,7 @@ ffma_kernel(Problem p, const T *__restrict__ In, const T *__restrict__ Flt, floa
 }
 
 __global__ void zero_fill_kernel(Problem p, float *__restrict__ O) {
+    asm volatile("griddepcontrol.launch_dependents;");   // a dependent launch waits for this grid's end where it needs the zeros
     int64_t total = (int64_t)p.M * p.N;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (int64_t)gridDim.x * blockDim.x) {
@@ -221,6 +222,7 @@ __global__ void zero_fill_kernel(Problem p, float *__restrict__ O) {
 // The output as one M x N matrix of contiguous, 16-byte aligned rows `pitch` floats apart
 // (what the tensor-core path requires of it): four columns per thread.
 __global__ void zero_fill_rows_kernel(float *__restrict__ O, int M, int n4, int64_t pitch) {
+    asm volatile("griddepcontrol.launch_dependents;");
     const int64_t total = (int64_t)M * n4;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const int m = (int)(i / n4), c = (int)(i - (int64_t)m * n4);

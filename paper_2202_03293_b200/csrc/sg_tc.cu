@@ -65,6 +65,8 @@ struct TcParams {
     int Ho, Wo, sh, sw, dh, dw;
     int accumulate;
     int b_blocked;       // 1: the filter map is blocked by sub-tile columns: one TMA load fetches the whole filter tile
+    int wait_prior;      // 1: the launch may start before the clearing kernel ahead of it has finished (programmatic
+                         //    dependent launch): nothing may be added into the output before griddepcontrol.wait
 };
 
 // 3xTF32 split of four f32 words.  hi = x rounded to the nearest tf32 value (10 mantissa bits;
@@ -552,6 +554,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         auto epi_sync = [] { asm volatile("bar.sync 1, 128;" ::: "memory"); };
         int tl = 0, chunk_count = 0;
         bool ok = true;
+        // a split reduction that overwrites follows a kernel that clears the output: this grid was allowed to start (and
+        // to run its whole first reduction) beside it, but the first reduce-add must see the cleared output
+        if (p.wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
         for (int t = group_id; t < num_tiles && ok; t += num_groups, ++tl) {
             int mt, nt;
             tile_coords(t / p.splits, p.num_m_tiles, p.num_n_tiles, mt, nt);
@@ -724,13 +729,15 @@ sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUt
     cfg.blockDim = dim3(C::THREADS, 1, 1);
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = CG;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = tp.wait_prior ? 2 : 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<BN, CG, F32, KPS, LAY>, mi, mf, mo, tp);
     count_launch();
     return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
@@ -956,7 +963,10 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     tp.kb_per_split = per;
     if (splits > 1) {
         // partial sums meet in the output by TMA reduce-add: an overwriting call clears it first
-        if (!p.accumulate && launch_zero_fill(p, O, stream) != cudaSuccess) return SG_ERR_CUDA;
+        if (!p.accumulate) {
+            if (launch_zero_fill(p, O, stream) != cudaSuccess) return SG_ERR_CUDA;
+            tp.wait_prior = 1;      // the clearing kernel lets its dependents start at once
+        }
         tp.accumulate = 1;
     }
     g_last_choice[0] = kVariants[pick].bn; g_last_choice[1] = kVariants[pick].cg; g_last_choice[2] = splits;
