@@ -254,6 +254,15 @@ sg_status sg_set_tile_override(int tile_n, int ctas_per_tile, int k_splits);
 /* {tile width, CTAs per tile, k ranges} of the most recent tensor-core launch of the process. */
 void sg_last_tile_choice(int out[3]);
 
+/*
+ * Stream-K tail of the most recent tensor-core launch of the process: when whole tiles are dealt out and the last
+ * wave of tiles would be partly filled, the tiles of that wave are cut along the reduction instead (every CTA or CTA
+ * pair gets an equal run of their k-blocks; the partial sums meet in the output by reduce-add).  out[0] = index of
+ * the first tile of the tail in the tile order (-1: no tail), out[1] = k-blocks per run.  SG_TC_SK=0 in the
+ * environment (read at the first call) turns the tail off.
+ */
+void sg_last_stream_k(int out[2]);
+
 /* Drops cached tensor maps and other host-side state.  Safe to call twice. */
 void sg_shutdown(void);
 

@@ -25,7 +25,7 @@ EXPORTS = [
     "sg_matmul", "sg_conv1d_nwc_wcf", "sg_conv2d_nhwc_hwcf", "sg_depthwise_conv1d_nwc_wc",
     "sg_depthwise_conv2d_nhwc_hwc", "sg_copy2d", "sg_transpose2d", "sg_colred2d", "sg_rowred2d", "sg_check", "sg_status_string",
     "sg_version", "sg_last_kernel", "sg_launch_count", "sg_set_kernel_override", "sg_set_tile_override",
-    "sg_last_tile_choice", "sg_shutdown",
+    "sg_last_tile_choice", "sg_last_stream_k", "sg_shutdown",
 ]
 
 
@@ -74,6 +74,8 @@ def lib() -> ctypes.CDLL:
         L.sg_set_tile_override.restype = ci
         L.sg_last_tile_choice.argtypes = [ctypes.POINTER(ctypes.c_int)]
         L.sg_last_tile_choice.restype = None
+        L.sg_last_stream_k.argtypes = [ctypes.POINTER(ctypes.c_int)]
+        L.sg_last_stream_k.restype = None
         L.sg_shutdown.restype = None
         _lib = L
     return _lib
@@ -263,6 +265,12 @@ def sg_last_tile_choice():
     out = (ctypes.c_int * 3)()
     lib().sg_last_tile_choice(out)
     return out[0], out[1], out[2]
+
+
+def sg_last_stream_k():
+    out = (ctypes.c_int * 2)()
+    lib().sg_last_stream_k(out)
+    return out[0], out[1]
 
 
 def sg_shutdown() -> None:

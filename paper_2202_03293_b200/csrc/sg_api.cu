@@ -299,6 +299,8 @@ void sg_last_tile_choice(int out[3]) {
     if (out) tensor_last_choice(out);
 }
 
+void sg_last_stream_k(int out[2]) { sg::tensor_last_stream_k(out); }
+
 void sg_shutdown(void) { tensor_shutdown(); }
 
 }  // extern "C"

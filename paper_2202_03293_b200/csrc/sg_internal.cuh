@@ -54,6 +54,7 @@ sg_status launch_conv_strip(const Problem &p, const void *In, const void *Flt, f
 sg_status conv_read_status(cudaStream_t stream);
 void tensor_set_tile_override(int bn, int cg, int splits);
 void tensor_last_choice(int out[3]);
+void tensor_last_stream_k(int out[2]);
 // Reads and clears the current device's status word (written by kernels whose bounded
 // waits expire); the caller has already synchronised the stream.
 sg_status tensor_read_status(cudaStream_t stream);

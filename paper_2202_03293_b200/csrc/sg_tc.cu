@@ -65,6 +65,8 @@ struct TcParams {
     int Ho, Wo, sh, sw, dh, dw;
     int accumulate;
     int b_blocked;       // 1: the filter map is blocked by sub-tile columns: one TMA load fetches the whole filter tile
+    int sk_first_tile;   // stream-K tail: tiles from this one on are not dealt out whole; their k-blocks, taken as one
+    int sk_units;        //   sequence, are cut into equal runs of `sk_units` k-blocks, one run per CTA (or pair); 0 = no tail
     int wait_prior;      // 1: the launch may start before the clearing kernel ahead of it has finished (programmatic
                          //    dependent launch): nothing may be added into the output before griddepcontrol.wait
 };
@@ -152,6 +154,20 @@ __device__ __forceinline__ void tile_coords(int t, int num_m_tiles, int num_n_ti
 // LAY (bf16 matmuls, one k-block per stage): bit 0 = the input operand is stored transposed
 // ([k][m], m contiguous: A^T B of Section 4.6.1) and consumed as an M-major operand; bit 1 = the
 // filter operand is stored transposed ([n][k], k contiguous: A B^T) and consumed K-major.
+// Clears the output tiles first_tile .. (one block per tile) ahead of a launch whose stream-K tail adds into them.
+__global__ void __launch_bounds__(256) zero_tiles_kernel(float *__restrict__ O, int64_t pitch, int M, int N, int tile_rows, int tile_cols,
+                                                         int num_m_tiles, int num_n_tiles, int first_tile) {
+    asm volatile("griddepcontrol.launch_dependents;");     // the launch behind waits for this grid before its first store
+    int mt, nt;
+    tile_coords(first_tile + (int)blockIdx.x, num_m_tiles, num_n_tiles, mt, nt);
+    const int m0 = mt * tile_rows, n0 = nt * tile_cols;
+    const int rows = min(tile_rows, M - m0), c4 = min(tile_cols, N - n0) / 4;      // N is a multiple of 4 on this path
+    for (int i = threadIdx.x; i < rows * c4; i += 256) {
+        const int r = i / c4, c = i - r * c4;
+        reinterpret_cast<float4 *>(O + (int64_t)(m0 + r) * pitch + n0)[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+}
+
 template <int BN, int CG, bool F32, int KPS, int LAY>
 __global__ void __launch_bounds__(Cfg<BN, CG, F32, KPS, (LAY & 4) != 0>::THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_flt,
@@ -222,12 +238,34 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     const uint32_t tmem_base = *tmem_ptr_slot;
 
     // work items: (tile of (CG*128) x BN, k range); the splits of one tile are neighbours in the
-    // order, so they run at the same time and their operands meet in L2
-    const int num_tiles = p.num_m_tiles * p.num_n_tiles * p.splits;
-    auto item_range = [&](int t, int &tile, int &kb0, int &kb1) {
-        tile = t / p.splits;
-        kb0 = (t - tile * p.splits) * p.kb_per_split;
-        kb1 = kb0 + p.kb_per_split < p.num_kb ? kb0 + p.kb_per_split : p.num_kb;
+    // order, so they run at the same time and their operands meet in L2.  Every role walks the same
+    // sequence: first the items dealt round-robin (whole tiles, or `splits` equal k ranges per tile), then
+    // this group's run of the stream-K tail: the tiles that would make a last, partly filled wave are
+    // not dealt out whole; their k-blocks, taken as one sequence, are cut into equal runs, one per group,
+    // and each run is one to three (tile, k range) items whose partial sums meet in the output by reduce-add.
+    const int total_tiles = p.num_m_tiles * p.num_n_tiles;
+    const int dealt_items = (p.sk_units > 0 ? p.sk_first_tile : total_tiles) * p.splits;
+    const int sk_total = p.sk_units > 0 ? (total_tiles - p.sk_first_tile) * p.num_kb : 0;
+    const int sk_u0 = min(sk_total, group_id * p.sk_units), sk_u1 = min(sk_total, sk_u0 + p.sk_units);
+    struct Cursor { int i, u; };
+    auto next_item = [&](Cursor &c, int &tile, int &kb0, int &kb1, int &add) -> bool {
+        const int t = group_id + c.i * num_groups;
+        if (t < dealt_items) {
+            tile = t / p.splits;
+            kb0 = (t - tile * p.splits) * p.kb_per_split;
+            kb1 = kb0 + p.kb_per_split < p.num_kb ? kb0 + p.kb_per_split : p.num_kb;
+            add = p.accumulate;
+            ++c.i;
+            return true;
+        }
+        if (c.u >= sk_u1) return false;
+        const int first = c.u / p.num_kb;
+        tile = p.sk_first_tile + first;
+        kb0 = c.u - first * p.num_kb;
+        kb1 = min(p.num_kb, kb0 + (sk_u1 - c.u));
+        c.u += kb1 - kb0;
+        add = 1;
+        return true;
     };
     // bf16 pairs count both CTAs' TMA bytes on the leader's barrier, which its MMA thread waits
     // on.  f32 pairs signal each CTA's own barrier (its converter warps wait there) and the
@@ -241,9 +279,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
             const bool input_side = warp == 0;
             int it = 0;   // k-block counter across all of this CTA's tiles
             bool ok = true;
-            for (int t = group_id; t < num_tiles && ok; t += num_groups) {
-                int mt, nt, tile, kb0, kb1;
-                item_range(t, tile, kb0, kb1);
+            Cursor cur{0, sk_u0};
+            int tile, kb0, kb1, add;
+            while (ok && next_item(cur, tile, kb0, kb1, add)) {
+                int mt, nt;
                 tile_coords(tile, p.num_m_tiles, p.num_n_tiles, mt, nt);
                 const int m0 = (mt * CG + (int)cta_rank) * BM;
                 const int n0 = nt * BN + (int)cta_rank * C::B_COLS;
@@ -343,13 +382,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
             };
             int it = 0, tl = 0;
             bool ok = true;
-            for (int t = group_id; t < num_tiles && ok; t += num_groups, ++tl) {
+            Cursor cur{0, sk_u0};
+            int tile, kb0, kb1, add;
+            for (; ok && next_item(cur, tile, kb0, kb1, add); ++tl) {
                 const int buf = tl % C::ACC_BUFS;
                 if (!wait_all(mbar_wait(acc_empty_bar(buf), ((tl / C::ACC_BUFS) & 1) ^ 1u, abort_flag))) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
-                int tile, kb0, kb1;
-                item_range(t, tile, kb0, kb1);
                 for (int kb = kb0; kb < kb1; kb += KPS, ++it) {
                     if constexpr (F32) {
                         const int s = it & 1;
@@ -436,9 +475,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
             const int ct = (int)threadIdx.x - 192;         // converter thread
             int it = 0;
             bool ok = true;
-            for (int t = group_id; t < num_tiles && ok; t += num_groups) {
-                int tile, kb0, kb1;
-                item_range(t, tile, kb0, kb1);
+            Cursor cur{0, sk_u0};
+            int tile, kb0, kb1, add;
+            while (ok && next_item(cur, tile, kb0, kb1, add)) {
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int r = it % C::STAGES, s = it & 1;
                     if (!mbar_wait(full_bar(r), (it / C::STAGES) & 1, abort_flag)) { ok = false; break; }
@@ -557,9 +596,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         // a split reduction that overwrites follows a kernel that clears the output: this grid was allowed to start (and
         // to run its whole first reduction) beside it, but the first reduce-add must see the cleared output
         if (p.wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
-        for (int t = group_id; t < num_tiles && ok; t += num_groups, ++tl) {
+        Cursor cur{0, sk_u0};
+        int tile, kb0, kb1, add;
+        for (; ok && next_item(cur, tile, kb0, kb1, add); ++tl) {
             int mt, nt;
-            tile_coords(t / p.splits, p.num_m_tiles, p.num_n_tiles, mt, nt);
+            tile_coords(tile, p.num_m_tiles, p.num_n_tiles, mt, nt);
             const int m0 = (mt * CG + (int)cta_rank) * BM, n0 = nt * BN;
             const int buf = tl % C::ACC_BUFS;
             // (the barrier's phase stays complete until these warps hand the buffer back, so the four
@@ -587,7 +628,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                 if (lane == 0 && ew == (chunk_count & 3)) {
                     const int x = n0 + j * 32;
                     if (x < p.N && m0 < p.M) {
-                        if (p.accumulate) tma_reduce_add_2d(&map_out, staging_addr + sb * 16384, x, m0);
+                        if (add) tma_reduce_add_2d(&map_out, staging_addr + sb * 16384, x, m0);
                         else tma_store_2d(&map_out, staging_addr + sb * 16384, x, m0);
                     }
                     bulk_commit();
@@ -648,6 +689,8 @@ int g_bn_override = -1;   // tile width forced by SG_TC_BN or sg_set_tile_overri
 int g_cg_override = 0;    // CTAs per tile (0: automatic)
 int g_split_override = 0; // k ranges per tile (0: automatic)
 int g_kps_override = 0;   // SG_TC_KPS=1 (testing): one k-block per stage everywhere
+int g_last_sk[2] = {-1, 0};
+int g_sk_override = -1;   // SG_TC_SK (testing): 0 = never cut the last wave into a stream-K tail
 int g_ta_override = -1;   // SG_TC_TA (testing): 0 never, 1 always keep the split f32 input tile in tensor memory
 int g_last_choice[3] = {0, 0, 0};
 
@@ -790,6 +833,8 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         g_kps_override = e ? atoi(e) : 0;
         e = getenv("SG_TC_TA");
         g_ta_override = e ? atoi(e) : -1;
+        e = getenv("SG_TC_SK");
+        g_sk_override = e ? atoi(e) : -1;
     }
 
     alignas(64) CUtensorMap map_in, map_flt, map_out;
@@ -969,7 +1014,39 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         }
         tp.accumulate = 1;
     }
+    // Stream-K tail.  When whole tiles are dealt out and the last wave would be partly filled, the tiles of that wave
+    // are cut along k instead: every CTA (pair) gets an equal run of their k-blocks (whole stages), so the launch ends
+    // after tiles/groups waves' worth of k-blocks instead of ceil(tiles/groups).  The runs' partial sums meet in the
+    // output by reduce-add (an overwriting call clears those tiles first).  Taken when the k-blocks saved clearly
+    // outweigh the extra epilogues and the clearing launch (4096^3 f32 alone on the GPU: 498 -> 468 us; inside a step
+    // of concurrent launches the other launches fill the last wave anyway and nothing changes).
+    {
+        const Variant &v = kVariants[pick];
+        const int groups = g_drv.num_sms / v.cg;
+        const int num_m_tiles = (p.M + v.cg * BM - 1) / (v.cg * BM), num_n_tiles = (p.N + v.bn - 1) / v.bn;
+        const int64_t tiles = (int64_t)num_m_tiles * num_n_tiles;
+        const int left = (int)(tiles % groups);
+        if (g_sk_override != 0 && splits == 1 && tiles > groups && left != 0 && tp.num_kb % kps == 0) {
+            const int64_t units = (int64_t)left * tp.num_kb;
+            int run = (int)((units + groups - 1) / groups);
+            run = (run + kps - 1) / kps * kps;
+            const double kb_ns = f32 ? v.mma_ns_f32 : v.mma_ns;
+            const double saved = (double)(tp.num_kb - run) * kb_ns;
+            const double extra = 2.0 * (1500.0 + (double)v.bn * (f32 ? 24.0 : 12.0)) + 2500.0;
+            if (run >= 4 * kps && saved > 2.0 * extra) {
+                tp.sk_first_tile = (int)(tiles - left);
+                tp.sk_units = run;
+                if (!p.accumulate) {
+                    zero_tiles_kernel<<<left, 256, 0, stream>>>(O, p.o_w, p.M, p.N, v.cg * BM, v.bn, num_m_tiles, num_n_tiles, tp.sk_first_tile);
+                    count_launch();
+                    if (cudaGetLastError() != cudaSuccess) return SG_ERR_CUDA;
+                    tp.wait_prior = 1;
+                }
+            }
+        }
+    }
     g_last_choice[0] = kVariants[pick].bn; g_last_choice[1] = kVariants[pick].cg; g_last_choice[2] = splits;
+    g_last_sk[0] = tp.sk_units > 0 ? tp.sk_first_tile : -1; g_last_sk[1] = tp.sk_units;
     // f32, input stored [m][k] (the filter may be stored either way): the split input tile goes to tensor memory.  With
     // 256-column tiles that costs the second accumulator buffer, which short reductions used to feel; since the
     // converters stopped being the bottleneck the sweep is no slower with it everywhere (5.72 to 5.79 ms per step
@@ -1030,6 +1107,11 @@ bool tensor_encode_tiled(CUtensorMap *map, CUtensorMapDataType type, int rank, v
 void tensor_set_tile_override(int bn, int cg, int splits) {
     std::lock_guard<std::mutex> lock(g_mu);
     g_bn_override = bn; g_cg_override = cg; g_split_override = splits;
+}
+
+void tensor_last_stream_k(int out[2]) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    out[0] = g_last_sk[0]; out[1] = g_last_sk[1];
 }
 
 void tensor_last_choice(int out[3]) {

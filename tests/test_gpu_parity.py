@@ -699,3 +699,43 @@ def test_random_shapes_layouts_and_modes():
         acc = bool(rng.integers(0, 2))
         O, want, S = run_conv2d(N, Ho, Wo, C, KH, KW, F, st, dl, dtype, accumulate=acc, seed=SEED + case)
         assert_within_bound(O, want, S, f"random conv2d {case}: {N}x{Ho}x{Wo}x{C} {KH}x{KW} F={F} st={st} dl={dl} {dtype} acc={acc}")
+
+
+# Stream-K tail: more tiles than CTAs and a partly filled last wave, so the last tiles are cut along k into equal
+# runs (one per CTA or pair) whose partial sums meet by reduce-add.  Sampled rows across all tiles against the oracle.
+@pytest.mark.parametrize("accumulate", [False, True])
+@pytest.mark.parametrize("dtype,M,N,K,tile", [("f32", 2176, 1280, 2048, (128, 1)), ("f32", 2304, 2560, 1024, (256, 2)),
+                                              ("bf16", 2176, 1280, 8192, (128, 1)), ("f32", 2090, 1300, 2048, (128, 1))])
+def test_stream_k_tail(dtype, M, N, K, tile, accumulate):
+    A, a = operand((M, K), SEED, 31, "uniform", dtype)
+    B, b = operand((K, N), SEED, 32, "uniform", dtype)
+    if accumulate:
+        C, c0 = operand((M, N), SEED, 33, "uniform", "f32")
+        C = C.clone()
+    else:
+        C, c0 = torch.full((M, N), float("nan"), device="cuda"), None
+    sg.sg_set_tile_override(tile[0], tile[1], 1)
+    sg.sg_matmul(A, B, C, sg.SG_ACCUMULATE if accumulate else sg.SG_OVERWRITE)
+    torch.cuda.synchronize()
+    sg.sg_check()
+    first, run = sg.sg_last_stream_k()
+    assert first > 0 and run > 0, "this shape was meant to take the stream-K tail"
+    rows = np.unique(np.concatenate([np.arange(0, M, 37), np.arange(M - 130, M)]))
+    want, S = ref.matmul(a[rows], b, C_in=None if c0 is None else c0[rows])
+    if accumulate:
+        S = S + np.abs(c0[rows])
+    assert_within_bound(C[torch.from_numpy(rows).cuda()], want, S, f"stream-K tail {dtype} {M}x{N}x{K}")
+    assert not torch.isnan(C).any()
+
+
+def test_stream_k_tail_exact_on_integers():
+    M, N, K = 2176, 1280, 2048
+    A, a = operand((M, K), SEED, 34, "ints", "f32")
+    B, b = operand((K, N), SEED, 35, "ints", "f32")
+    C = torch.full((M, N), float("nan"), device="cuda")
+    sg.sg_set_tile_override(128, 1, 1)
+    sg.sg_matmul(A, B, C)
+    torch.cuda.synchronize()
+    assert sg.sg_last_stream_k()[1] > 0
+    want = (a.astype(np.float64) @ b.astype(np.float64))       # small integers: every partial sum is exact
+    assert np.array_equal(C.cpu().numpy().astype(np.float64), want)
