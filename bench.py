@@ -42,7 +42,7 @@ FLOPS_PER_STEP = 2 * FLOPS_PER_DTYPE
 
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture; None when the
 # kernel changed after the capture was taken.
-NCU_TRAFFIC_BYTES = 25.4e6   # profiles/bench_sweep_launch_list.md: average over the 125 f32 launches of a step
+NCU_TRAFFIC_BYTES = 25.6e6   # profiles/bench_sweep_launch_list.md: average over the 125 f32 launches of a step
 # tf32 : bf16 dense tensor throughput (nominal 1.1 : 2.25 PFLOP/s; the issue rate measured on
 # this chip is exactly half)
 TF32_OVER_BF16 = 0.5
