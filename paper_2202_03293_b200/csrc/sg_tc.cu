@@ -1,7 +1,8 @@
 // Tensor-core path for sm_100a: TMA -> swizzled shared memory -> tcgen05.mma -> TMEM -> TMA store.
 //
-// One persistent CTA per SM walks a static list of 128 x BN output tiles.  Inside a CTA
-// the work is split by warp role:
+// One persistent CTA per SM (or CTA pair per two SMs) walks a static list of work items: whole
+// output tiles, equal k ranges of a tile (split reduction), or its run of the stream-K tail that
+// replaces a partly filled last wave of tiles.  Inside a CTA the work is split by warp role:
 //
 //   warp 0  producer : per k-block waits for a free stage, then issues the TMA loads of the
 //                      input tile (tiled mode for matmul, im2col mode for the convolutions:
