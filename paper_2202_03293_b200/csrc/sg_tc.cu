@@ -691,7 +691,7 @@ int g_cg_override = 0;    // CTAs per tile (0: automatic)
 int g_split_override = 0; // k ranges per tile (0: automatic)
 int g_kps_override = 0;   // SG_TC_KPS=1 (testing): one k-block per stage everywhere
 int g_last_sk[2] = {-1, 0};
-int g_sk_override = -1;   // SG_TC_SK (testing): 0 = never cut the last wave into a stream-K tail
+int g_sk_override = -1;   // SG_TC_SK (testing): 0 = never cut the last wave into a stream-K tail, 2 = whenever it is possible
 int g_ta_override = -1;   // SG_TC_TA (testing): 0 never, 1 always keep the split f32 input tile in tensor memory
 int g_last_choice[3] = {0, 0, 0};
 
@@ -1034,7 +1034,7 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
             const double kb_ns = f32 ? v.mma_ns_f32 : v.mma_ns;
             const double saved = (double)(tp.num_kb - run) * kb_ns;
             const double extra = 2.0 * (1500.0 + (double)v.bn * (f32 ? 24.0 : 12.0)) + 2500.0;
-            if (run >= 4 * kps && saved > 2.0 * extra) {
+            if (run >= 4 * kps && (saved > 2.0 * extra || g_sk_override == 2)) {
                 tp.sk_first_tile = (int)(tiles - left);
                 tp.sk_units = run;
                 if (!p.accumulate) {
