@@ -175,7 +175,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                const __grid_constant__ CUtensorMap map_out, const TcParams p) {
     constexpr bool A_MN = (LAY & 1) != 0, B_KM = (LAY & 2) != 0, TA = (LAY & 4) != 0;
     using C = Cfg<BN, CG, F32, KPS, TA>;
-    static_assert(!TA || (F32 && !A_MN), "tensor-memory input operand: f32, input stored [m][k]");
+    static_assert(!TA || F32, "tensor-memory input operand: f32 path only");
     static_assert(LAY == 0 || KPS == 1, "transposed layouts: one k-block per stage");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -541,11 +541,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                         // input tile -> tensor memory: this warp may touch lane quarter (warp & 3); the four warps
                         // of a quarter take 8 of the 32 k columns each.  Lane = row reads its 32 bytes of the
                         // swizzled raw tile and stores 8 hi and 8 lo words.
-                        const int row = (warp & 3) * 32 + lane;
-                        const uint8_t *rp = raw + row * 128;
+                        if constexpr (A_MN) {
+                            // stored transposed: the raw tile is four [32 k][32 rows] sub-tiles (128-byte rows, not
+                            // swizzled); sub-tile (warp & 3) holds this warp's rows, lane = row reads its 8 k values
+                            // down a column (every load a whole 128-byte row across the warp)
+                            const float *col = reinterpret_cast<const float *>(raw) + (warp & 3) * (C::SUB_BYTES / 4) + (cw >> 2) * 8 * 32 + lane;
+                            a_raw[0] = make_uint4(__float_as_uint(col[0]), __float_as_uint(col[32]), __float_as_uint(col[64]), __float_as_uint(col[96]));
+                            a_raw[1] = make_uint4(__float_as_uint(col[128]), __float_as_uint(col[160]), __float_as_uint(col[192]), __float_as_uint(col[224]));
+                        } else {
+                            const int row = (warp & 3) * 32 + lane;
+                            const uint8_t *rp = raw + row * 128;
 #pragma unroll
-                        for (int i = 0; i < 2; ++i)
-                            a_raw[i] = *reinterpret_cast<const uint4 *>(rp + ((((cw >> 2) * 2 + i) ^ (row & 7)) << 4));
+                            for (int i = 0; i < 2; ++i)
+                                a_raw[i] = *reinterpret_cast<const uint4 *>(rp + ((((cw >> 2) * 2 + i) ^ (row & 7)) << 4));
+                        }
                     } else if constexpr (A_MN) {
                         split_transpose(raw, slot, slot + A_STAGE_BYTES, std::integral_constant<int, BM>{});
                     } else {
@@ -754,7 +763,7 @@ sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUt
                          int slot, cudaStream_t stream) {
   if constexpr ((F32 && BN == 256 && CG == 1) || (KPS == 2 && (F32 || (BN == 256 && CG == 1))) ||
                 ((LAY & 3) != 0 && (KPS != 1 || (BN == 256 && CG == 1) || (BN == 128 && CG == 2))) ||
-                ((LAY & 4) != 0 && (!F32 || (LAY & 1) != 0))) {
+                ((LAY & 4) != 0 && !F32)) {
     return SG_ERR_INTERNAL;   // the split slots of a 128 x 256 f32 tile do not fit beside a TMA ring
   } else {
     using C = Cfg<BN, CG, F32, KPS, (LAY & 4) != 0>;
@@ -1048,15 +1057,17 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     }
     g_last_choice[0] = kVariants[pick].bn; g_last_choice[1] = kVariants[pick].cg; g_last_choice[2] = splits;
     g_last_sk[0] = tp.sk_units > 0 ? tp.sk_first_tile : -1; g_last_sk[1] = tp.sk_units;
-    // f32, input stored [m][k] (the filter may be stored either way): the split input tile goes to tensor memory.  With
+    // f32 (either operand stored either way): the split input tile goes to tensor memory.  With
     // 256-column tiles that costs the second accumulator buffer, which short reductions used to feel; since the
     // converters stopped being the bottleneck the sweep is no slower with it everywhere (5.72 to 5.79 ms per step
     // either way), so there is one rule.
-    const int lay_k = (f32 && (lay & 1) == 0 && g_ta_override != 0) ? (lay | 4) : lay;
+    const int lay_k = (f32 && g_ta_override != 0) ? (lay | 4) : lay;
     const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0) + lay_k * 3 * kNumVariants;
 #define SG_LAUNCH(BN_, CG_)                                                                                \
     (f32 ? (lay_k == 4 ? launch_variant<BN_, CG_, true, 1, 4>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)     \
             : lay_k == 6 ? launch_variant<BN_, CG_, true, 1, 6>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)   \
+            : lay_k == 5 ? launch_variant<BN_, CG_, true, 1, 5>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)   \
+            : lay_k == 7 ? launch_variant<BN_, CG_, true, 1, 7>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)   \
             : lay == 0 ? launch_variant<BN_, CG_, true, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)         \
             : lay == 1 ? launch_variant<BN_, CG_, true, 1, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
             : lay == 2 ? launch_variant<BN_, CG_, true, 1, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
