@@ -739,3 +739,11 @@ def test_stream_k_tail_exact_on_integers():
     assert sg.sg_last_stream_k()[1] > 0
     want = (a.astype(np.float64) @ b.astype(np.float64))       # small integers: every partial sum is exact
     assert np.array_equal(C.cpu().numpy().astype(np.float64), want)
+
+
+def test_stream_k_tail_on_a_convolution():
+    # 4 x 72 x 72 output pixels = 162 row tiles of 128 on 148 SMs, 72 k-blocks (3 x 3 taps x 256 channels, f32)
+    sg.sg_set_tile_override(128, 1, 1)
+    O, want, S = run_conv2d(4, 72, 72, 256, 3, 3, 128, (1, 1), (1, 1), "f32", family=TENSOR)
+    assert sg.sg_last_stream_k()[1] > 0, "this shape was meant to take the stream-K tail"
+    assert_within_bound(O, want, S, "stream-K tail, conv2d f32")
