@@ -776,7 +776,8 @@ sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUt
     tp.num_n_tiles = (N + BN - 1) / BN;
     const int tiles = tp.num_m_tiles * tp.num_n_tiles * tp.splits;
     const int groups = g_drv.num_sms / CG;
-    const int grid = CG * (tiles < groups ? tiles : groups);
+    // (a stream-K tail deals its runs to every group, also when there are fewer tiles than groups)
+    const int grid = CG * ((tiles < groups && tp.sk_units == 0) ? tiles : groups);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
     cfg.blockDim = dim3(C::THREADS, 1, 1);
