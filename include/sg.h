@@ -19,14 +19,19 @@
  *     read only; the output is written (SG_OVERWRITE) or read and written
  *     (SG_ACCUMULATE).  The output must not overlap an input.
  *   - Strides are in ELEMENTS of the operand's type (the strided-buffer
- *     convention of the paper's memref type, Section 2.2), may be any
- *     positive value and need not be dense.
+ *     convention of the paper's memref type, Section 2.2) and need not be
+ *     dense.  Negative strides are rejected.  An input stride may be 0 (the
+ *     operand is broadcast along that dimension); an output stride of 0
+ *     along a dimension of extent > 1 is rejected (SG_ERR_INVALID_ARG): the
+ *     output's elements must be distinct.
  *   - `in_dtype` is the element type of BOTH inputs.  The output is always
  *     f32 and products are accumulated in f32 (bf16 inputs are widened
  *     exactly; f32 inputs keep f32 accuracy).
  *   - Calls only enqueue work on `stream` and return; they never synchronise
  *     and never allocate device memory.  The first call on a device creates
- *     small host-side state (driver entry points, a tensor-map cache).
+ *     small host-side state (driver entry points, kernel attributes); the
+ *     tensor-core paths keep a bounded, process-wide cache of encoded tensor
+ *     maps keyed by pointer, extents, strides and box (sg_shutdown drops it).
  *   - The return value reports argument and launch errors.  Device-side
  *     pipeline time-outs (which indicate a library bug, not a user error) are
  *     recorded in a per-device status word that sg_check() reads.
@@ -223,6 +228,16 @@ int sg_version(void);
 int sg_last_kernel(void);
 
 /*
+ * Name of the compute kernel that call launched (a static string, "" before any call; clearing
+ * kernels launched ahead of it are not named): "tc_gemm_kernel<bf16>", "tc_gemm_kernel<f32>",
+ * "conv_strip_kernel<bf16>", "conv_strip_kernel<f32>", "ffma_kernel", "depthwise_tma_kernel",
+ * "depthwise_roll_kernel", "depthwise_vec_kernel", "depthwise_generic_kernel", "copy_tma_kernel",
+ * "transpose_tma_kernel", "tile_move_kernel", "colred_kernel<vec>", "colred_kernel<scalar>",
+ * "rowred_kernel<vec>", "rowred_kernel<scalar>".  For tests and benchmarks.
+ */
+const char *sg_last_kernel_name(void);
+
+/*
  * Number of kernels this library has launched in this process so far
  * (monotonic, all threads).  Used by benchmarks to report launch counts.
  */
@@ -262,6 +277,25 @@ void sg_last_tile_choice(int out[3]);
  * environment (read at the first call) turns the tail off.
  */
 void sg_last_stream_k(int out[2]);
+
+/*
+ * Self-test of the device-side time-out path (the paper has no counterpart): launches one warp
+ * that waits `budget_cycles` SM clock cycles (1e3 .. 2e7, i.e. at most about 10 ms) on a barrier
+ * that nothing signals, then gives up exactly as a pipeline wait of the kernels above would: it
+ * sets the device status word and returns normally.  The next sg_check() on that device reports
+ * SG_ERR_DEVICE_TIMEOUT once and clears the word.  Nothing traps and nothing spins past the budget.
+ */
+sg_status sg_selftest_wait_timeout(int64_t budget_cycles, sg_stream_t stream);
+
+/*
+ * Environment switches, all for testing and benchmarking, all read once at the first tensor-core
+ * call of the process:
+ *   SG_TC_BN, SG_TC_CG, SG_TC_SPLIT   as sg_set_tile_override
+ *   SG_TC_SK        0: never cut the last wave into a stream-K tail; 2: whenever the shape allows it
+ *   SG_TC_KPS       1: one k-block per pipeline stage everywhere (bf16 matmuls normally move two)
+ *   SG_TC_TA        0: keep the split f32 input tile in shared memory instead of tensor memory
+ *   SG_CONV_SINGLE  1: the stride-1 convolution kernel never uses CTA pairs
+ */
 
 /* Drops cached tensor maps and other host-side state.  Safe to call twice. */
 void sg_shutdown(void);

@@ -41,6 +41,8 @@
 #include <stdint.h>
 #include <stddef.h>
 #include <math.h>
+
+#include "sg_ref.h"    /* the declarations of everything below: the compiler checks that they agree */
 #ifdef _OPENMP
 #include <omp.h>
 #endif

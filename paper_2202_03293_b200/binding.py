@@ -25,7 +25,7 @@ EXPORTS = [
     "sg_matmul", "sg_conv1d_nwc_wcf", "sg_conv2d_nhwc_hwcf", "sg_depthwise_conv1d_nwc_wc",
     "sg_depthwise_conv2d_nhwc_hwc", "sg_copy2d", "sg_transpose2d", "sg_colred2d", "sg_rowred2d", "sg_check", "sg_status_string",
     "sg_version", "sg_last_kernel", "sg_launch_count", "sg_set_kernel_override", "sg_set_tile_override",
-    "sg_last_tile_choice", "sg_last_stream_k", "sg_shutdown",
+    "sg_last_tile_choice", "sg_last_stream_k", "sg_shutdown", "sg_last_kernel_name", "sg_selftest_wait_timeout",
 ]
 
 
@@ -77,6 +77,9 @@ def lib() -> ctypes.CDLL:
         L.sg_last_stream_k.argtypes = [ctypes.POINTER(ctypes.c_int)]
         L.sg_last_stream_k.restype = None
         L.sg_shutdown.restype = None
+        L.sg_last_kernel_name.restype = ctypes.c_char_p
+        L.sg_selftest_wait_timeout.argtypes = [i64, vp]
+        L.sg_selftest_wait_timeout.restype = ci
         _lib = L
     return _lib
 
@@ -275,3 +278,13 @@ def sg_last_stream_k():
 
 def sg_shutdown() -> None:
     lib().sg_shutdown()
+
+
+def sg_last_kernel_name() -> str:
+    return lib().sg_last_kernel_name().decode()
+
+
+def sg_selftest_wait_timeout(budget_cycles: int = 2_000_000, stream=None) -> None:
+    rc = lib().sg_selftest_wait_timeout(int(budget_cycles), _stream(stream))
+    if rc != SG_OK:
+        raise SgError(rc, "sg_selftest_wait_timeout")

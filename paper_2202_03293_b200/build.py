@@ -1,18 +1,24 @@
-"""Builds libsg.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a."""
+"""Builds libsg.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
+
+Every .cu file is its own translation unit (no relocatable device code), so the files are
+compiled side by side into objects under csrc/_build/ and linked into one shared library.
+"""
 from __future__ import annotations
 
 import glob
 import os
 import subprocess
+from concurrent.futures import ThreadPoolExecutor
 
 PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
+OBJ = os.path.join(CSRC, "_build")
 LIB = os.path.join(PKG, "libsg.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v",
+    "-Xcompiler", "-fPIC", "-Xptxas", "-v",
 ]
 
 
@@ -20,26 +26,53 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def headers():
+    return glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
+
+
+def _stale(target: str, deps) -> bool:
+    if not os.path.exists(target):
         return True
-    t = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
+    t = os.path.getmtime(target)
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+def needs_build() -> bool:
+    return _stale(LIB, sources() + headers())
+
+
 def build_library(force: bool = False, verbose: bool = False) -> str:
-    if force or needs_build():
-        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        cmd = [nvcc] + NVCC_FLAGS + ["-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB] + sources()
-        res = subprocess.run(cmd, capture_output=True, text=True)
-        if verbose or res.returncode != 0:
-            print(res.stdout)
-            print(res.stderr)
-        if res.returncode != 0:
-            raise RuntimeError("nvcc failed building libsg.so")
+    if not (force or needs_build()):
+        return LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    os.makedirs(OBJ, exist_ok=True)
+    inc = ["-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    hdrs = headers()
+
+    def compile_one(src):
+        obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
+        if not force and not _stale(obj, [src] + hdrs):
+            return obj, 0, ""
+        res = subprocess.run([nvcc] + NVCC_FLAGS + inc + ["-c", src, "-o", obj], capture_output=True, text=True)
+        return obj, res.returncode, res.stdout + res.stderr
+
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        results = list(pool.map(compile_one, sources()))
+    failed = [r for r in results if r[1] != 0]
+    for obj, rc, log in results:
+        if log and (verbose or rc != 0):
+            print(log)
+    if failed:
+        raise RuntimeError("nvcc failed building libsg.so")
+    res = subprocess.run([nvcc, "-shared", "-Xcompiler", "-fPIC", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB] +
+                         [r[0] for r in results], capture_output=True, text=True)
+    if verbose or res.returncode != 0:
+        print(res.stdout + res.stderr)
+    if res.returncode != 0:
+        raise RuntimeError("linking libsg.so failed")
     return LIB
 
 
 if __name__ == "__main__":
-    build_library(force=True, verbose=True)
+    import sys
+    build_library(force="--incremental" not in sys.argv, verbose=True)

@@ -10,6 +10,7 @@ namespace {
 std::atomic<int64_t> g_launches{0};
 std::atomic<int> g_override{SG_KERNEL_AUTO};
 thread_local int t_last_kernel = 0;
+thread_local const char *t_last_kernel_name = "";
 
 constexpr int64_t kMaxDim = std::numeric_limits<int32_t>::max();
 
@@ -52,6 +53,7 @@ sg_status check_common(const void *a, const void *b, const void *o, sg_dtype dt,
 }  // namespace
 
 void count_launch(int n) { g_launches.fetch_add(n); }
+void note_kernel(const char *name) { t_last_kernel_name = name; }
 
 }  // namespace sg
 
@@ -71,6 +73,7 @@ sg_status sg_matmul(int64_t M, int64_t N, int64_t K, const void *A, int64_t a_st
     if (has_out && K > 0 && (!A || !B)) return SG_ERR_INVALID_ARG;
     if (a_stride_m < 0 || a_stride_k < 0 || b_stride_k < 0 || b_stride_n < 0 || c_stride_m < 0 || c_stride_n < 0)
         return SG_ERR_INVALID_ARG;
+    if ((M > 1 && c_stride_m == 0) || (N > 1 && c_stride_n == 0)) return SG_ERR_INVALID_ARG;   // output elements would coincide
     Problem p{};
     p.M = (int)M; p.N = (int)N; p.K = (int)K;
     p.batch = 1; p.Ho = 1; p.Wo = (int)M;
@@ -95,6 +98,7 @@ sg_status sg_conv1d_nwc_wcf(int64_t N, int64_t W_out, int64_t F, int64_t KW, int
     if (st != SG_OK) return st;
     for (int i = 0; i < 3; ++i)
         if (i_strides[i] < 0 || k_strides[i] < 0 || o_strides[i] < 0) return SG_ERR_INVALID_ARG;
+    if ((N > 1 && o_strides[0] == 0) || (W_out > 1 && o_strides[1] == 0) || (F > 1 && o_strides[2] == 0)) return SG_ERR_INVALID_ARG;
     if (!fits(N) || !fits(W_out) || !fits(F) || !fits(KW) || !fits(C) || !fits(W_in) || !fits(stride_w) ||
         !fits(dilation_w)) return SG_ERR_UNSUPPORTED;
     if (W_out > 0 && KW > 0 && W_in < (W_out - 1) * stride_w + (KW - 1) * dilation_w + 1) return SG_ERR_INVALID_ARG;
@@ -128,6 +132,8 @@ sg_status sg_conv2d_nhwc_hwcf(int64_t N, int64_t H_out, int64_t W_out, int64_t F
     if (st != SG_OK) return st;
     for (int i = 0; i < 4; ++i)
         if (i_strides[i] < 0 || k_strides[i] < 0 || o_strides[i] < 0) return SG_ERR_INVALID_ARG;
+    if ((N > 1 && o_strides[0] == 0) || (H_out > 1 && o_strides[1] == 0) || (W_out > 1 && o_strides[2] == 0) ||
+        (F > 1 && o_strides[3] == 0)) return SG_ERR_INVALID_ARG;
     if (!fits(N) || !fits(H_out) || !fits(W_out) || !fits(F) || !fits(KH) || !fits(KW) || !fits(C) || !fits(H_in) ||
         !fits(W_in) || !fits(stride_h) || !fits(stride_w) || !fits(dilation_h) || !fits(dilation_w))
         return SG_ERR_UNSUPPORTED;
@@ -163,6 +169,8 @@ sg_status sg_depthwise_conv2d_nhwc_hwc(int64_t N, int64_t H_out, int64_t W_out, 
     if (st != SG_OK) return st;
     for (int i = 0; i < 4; ++i)
         if (i_strides[i] < 0 || o_strides[i] < 0 || (i < 3 && k_strides[i] < 0)) return SG_ERR_INVALID_ARG;
+    if ((N > 1 && o_strides[0] == 0) || (H_out > 1 && o_strides[1] == 0) || (W_out > 1 && o_strides[2] == 0) ||
+        (C > 1 && o_strides[3] == 0)) return SG_ERR_INVALID_ARG;
     if (!fits(N) || !fits(H_out) || !fits(W_out) || !fits(C) || !fits(KH) || !fits(KW) || !fits(H_in) || !fits(W_in) ||
         !fits(stride_h) || !fits(stride_w) || !fits(dilation_h) || !fits(dilation_w)) return SG_ERR_UNSUPPORTED;
     if (H_out > 0 && KH > 0 && H_in < (H_out - 1) * stride_h + (KH - 1) * dilation_h + 1) return SG_ERR_INVALID_ARG;
@@ -190,7 +198,7 @@ sg_status sg_depthwise_conv1d_nwc_wc(int64_t N, int64_t W_out, int64_t C, int64_
                                      const int64_t k_strides[2], float *O, const int64_t o_strides[3], sg_dtype in_dtype,
                                      int mode, sg_stream_t stream) {
     if (!i_strides || !k_strides || !o_strides) return SG_ERR_INVALID_ARG;
-    // the 2-D op with H = KH = 1 (Section 4.6.3: "K_h and H are 1 in the 1-D case")
+    // the 1-D op is the 2-D op with H = KH = 1 (Section 4.6.3)
     const int64_t is4[4] = {i_strides[0], 0, i_strides[1], i_strides[2]};
     const int64_t ks3[3] = {0, k_strides[0], k_strides[1]};
     const int64_t os4[4] = {o_strides[0], 0, o_strides[1], o_strides[2]};
@@ -207,6 +215,8 @@ sg_status move2d(bool transpose, int64_t R, int64_t C, const void *src, int64_t 
     if (!fits(R + kTileSlack) || !fits(C + kTileSlack)) return SG_ERR_UNSUPPORTED;   // tile coordinates stay in int32
     if (R == 0 || C == 0) return SG_OK;
     if (!src || !dst) return SG_ERR_INVALID_ARG;
+    // destination elements must not coincide (dst is R x C for a copy, C x R for a transpose)
+    if (((transpose ? C : R) > 1 && d_r == 0) || ((transpose ? R : C) > 1 && d_c == 0)) return SG_ERR_INVALID_ARG;
     const int es = dtype == SG_BF16 ? 2 : 4;
     if (reinterpret_cast<uintptr_t>(src) % es || reinterpret_cast<uintptr_t>(dst) % es) return SG_ERR_ALIGNMENT;
     const int ov = g_override.load();
@@ -227,6 +237,7 @@ sg_status reduce2d(bool colred, int64_t R, int64_t C, const void *A, int64_t a_r
     const int64_t n_out = colred ? C : R, n_red = colred ? R : C;
     if (n_out == 0) return SG_OK;
     if (!out || (n_red > 0 && !A)) return SG_ERR_INVALID_ARG;
+    if (n_out > 1 && out_stride == 0) return SG_ERR_INVALID_ARG;      // output elements would coincide
     if (n_red == 0 && mode == SG_ACCUMULATE) return SG_OK;
     st = launch_reduce2d(colred, R, C, A, a_r, a_c, in_dtype == SG_BF16, out, out_stride, mode == SG_ACCUMULATE,
                          static_cast<cudaStream_t>(stream));
@@ -278,6 +289,8 @@ int sg_version(void) { return 200; }   // 0.2.0: depthwise convolutions and the 
 
 int sg_last_kernel(void) { return t_last_kernel; }
 
+const char *sg_last_kernel_name(void) { return t_last_kernel_name; }
+
 int64_t sg_launch_count(void) { return g_launches.load(); }
 
 sg_status sg_set_kernel_override(int kernel_family) {
@@ -299,7 +312,14 @@ void sg_last_tile_choice(int out[3]) {
     if (out) tensor_last_choice(out);
 }
 
-void sg_last_stream_k(int out[2]) { sg::tensor_last_stream_k(out); }
+void sg_last_stream_k(int out[2]) {
+    if (out) sg::tensor_last_stream_k(out);
+}
+
+sg_status sg_selftest_wait_timeout(int64_t budget_cycles, sg_stream_t stream) {
+    if (budget_cycles < 1000 || budget_cycles > 20000000) return SG_ERR_INVALID_ARG;    // at most ~10 ms of spinning
+    return launch_wait_timeout_selftest((long long)budget_cycles, static_cast<cudaStream_t>(stream)) == cudaSuccess ? SG_OK : SG_ERR_CUDA;
+}
 
 void sg_shutdown(void) { tensor_shutdown(); }
 

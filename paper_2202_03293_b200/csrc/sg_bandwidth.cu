@@ -507,6 +507,7 @@ cudaError_t launch_reduce_typed(bool colred, const T *A, int64_t ld, int64_t sc,
         const cudaError_t e = launch_reduction(rowred_kernel<T, VEC>, dim3((unsigned)row_ctas, (unsigned)splits), use_atomic && !accumulate, stream,
                                                A, ld, sc, R, C, out, os, lanes, chunks_per_split * VEC, use_atomic, accumulate);
         count_launch();
+        note_kernel(VEC > 1 ? "rowred_kernel<vec>" : "rowred_kernel<scalar>");
         return e;
     } else {
         // ColRed2D: one output per column
@@ -538,13 +539,14 @@ cudaError_t launch_reduce_typed(bool colred, const T *A, int64_t ld, int64_t sc,
         const cudaError_t e = launch_reduction(colred_kernel<T, VEC>, dim3((unsigned)col_blocks, (unsigned)splits), use_atomic && !accumulate, stream,
                                                A, ld, sc, R, C, out, os, cw, rp, rows_per_split, use_atomic, accumulate);
         count_launch();
+        note_kernel(VEC > 1 ? "colred_kernel<vec>" : "colred_kernel<scalar>");
         return e;
     }
 }
 
 template <typename U>
 cudaError_t launch_tile_move(const U *src, int64_t s_i, int64_t s_j, U *dst, int64_t d_i, int64_t d_j, int R, int C, int num_sms,
-                             cudaStream_t stream) {
+                             cudaStream_t stream, bool note = true) {
     const int tiles_j = (C + 31) / 32;
     const int64_t num_tiles = (int64_t)((R + 31) / 32) * tiles_j;
     const int grid = (int)std::min<int64_t>(num_tiles, (int64_t)num_sms * 8);
@@ -552,6 +554,7 @@ cudaError_t launch_tile_move(const U *src, int64_t s_i, int64_t s_j, U *dst, int
     if (d_i < d_j) tile_move_kernel<U, true><<<grid, 256, 0, stream>>>(src, s_i, s_j, dst, d_i, d_j, R, C, tiles_j, num_tiles);
     else tile_move_kernel<U, false><<<grid, 256, 0, stream>>>(src, s_i, s_j, dst, d_i, d_j, R, C, tiles_j, num_tiles);
     count_launch();
+    if (note) note_kernel("tile_move_kernel");
     return cudaGetLastError();
 }
 
@@ -634,6 +637,7 @@ sg_status launch_move2d(bool transpose, int64_t R, int64_t C, const void *src, i
         }
         if (launched) {
             count_launch();
+            note_kernel(transpose ? "transpose_tma_kernel" : "copy_tma_kernel");
             *used_tma = 1;
             if (cudaGetLastError() != cudaSuccess) return SG_ERR_CUDA;
             if (tail == 0) return SG_OK;
@@ -643,8 +647,8 @@ sg_status launch_move2d(bool transpose, int64_t R, int64_t C, const void *src, i
             const int64_t Rt = transpose ? tail : R, Ct = transpose ? C : tail;
             const int64_t di = transpose ? d_c : d_r, dj = transpose ? d_r : d_c;
             const cudaError_t e = esize == 4
-                ? launch_tile_move(reinterpret_cast<const uint32_t *>(s_tail), s_r, s_c, reinterpret_cast<uint32_t *>(d_tail), di, dj, (int)Rt, (int)Ct, num_sms, stream)
-                : launch_tile_move(reinterpret_cast<const uint16_t *>(s_tail), s_r, s_c, reinterpret_cast<uint16_t *>(d_tail), di, dj, (int)Rt, (int)Ct, num_sms, stream);
+                ? launch_tile_move(reinterpret_cast<const uint32_t *>(s_tail), s_r, s_c, reinterpret_cast<uint32_t *>(d_tail), di, dj, (int)Rt, (int)Ct, num_sms, stream, false)
+                : launch_tile_move(reinterpret_cast<const uint16_t *>(s_tail), s_r, s_c, reinterpret_cast<uint16_t *>(d_tail), di, dj, (int)Rt, (int)Ct, num_sms, stream, false);
             return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
         }
     }

@@ -461,6 +461,7 @@ sg_status launch_conv_strip(const Problem &p, const void *In, const void *Flt, f
     cfg.numAttrs = 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, map_in, map_flt, cp);
     count_launch();
+    note_kernel("conv_strip_kernel");
     return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
 }
 

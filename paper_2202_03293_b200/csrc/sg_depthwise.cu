@@ -391,6 +391,7 @@ bool try_launch_tma(const DepthwiseProblem &p, const T *I, const T *Kf, float *O
     grid -= grid % c_blocks;
     depthwise_tma_kernel<T, CB, S><<<(int)grid, DT_THREADS, smem, stream>>>(map_in, p, Kf, O, tiles_w, tiles_h, c_blocks, (int)tiles);
     count_launch();
+    note_kernel("depthwise_tma_kernel");
     *err = cudaGetLastError();
     return true;
 }
@@ -429,6 +430,7 @@ cudaError_t launch_typed(const DepthwiseProblem &p, const T *I, const T *Kf, flo
         if (items >= (int64_t)148 * 256 * 2 && items < ((int64_t)1 << 32) - 256 && 9 * p.C * 4 <= 48 * 1024) {
             depthwise_roll_kernel<T><<<(unsigned)((items + ROLL_BLOCK - 1) / ROLL_BLOCK), ROLL_BLOCK, 9 * p.C * 4, stream>>>(p, I, Kf, O);
             count_launch();
+            note_kernel("depthwise_roll_kernel");
             return cudaGetLastError();
         }
     }
@@ -438,6 +440,7 @@ cudaError_t launch_typed(const DepthwiseProblem &p, const T *I, const T *Kf, flo
     else { if (small) SG_DW((depthwise_generic_kernel<T, uint32_t>)); else SG_DW((depthwise_generic_kernel<T, uint64_t>)); }
 #undef SG_DW
     count_launch();
+    note_kernel(vec ? "depthwise_vec_kernel" : "depthwise_generic_kernel");
     return cudaGetLastError();
 }
 

@@ -250,6 +250,7 @@ cudaError_t launch_typed(const Problem &p, const T *In, const T *Flt, float *O, 
     else if (vec_b) ffma_kernel<T, false, true><<<grid, THREADS, 0, stream>>>(p, In, Flt, O, vec_c);
     else ffma_kernel<T, false, false><<<grid, THREADS, 0, stream>>>(p, In, Flt, O, vec_c);
     count_launch();
+    note_kernel("ffma_kernel");
     return cudaGetLastError();
 }
 

@@ -41,6 +41,8 @@ cudaError_t launch_zero_fill(const Problem &p, float *O, cudaStream_t stream);
 sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float *O,
                         cudaStream_t stream);
 void tensor_shutdown();
+// One warp that waits `budget_cycles` on a barrier nobody signals, then reports the time-out like any pipeline wait.
+cudaError_t launch_wait_timeout_selftest(long long budget_cycles, cudaStream_t stream);
 // Driver entry points resolved by the tensor path, for the other tensor-core kernels: whether the
 // current device is usable (and its SM count), and a tiled tensor-map encoder (interleave none,
 // element strides 1, out-of-bounds elements read as zero).  Call with no library lock held.
@@ -82,5 +84,7 @@ sg_status launch_reduce2d(bool colred, int64_t R, int64_t C, const void *A, int6
 sg_status bandwidth_read_status(cudaStream_t stream);
 
 void count_launch(int n = 1);
+// Records the name of the compute kernel a call launched (a static string), for sg_last_kernel_name().
+void note_kernel(const char *name);
 
 }  // namespace sg

@@ -676,6 +676,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     }
 }
 
+// Self-test of the time-out path: one warp waits, with a short budget, on an mbarrier that nothing ever signals, gives
+// up the way the pipelines above do (abort flag, status bit) and returns normally.
+__global__ void __launch_bounds__(32) wait_timeout_selftest_kernel(long long budget_cycles) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0, &abort_flag, budget_cycles);
+    __syncwarp();
+}
+
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -794,6 +809,7 @@ sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUt
     cfg.numAttrs = tp.wait_prior ? 2 : 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, tc_gemm_kernel<BN, CG, F32, KPS, LAY>, mi, mf, mo, tp);
     count_launch();
+    note_kernel(F32 ? "tc_gemm_kernel<f32>" : "tc_gemm_kernel<bf16>");
     return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
   }
 }
@@ -925,18 +941,27 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     if (pick >= 0) {
         splits = g_split_override > 0 && valid_split(g_split_override) ? g_split_override : 1;
     } else {
+        // A forced split is taken as given when it fits the reduction (every range non-empty), with the variant that
+        // is cheapest for it; one that does not fit is ignored and the estimate chooses the split as well.
+        const int forced = g_split_override > 0 && valid_split(g_split_override) ? g_split_override : 0;
         double best = 1e300;
+        // (a forced pair count that no variant can honour on this shape is dropped in a second pass)
+        for (int pass = 0; pass < 2 && pick < 0; ++pass)
         for (int i = 0; i < kNumVariants; ++i) {
             const Variant &v = kVariants[i];
-            if (g_cg_override > 0 && v.cg != g_cg_override && !(v.cg == 1 && p.M <= BM)) continue;
+            if (pass == 0 && g_cg_override > 0 && v.cg != g_cg_override && !(v.cg == 1 && p.M <= BM)) continue;
             if (f32 && v.bn == 256 && v.cg == 1) continue;       // not built (shared-memory budget)
             if (lay != 0 && ((v.bn == 256 && v.cg == 1) || (v.bn == 128 && v.cg == 2))) continue;   // not built for transposed operands
             if (v.bn > 64 && v.bn / 2 >= p.N) continue;          // at most half of the tile would be used
             if (v.cg == 2 && p.M <= BM) continue;                // the second CTA would have no rows
             const int64_t tiles = (int64_t)((p.M + v.cg * BM - 1) / (v.cg * BM)) * ((p.N + v.bn - 1) / v.bn);
             const int64_t groups = g_drv.num_sms / v.cg;
+            if (forced) {
+                const double c = estimate_ns(v, f32, tiles, groups, tp.num_kb, forced, p.accumulate != 0);
+                if (c < best) { best = c; pick = i; splits = forced; }
+                continue;
+            }
             for (int sp = 1; sp <= 32; sp *= 2) {
-                if (g_split_override > 0 && sp != g_split_override) continue;
                 if (!valid_split(sp)) break;
                 if (sp > 1 && tiles * (sp / 2) >= 2 * groups) break;   // already two waves without this split
                 const double c = estimate_ns(v, f32, tiles, groups, tp.num_kb, sp, p.accumulate != 0);
@@ -1094,6 +1119,12 @@ sg_status tensor_read_status(cudaStream_t stream) {
     const sg_status c = bandwidth_read_status(stream);
     const sg_status d = depthwise_read_status(stream);
     return a != SG_OK ? a : (b != SG_OK ? b : (c != SG_OK ? c : d));
+}
+
+cudaError_t launch_wait_timeout_selftest(long long budget_cycles, cudaStream_t stream) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(budget_cycles);
+    count_launch();
+    return cudaGetLastError();
 }
 
 bool tensor_driver_ready(int *num_sms) {

@@ -52,9 +52,10 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the budget expired or another role already aborted.
+// Bounded wait.  Returns false when the budget (in SM clock cycles) expired or another role already aborted.
 template <bool CLUSTER_SCOPE = false>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          long long budget_cycles = WAIT_BUDGET_CYCLES) {
     auto test = [&]() { return CLUSTER_SCOPE ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
     if (test()) return true;
     const long long t0 = clock64();
@@ -62,7 +63,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (test()) return true;
         if ((it & 63u) == 63u) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_BUDGET_CYCLES) {
+            if (clock64() - t0 > budget_cycles) {
                 *abort_flag = 1;
                 atomicOr(&g_status_word, 1u);
                 return false;

@@ -67,6 +67,38 @@ def test_argument_validation_needs_no_gpu(lib):
     assert c2(1, 4, 0, 2, 3, 3, 2, 6, 6, 1, 1, 1, 1, null, i4, null, i4, null, i4, 1, 0, null) == 0
     assert lib.sg_set_kernel_override(9) == 1
     assert lib.sg_set_kernel_override(0) == 0
+    # an output stride of 0 along a dimension with more than one element: the elements would coincide
+    assert mm(4, 4, 4, fake, 4, 1, fake, 4, 1, fake, 0, 1, 0, 0, null) == 1
+    assert mm(4, 4, 4, fake, 4, 1, fake, 4, 1, fake, 4, 0, 0, 0, null) == 1
+    o3 = (ctypes.c_int64 * 3)(1, 0, 1)
+    assert c1(1, 8, 4, 3, 4, 10, 1, 1, fake, i3, fake, i3, fake, o3, 0, 0, null) == 1
+    o4 = (ctypes.c_int64 * 4)(1, 1, 1, 0)
+    assert c2(1, 4, 4, 2, 3, 3, 2, 6, 6, 1, 1, 1, 1, fake, i4, fake, i4, fake, o4, 1, 0, null) == 1
+    assert lib.sg_copy2d(4, 4, fake, 4, 1, fake, 0, 1, 0, null) == 1
+    assert lib.sg_transpose2d(4, 4, fake, 4, 1, fake, 4, 0, 0, null) == 1
+    assert lib.sg_colred2d(4, 4, fake, 4, 1, fake, 0, 0, 0, null) == 1
+    assert lib.sg_rowred2d(4, 1, fake, 4, 1, fake, 0, 0, 0, null) == 1
+    # the time-out self-test takes a bounded budget only
+    assert lib.sg_selftest_wait_timeout(0, null) == 1
+    assert lib.sg_selftest_wait_timeout(10 ** 9, null) == 1
+    # null result pointers are ignored
+    lib.sg_last_stream_k(None)
+    lib.sg_last_tile_choice(None)
+    assert binding.sg_last_kernel_name() == ""
+
+
+def test_oracle_header_and_library_agree():
+    """oracle/sg_ref.h declares the reference counterparts of the entry points; libsgref.so exports each of them."""
+    from oracle import ref
+    text = open(os.path.join(ROOT, "oracle", "sg_ref.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    syms = sorted(set(re.findall(r"\b(sg_ref_[a-z0-9_]+)\s*\(", text)))
+    assert {"sg_ref_matmul", "sg_ref_conv1d_nwc_wcf", "sg_ref_conv2d_nhwc_hwcf"} <= set(syms)
+    L = ref.lib()
+    for s in syms:
+        assert hasattr(L, s), f"libsgref.so does not export {s}"
+    # and the product's header does not mention the oracle
+    assert "sg_ref" not in open(os.path.join(ROOT, "include", "sg.h")).read()
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

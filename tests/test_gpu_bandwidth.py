@@ -257,3 +257,36 @@ def test_random_shapes_and_pitches():
         op = str(rng.choice(["col", "row"]))
         pitch = up8(C) if rng.integers(0, 2) else C + int(rng.integers(0, 5))
         run_reduce(op, R, C, dtype, accumulate=bool(rng.integers(0, 2)), pitch=pitch)
+
+
+def test_bandwidth_kernel_selection():
+    """sg_last_kernel_name names the exact kernel: TMA movers for aligned layouts, the strided mover otherwise; the
+    vector or the scalar form of each reduction."""
+    src = torch.zeros((256, 512), device="cuda")
+    sg.sg_copy2d(src, torch.empty_like(src))
+    assert sg.sg_last_kernel_name() == "copy_tma_kernel"
+    sg.sg_transpose2d(src, torch.empty((512, 256), device="cuda"))
+    assert sg.sg_last_kernel_name() == "transpose_tma_kernel"
+    odd = torch.zeros((255, 511), device="cuda")
+    sg.sg_copy2d(odd, torch.empty_like(odd))                 # pitch of 511 floats: not a multiple of 16 bytes
+    assert sg.sg_last_kernel_name() == "tile_move_kernel"
+    sg.sg_transpose2d(src.t(), torch.empty((256, 512), device="cuda"))     # column-major source
+    assert sg.sg_last_kernel_name() == "tile_move_kernel"
+    for dt in (torch.float32, torch.bfloat16):
+        A = torch.ones((300, 512), device="cuda", dtype=dt)
+        out_c, out_r = torch.empty(512, device="cuda"), torch.empty(300, device="cuda")
+        sg.sg_colred2d(A, out_c)
+        assert sg.sg_last_kernel_name() == "colred_kernel<vec>"
+        sg.sg_rowred2d(A, out_r)
+        assert sg.sg_last_kernel_name() == "rowred_kernel<vec>"
+        torch.cuda.synchronize()
+        assert torch.all(out_c == 300) and torch.all(out_r == 512)
+        B = torch.ones((300, 515), device="cuda", dtype=dt)[:, 1:514]       # unaligned base and pitch
+        out_c = torch.empty(513, device="cuda")
+        sg.sg_colred2d(B, out_c)
+        assert sg.sg_last_kernel_name() == "colred_kernel<scalar>"
+        sg.sg_rowred2d(B, out_r)
+        assert sg.sg_last_kernel_name() == "rowred_kernel<scalar>"
+        torch.cuda.synchronize()
+        assert torch.all(out_c == 300) and torch.all(out_r == 513)
+    sg.sg_check()

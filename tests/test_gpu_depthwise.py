@@ -135,3 +135,37 @@ def test_depthwise_conv2d_tiled_channel_slice(dtype):
     want, S = ref.depthwise_conv2d_nhwc_hwc(np.ascontiguousarray(i[..., 8:72]), k)
     assert_within_bound(Obig[..., 4:68], want, S, "channel slice, tiled")
     assert torch.all(torch.isnan(Obig[..., :4])) and torch.all(torch.isnan(Obig[..., 68:]))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_depthwise_kernel_selection(dtype):
+    """Which of the four depthwise kernels takes a shape (sg_last_kernel_name names the exact kernel)."""
+    # 3 x 3, stride 1 or 2, aligned NHWC, at least one tile per SM: whole input tiles staged by TMA
+    for st in (1, 2):
+        O, want, S = run2d(32, 112, 112, 64, 3, 3, (st, st), (1, 1), dtype)
+        assert sg.sg_last_kernel_name() == "depthwise_tma_kernel"
+        assert_within_bound(O, want, S, "tma kernel")
+    # the same walk down the rows with ordinary loads, for layouts outside the TMA rules: a bf16 channel slice whose
+    # base is 8-byte but not 16-byte aligned (f32 vector loads need 16 bytes themselves, so only bf16 gets here)
+    if dtype == "bf16":
+        N, Ho, Wo, C = 16, 100, 100, 64
+        Ibig, i = operand((N, Ho + 2, Wo + 2, 72), SEED, 30, "normal", dtype)
+        K, k = operand((3, 3, C), SEED, 31, "normal", dtype)
+        O = torch.full((N, Ho, Wo, C), float("nan"), device="cuda")
+        sg.sg_depthwise_conv2d_nhwc_hwc(Ibig[..., 4:68], K, O)       # base offset 8 bytes
+        torch.cuda.synchronize()
+        assert sg.sg_last_kernel_name() == "depthwise_roll_kernel"
+        want, S = ref.depthwise_conv2d_nhwc_hwc(np.ascontiguousarray(i[..., 4:68]), k)
+        assert_within_bound(O, want, S, "rolling-window kernel")
+    # too few tiles for the tiled kernels, or a window / dilation they do not take: four channels x four columns per thread
+    O, want, S = run2d(1, 7, 7, 1024, 3, 3, (1, 1), (1, 1), dtype)
+    assert sg.sg_last_kernel_name() == "depthwise_vec_kernel"
+    assert_within_bound(O, want, S, "vec kernel, 3x3")
+    O, want, S = run2d(2, 20, 21, 64, 5, 5, (2, 2), (2, 2), dtype)
+    assert sg.sg_last_kernel_name() == "depthwise_vec_kernel"
+    assert_within_bound(O, want, S, "vec kernel, 5x5 dilated")
+    # channels not a multiple of 4: one element per thread
+    O, want, S = run2d(2, 9, 10, 7, 3, 3, (1, 1), (1, 1), dtype)
+    assert sg.sg_last_kernel_name() == "depthwise_generic_kernel"
+    assert_within_bound(O, want, S, "generic kernel")
+    assert sg.sg_last_kernel() == sg.SG_KERNEL_FFMA

@@ -747,3 +747,132 @@ def test_stream_k_tail_on_a_convolution():
     O, want, S = run_conv2d(4, 72, 72, 256, 3, 3, 128, (1, 1), (1, 1), "f32", family=TENSOR)
     assert sg.sg_last_stream_k()[1] > 0, "this shape was meant to take the stream-K tail"
     assert_within_bound(O, want, S, "stream-K tail, conv2d f32")
+
+
+# ------------------------------------------------------------------ config 2: every shape of the sweep, both dtypes
+
+SWEEP = (256, 512, 1024, 2048, 4096)
+SWEEP_SHAPES = [(m, n, k) for m in SWEEP for n in SWEEP for k in SWEEP]
+_sweep_cache = {}
+
+
+def sweep_operands(dtype):
+    """One seeded 4096 x 4096 sample per operand and dtype (as the benchmark draws them); a shape's operands are the
+    leading sub-blocks, copied into dense buffers of their own."""
+    if dtype not in _sweep_cache:
+        _sweep_cache[dtype] = (operand((4096, 4096), SEED + 1, 1, "uniform", dtype), operand((4096, 4096), SEED + 1, 2, "uniform", dtype))
+    return _sweep_cache[dtype]
+
+
+def seam_points(M, N, count, seed):
+    """`count` hashed points plus the corners and both sides of every 128-row / 64-column tile seam along two lines."""
+    pm, pn = sample_points(M, N, count, seed)
+    sm = np.array([m for t in range(128, M, 128) for m in (t - 1, t)], np.int64)
+    sn = np.array([n for t in range(64, N, 64) for n in (t - 1, t)], np.int64)
+    pm = np.concatenate([pm, sm, np.full(sn.size, M - 1, np.int64), np.full(sn.size, M // 3, np.int64)])
+    pn = np.concatenate([pn, np.full(sm.size, N - 1, np.int64), sn, sn])
+    return pm, pn
+
+
+def check_sweep_point(C, a, b, M, N, K, dtype, what):
+    pm, pn = seam_points(M, N, 512, 1000 + M + 2 * N + 3 * K)
+    want, S = ref.matmul_points(a[:M, :K], b[:K, :N], pm, pn)
+    got = C[torch.from_numpy(pm).cuda(), torch.from_numpy(pn).cuda()]
+    ratio = assert_within_bound(got, want, S, f"{what} {dtype} {M}x{N}x{K}")
+    assert not torch.isnan(C).any(), f"{what} {dtype} {M}x{N}x{K}: unwritten elements"
+    if dtype == "f32":
+        assert ratio < F32_TENSOR_RATIO, ratio
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("M", SWEEP)
+def test_sweep_every_shape(dtype, M):
+    """All 125 shapes {256..4096}^3 of the benchmark's sweep (25 per test case), each into a NaN-filled output:
+    >= 512 sampled points plus tile seams and corners against the oracle, no element left unwritten."""
+    (A, a), (B, b) = sweep_operands(dtype)
+    for N in SWEEP:
+        for K in SWEEP:
+            Ad, Bd = A[:M, :K].contiguous(), B[:K, :N].contiguous()
+            C = torch.full((M, N), float("nan"), device="cuda")
+            sg.sg_matmul(Ad, Bd, C)
+            torch.cuda.synchronize()
+            assert sg.sg_last_kernel() == TENSOR
+            check_sweep_point(C, a, b, M, N, K, dtype, "sweep")
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_sweep_in_the_benchmark_launch_configuration(dtype):
+    """The 64 sweep shapes without a 4096 extent, launched the way bench.py launches a step: captured once into a CUDA
+    graph on four parallel branches, largest first, replayed twice; every shape checked as above."""
+    (A, a), (B, b) = sweep_operands(dtype)
+    shapes = sorted([s for s in SWEEP_SHAPES if 4096 not in s], key=lambda s: -s[0] * s[1] * s[2])
+    work = [(A[:m, :k].contiguous(), B[:k, :n].contiguous(), torch.full((m, n), float("nan"), device="cuda")) for m, n, k in shapes]
+    for Ad, Bd, C in work[:2]:
+        sg.sg_matmul(Ad, Bd, C)          # first calls outside capture (driver entry points, attributes)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    lanes = [torch.cuda.Stream() for _ in range(3)]
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        for ln in lanes:
+            ln.wait_stream(side)
+        for i, (Ad, Bd, C) in enumerate(work):
+            if i % 4 == 0:
+                sg.sg_matmul(Ad, Bd, C)
+            else:
+                with torch.cuda.stream(lanes[i % 4 - 1]):
+                    sg.sg_matmul(Ad, Bd, C)
+        for ln in lanes:
+            side.wait_stream(ln)
+    for _, _, C in work:
+        C.fill_(float("nan"))
+    g.replay()
+    g.replay()
+    torch.cuda.synchronize()
+    sg.sg_check()
+    for (m, n, k), (_, _, C) in zip(shapes, work):
+        check_sweep_point(C, a, b, m, n, k, dtype, "graph replay")
+
+
+# ------------------------------------------------------------------ forced k splits without a forced tile
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("splits", [2, 3, 8, 64])
+def test_forced_split_alone_never_fails(dtype, splits):
+    # a forced number of k ranges with the tile left to the library is taken when every range gets at least one
+    # k-block (4 k-blocks of 64 bf16, 8 of 32 f32 here) and ignored otherwise; the call succeeds either way
+    M, N, K = 4096, 4096, 256
+    (A, a), (B, b) = sweep_operands(dtype)
+    Ad, Bd = A[:M, :K].contiguous(), B[:K, :N].contiguous()
+    C = torch.full((M, N), float("nan"), device="cuda")
+    sg.sg_set_tile_override(0, 0, splits)
+    sg.sg_matmul(Ad, Bd, C)
+    torch.cuda.synchronize()
+    honoured = {("bf16", 2), ("f32", 2), ("f32", 3), ("f32", 8)}
+    if (dtype, splits) in honoured:
+        assert sg.sg_last_tile_choice()[2] == splits
+    check_sweep_point(C, a, b, M, N, K, dtype, f"forced split {splits}")
+
+
+def test_forced_pair_count_that_no_variant_can_honour():
+    # 64 columns: only the single-CTA 64-column tile applies; asking for pairs falls back to it
+    sg.sg_set_tile_override(0, 2, 0)
+    C, want, S = run_matmul(512, 64, 256, "bf16", family=TENSOR, seed=SEED + 40)
+    assert sg.sg_last_tile_choice()[:2] == (64, 1)
+    assert_within_bound(C, want, S, "forced pairs on a 64-column problem")
+
+
+# ------------------------------------------------------------------ the time-out path
+
+def test_device_timeout_is_reported_once_and_cleared():
+    """A warp that waits about a millisecond on a barrier nobody signals gives up like any pipeline wait: the status
+    word is set, the kernel returns, sg_check reports SG_ERR_DEVICE_TIMEOUT exactly once, and the device stays usable."""
+    sg.sg_check()
+    sg.sg_selftest_wait_timeout(2_000_000)
+    with pytest.raises(sg.SgError) as err:
+        sg.sg_check()
+    assert err.value.code == 5 and "wait expired" in str(err.value)
+    sg.sg_check()                                   # cleared by the read
+    C, want, S = run_matmul(256, 256, 256, "bf16", family=TENSOR, seed=SEED + 41)
+    assert_within_bound(C, want, S, "after a reported time-out")
+    sg.sg_check()
