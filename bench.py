@@ -40,12 +40,53 @@ WORKLOAD = ("matmul sweep M,N,K in {256,512,1024,2048,4096} (125 shapes), bf16 i
 FLOPS_PER_DTYPE = sum(2.0 * m * n * k for m, n, k in SHAPES)
 FLOPS_PER_STEP = 2 * FLOPS_PER_DTYPE
 
-# DRAM bytes per launch of the dominant kernel from the committed ncu capture; None when the
-# kernel changed after the capture was taken.
-NCU_TRAFFIC_BYTES = 25.6e6   # profiles/bench_sweep_launch_list.md: average over the 125 f32 launches of a step
+METRIC = "matmul sweep GFLOP/s"      # the same string in both arms (ours and --impl reference)
+UNIT = "GFLOP/s"
 # tf32 : bf16 dense tensor throughput (nominal 1.1 : 2.25 PFLOP/s; the issue rate measured on
 # this chip is exactly half)
 TF32_OVER_BF16 = 0.5
+NOMINAL_BF16_TFLOPS = 2250.0         # the chip's dense bf16 tensor rate as NVIDIA states it; tf32 is half of it
+SAMPLES = 100                        # timing protocol of the paper's Section 4.3: 100 measurements, median and quartiles
+# DRAM traffic of the dominant kernel: written next to the ncu summary it was read from, with a hash of the
+# kernel's source files at capture time; None when the file is absent or the sources changed since
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "tc_gemm_f32_traffic.txt")
+KERNEL_SOURCES = ("paper_2202_03293_b200/csrc/sg_tc.cu", "paper_2202_03293_b200/csrc/sg_tc_ptx.cuh")
+
+
+def kernel_source_hash():
+    import hashlib
+    h = hashlib.sha256()
+    for rel in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def traffic_per_launch(avg_algorithmic_bytes):
+    """DRAM bytes per launch of the f32 tensor-core kernel, from one small ncu capture of a single shape scaled by
+    algorithmic bytes to the step's average launch.  (bytes or None, note)."""
+    if not os.path.exists(TRAFFIC_FILE):
+        return None, "no capture on file"
+    kv = {}
+    with open(TRAFFIC_FILE) as f:
+        for line in f:
+            if ":" in line and not line.lstrip().startswith("#"):
+                k, v = line.split(":", 1)
+                kv[k.strip()] = v.strip()
+    try:
+        if kv["source_hash"] != kernel_source_hash():
+            return None, "kernel sources changed since the capture"
+        scale = avg_algorithmic_bytes / float(kv["algorithmic_bytes_of_captured_launch"])
+        return round(float(kv["dram_bytes_per_launch"]) * scale), f"{kv.get('shape', '?')} captured, scaled by algorithmic bytes x{scale:.3f}"
+    except (KeyError, ValueError):
+        return None, "capture file unreadable"
+
+
+def quartiles(xs):
+    """median, p25, p75, mean of a list of samples."""
+    xs = sorted(xs)
+    q = statistics.quantiles(xs, n=4, method="inclusive") if len(xs) > 1 else [xs[0]] * 3
+    return {"median": q[1], "p25": q[0], "p75": q[2], "mean": statistics.fmean(xs), "n": len(xs)}
 BW_ROWS, BW_COLS = 16384, 12288   # shape of the memory-bound 2-D kernels' rows in the per-op table (805 MB of f32)
 
 
@@ -134,9 +175,9 @@ def time_launches(fn, iters, warmup):
     return e0.elapsed_time(e1) / iters
 
 
-def time_graph(calls, reps, warmup=3):
-    """Average device time per call in ms with the calls captured once into a CUDA graph
-    and replayed, so that host-side call overhead is outside the measurement."""
+def time_graph(calls, samples, warmup=3):
+    """Device time per call in ms, `samples` measurements: the calls are captured once into a CUDA graph (host-side
+    call overhead stays outside) and every replay is one sample, bracketed by CUDA events on the launching stream."""
     import torch
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
@@ -150,13 +191,13 @@ def time_graph(calls, reps, warmup=3):
     for _ in range(warmup):
         graph.replay()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(samples + 1)]
+    ev[0].record()
+    for i in range(samples):
         graph.replay()
-    e1.record()
+        ev[i + 1].record()
     torch.cuda.synchronize()
-    return e0.elapsed_time(e1) / reps / len(calls)
+    return [ev[i].elapsed_time(ev[i + 1]) / len(calls) for i in range(samples)]
 
 
 def op_specs(sg, seed, bw_rows=None):
@@ -253,8 +294,10 @@ def op_specs(sg, seed, bw_rows=None):
     }
 
 
-def measure_op(sg, peaks, spec, reps=None):
-    """Times one op: buffers rotate over enough sets to exceed L2 between reuses."""
+def measure_op(sg, peaks, spec, samples=SAMPLES):
+    """Times one op, `samples` measurements.  Cold regime (the one the roofline fraction is quoted from): buffers rotate
+    over enough sets to exceed L2 between reuses.  Warm regime, for ops whose operands fit in L2: the same buffers
+    every call (the paper's "steady state")."""
     import torch
     label, flops, bytes_, dtype, make, call = spec
     ffma_peak = 148 * 128 * 2 * 1.965e9 / 1e12      # TFLOP/s at the maximum SM clock
@@ -264,29 +307,39 @@ def measure_op(sg, peaks, spec, reps=None):
     calls = [(lambda b=bufs[i % sets]: call(*b)) for i in range(ncalls)]
     call(*bufs[0])
     torch.cuda.synchronize()
-    fam = sg.sg_last_kernel()
-    est_ms = max(flops / 3e14, 5e-3)
-    if reps is None:
-        reps = int(max(3, min(50, 0.25 / (est_ms * 1e-3 * ncalls))))
-    ms = time_graph(calls, reps)
+    fam, name = sg.sg_last_kernel(), sg.sg_last_kernel_name()
+    est_ms = max(flops / 3e14, 5e-3) * ncalls
+    samples = int(max(5, min(samples, 2000.0 / est_ms)))        # at most ~2 s of device time per op
+    q = quartiles(time_graph(calls, samples))
+    ms = q["median"]
+    warm = None
+    if bytes_ < 100e6:
+        warm = quartiles(time_graph([(lambda b=bufs[0]: call(*b)) for _ in range(ncalls)], min(samples, 30)))
     host_ms = time_launches(lambda i: call(*bufs[i % sets]), max(3, min(100, ncalls * 2)), 2)
     tf = flops / (ms * 1e-3) / 1e12
     tensor_peak = peaks["bf16_tflops"] * (TF32_OVER_BF16 if dtype == "f32" else 1.0)
+    nominal_peak = NOMINAL_BF16_TFLOPS * (TF32_OVER_BF16 if dtype == "f32" else 1.0)
     on_tensor = fam in (sg.SG_KERNEL_TENSOR, sg.SG_KERNEL_CONV_STRIP)
-    kernel_name = {sg.SG_KERNEL_TENSOR: "tensor", sg.SG_KERNEL_CONV_STRIP: "tensor (conv strip)",
-                   sg.SG_KERNEL_TMA_MOVE: "tma move"}.get(fam, "cuda cores")
     t_compute = flops / ((tensor_peak if on_tensor else ffma_peak) * 1e12)
     t_bytes = bytes_ / (peaks["hbm_gbs"] * 1e9)
     bound = max(t_compute, t_bytes)
-    row = {"op": label, "dtype": dtype, "kernel": kernel_name,
-           "us": round(ms * 1e3, 2), "us_with_host_call": round(host_ms * 1e3, 2), "gflops": round(tf * 1e3, 1),
+    row = {"op": label, "dtype": dtype, "kernel": name,
+           "us": round(ms * 1e3, 2), "us_p25": round(q["p25"] * 1e3, 2), "us_p75": round(q["p75"] * 1e3, 2),
+           "us_mean": round(q["mean"] * 1e3, 2), "samples": q["n"],
+           "us_with_host_call": round(host_ms * 1e3, 2), "gflops": round(tf * 1e3, 1),
            "gbs": round(bytes_ / (ms * 1e-3) / 1e9, 1),
            "bound": "hbm" if t_bytes > t_compute else ("tensor" if on_tensor else "ffma"),
            "roofline_us": round(bound * 1e6, 2), "frac": round(bound / (ms * 1e-3), 4), "rotating_sets": sets,
-           "timing": "CUDA graph replay"}
+           "timing": "CUDA graph replay, one sample per replay, cold (rotating buffers > L2)"}
+    if warm is not None:
+        row["us_warm_l2"] = round(warm["median"] * 1e3, 2)
+    if on_tensor:
+        # against the chip's nominal dense tensor rate (bf16 2250 TFLOP/s, tf32 half of it)
+        row["frac_of_nominal_tensor_peak"] = round(tf / nominal_peak, 4)
     if dtype == "f32" and on_tensor:
-        # the f32 path issues three tf32 products per term: its own ceiling is a third of the tf32 peak
-        row["frac_of_3xtf32_ceiling"] = round(max(3 * t_compute, t_bytes) / (ms * 1e-3), 4)
+        # the f32 path issues three tf32 products per term; relative to a third of the MEASURED tf32-equivalent rate
+        # (a cuBLAS-derived figure, not a limit of the chip: this ratio can exceed 1)
+        row["frac_x3_products_vs_measured"] = round(max(3 * t_compute, t_bytes) / (ms * 1e-3), 4)
     del bufs, calls
     torch.cuda.empty_cache()
     return row
@@ -297,47 +350,76 @@ def per_op_table(sg, peaks, seed):
     return [measure_op(sg, peaks, specs[name]) for name in specs]
 
 
-def cpu_baseline(target_seconds=12.0):
-    """Times the oracle on a bounded sample (leading rows of the 4096^3 matmul) on the host cores."""
+def cpu_baseline(target_seconds=12.0, extras=True):
+    """Times the oracle, as it stands, on bounded samples of the workloads on the host cores: leading rows of the
+    sweep's 4096^3 point with every thread (the contract's `value`) and with one thread, and configs 1, 3 and 4 with
+    one thread and with every thread (the paper's own numbers are single-threaded)."""
+    import numpy as np
     from oracle import ref
     from paper_2202_03293_b200 import inputs
     seed = inputs.BASE_SEED + 1
     _, b = inputs.make((K, N), seed, 2, "uniform", "bf16")
     threads = ref.max_threads()
-    rows = threads
-    _, a = inputs.make((rows, K), seed, 1, "uniform", "bf16")
-    t0 = time.perf_counter()
-    ref.matmul(a, b)
-    dt = time.perf_counter() - t0
-    rows_full = int(min(M, max(rows, rows * target_seconds / max(dt, 1e-6))))
-    rows_full -= rows_full % threads
-    rows_full = max(rows_full, threads)
-    _, a = inputs.make((rows_full, K), seed, 1, "uniform", "bf16")
-    t0 = time.perf_counter()
-    ref.matmul(a, b)
-    dt = time.perf_counter() - t0
+
+    def mm_rows(rows, nthreads):
+        _, a = inputs.make((rows, K), seed, 1, "uniform", "bf16")
+        t0 = time.perf_counter()
+        ref.matmul(a, b, threads=nthreads)
+        return time.perf_counter() - t0
+
+    dt = mm_rows(threads, threads)
+    rows_full = int(min(M, max(threads, threads * target_seconds / max(dt, 1e-6))))
+    rows_full = max(rows_full - rows_full % threads, threads)
+    dt = mm_rows(rows_full, threads)
     gflops = 2.0 * rows_full * N * K / dt / 1e9
-    return {"value": round(gflops, 3), "unit": "GFLOP/s", "cores": threads, "kind": "oracle",
-            "sample": f"first {rows_full} of {M} rows of the 4096^3 matmul ({dt:.1f} s)"}, dt, rows_full
+    info = {"value": round(gflops, 3), "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"first {rows_full} of {M} rows of the 4096^3 matmul ({dt:.1f} s)"}
+    if extras:
+        others = []
+        rows1 = max(1, int(rows_full / threads / 4))
+        d1 = mm_rows(rows1, 1)
+        others.append({"op": "matmul 4096^3 (sweep corner)", "threads": 1, "gflops": round(2.0 * rows1 * N * K / d1 / 1e9, 3),
+                       "sample": f"first {rows1} rows ({d1:.1f} s)"})
+        a1, b1 = inputs.uniform((128, 128), seed, 3), inputs.uniform((128, 128), seed, 4)
+        i3, k3 = inputs.uniform((16, 1026, 64), seed, 5), inputs.uniform((3, 64, 128), seed, 6)
+        i4 = inputs.make((4, 58, 58, 64), seed, 7, "normal", "bf16")[1]
+        k4 = inputs.make((3, 3, 64, 128), seed, 8, "normal", "bf16")[1]
+        cases = [("matmul 128^3 f32 (config 1)", 2.0 * 128 ** 3, "whole problem", lambda t: ref.matmul(a1, b1, threads=t)),
+                 ("conv_1d_nwc_wcf config 3", 2.0 * 16 * 1024 * 128 * 3 * 64, "16 of 32 batch entries", lambda t: ref.conv1d_nwc_wcf(i3, k3, threads=t)),
+                 ("conv_2d_nhwc_hwcf config 4", 2.0 * 4 * 56 * 56 * 128 * 9 * 64, "4 of 16 images", lambda t: ref.conv2d_nhwc_hwcf(i4, k4, threads=t))]
+        for label, flops, sample, fn in cases:
+            for t in (1, threads):
+                fn(t)                                   # (the first call also builds and loads the library)
+                t0 = time.perf_counter()
+                fn(t)
+                d = time.perf_counter() - t0
+                others.append({"op": label, "threads": t, "gflops": round(flops / d / 1e9, 3), "sample": f"{sample} ({d:.2f} s)"})
+        info["others"] = others
+    return info, dt, rows_full
 
 
 def run_reference(args, rank):
+    """The reference arm: the paper ships no code, so the CPU oracle is timed, as it stands, on the host cores; a step
+    is a bounded sample of the same workload (leading rows of the sweep's largest point)."""
     if rank != 0:
         return
-    vals = []
+    vals, times = [], []
     info = None
-    for i in range(args.warmup + args.steps):
-        info, dt, rows = cpu_baseline(target_seconds=max(2.0, 60.0 / max(1, args.warmup + args.steps)))
+    n = max(1, args.warmup + args.steps)
+    for i in range(n):
+        info, dt, rows = cpu_baseline(target_seconds=max(1.0, min(10.0, 90.0 / n)), extras=False)
         if i >= args.warmup:
             vals.append(info["value"])
-    value = statistics.mean(vals)
+            times.append(dt)
+    value = statistics.fmean(vals)
     info["value"] = round(value, 3)
-    line = {"impl": "reference", "metric": "matmul sweep GFLOP/s (f64 CPU oracle on a bounded sample)", "value": round(value, 3),
-            "unit": "GFLOP/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": round(FLOPS_PER_STEP / (value * 1e9) * 1e3, 1), "higher_is_better": True, "scaling": "weak",
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 3),
+            "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(statistics.fmean(times) * 1e3, 1), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "sample": "leading rows of the sweep's 4096^3 point, bf16-valued inputs"},
-            "cpu_baseline": info, "e2e": {"value": round(value, 3), "unit": "GFLOP/s", "h2d_bytes_per_step": 0,
+            "config": {"workload": WORKLOAD, "sample": "each step: leading rows of the sweep's 4096^3 point, bf16-valued inputs; "
+                                                       "ms_per_step is the time of that sample, not of the whole sweep"},
+            "cpu_baseline": info, "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0,
                                            "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
@@ -404,6 +486,23 @@ def main():
         return
 
     import torch
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started as a plain process: start one rank per GPU ourselves (as many as the node has, at most --gpus)
+        ranks = min(args.gpus, torch.cuda.device_count())
+        if ranks > 1:
+            import socket
+            with socket.socket() as sock:
+                sock.bind(("127.0.0.1", 0))
+                port = sock.getsockname()[1]
+            argv = [a for a in sys.argv[1:]]
+            for i, a in enumerate(argv):            # the ranks are told how many of them there are
+                if a == "--gpus":
+                    argv[i + 1] = str(ranks)
+                elif a.startswith("--gpus="):
+                    argv[i] = f"--gpus={ranks}"
+            cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={ranks}",
+                   "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + argv
+            raise SystemExit(subprocess.call(cmd))
     import torch.distributed as dist
     from paper_2202_03293_b200 import binding as sg
     from paper_2202_03293_b200 import inputs, sharding
@@ -423,7 +522,7 @@ def main():
         specs = op_specs(sg, seed, args.bw_rows)
         if args.op not in specs:
             raise SystemExit(f"--op must be one of {sorted(specs)}")
-        print(json.dumps(measure_op(sg, peaks, specs[args.op], reps=max(1, min(args.steps, 5)))), flush=True)
+        print(json.dumps(measure_op(sg, peaks, specs[args.op], samples=max(1, min(args.steps, 5)))), flush=True)
         return
 
     bufs = sweep_buffers(torch, seed)
@@ -495,16 +594,18 @@ def main():
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    e0.record()
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    marks[0].record()
     for i in range(args.steps):
         graph_step()
-    e1.record()
+        marks[i + 1].record()
     barrier()
     launches = launches_per_step * args.steps
     clocks = sampler.stop()
     sg.sg_check()
-    ms_total = sharding.max_over_ranks(e0.elapsed_time(e1), device="cuda")
+    ms_total = sharding.max_over_ranks(marks[0].elapsed_time(marks[-1]), device="cuda")
     ms_per_step = ms_total / args.steps
+    step_q = quartiles([marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)])      # this rank's steps
     value = world * FLOPS_PER_STEP / (ms_per_step * 1e-3) / 1e9      # GFLOP/s, all ranks
 
     eager_steps = max(3, min(20, args.steps))
@@ -562,7 +663,7 @@ def main():
         e1.record()
         barrier()
         e2e_ms = sharding.max_over_ranks(e0.elapsed_time(e1), device="cuda")
-        e2e = {"value": round(world * FLOPS_PER_STEP / (e2e_ms / e2e_steps * 1e-3) / 1e9, 1), "unit": "GFLOP/s",
+        e2e = {"value": round(world * FLOPS_PER_STEP / (e2e_ms / e2e_steps * 1e-3) / 1e9, 1), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
         del host
 
@@ -580,19 +681,26 @@ def main():
     share_f32 = f32_ms / (f32_ms + bf16_ms)
     f32_tf = FLOPS_PER_DTYPE / (ms_per_step * share_f32 * 1e-3) / 1e12
     bf16_tf = FLOPS_PER_DTYPE / (ms_per_step * (1 - share_f32) * 1e-3) / 1e12
+    avg_alg_bytes = sum((m * k + k * n) * 4 + m * n * 4 for m, n, k in SHAPES) / len(SHAPES)
+    traffic, traffic_note = traffic_per_launch(avg_alg_bytes)
     roofline = {"bound": "tensor", "achieved": round(f32_tf, 1), "peak": round(tf32_peak, 1), "unit": "TFLOP/s",
-                "frac": round(f32_tf / tf32_peak, 4), "traffic": NCU_TRAFFIC_BYTES,
+                "frac": round(f32_tf / tf32_peak, 4), "traffic": traffic, "traffic_source": traffic_note,
+                "algorithmic_bytes_per_launch": round(avg_alg_bytes),
                 "kernel": "tc_gemm_kernel<BN, CG, f32> (125 launches per step, %.0f%% of the step)" % (100 * share_f32),
                 "peak_source": f"{peaks['source']} {peak_kind} x {TF32_OVER_BF16} (tf32 : bf16 tensor rate); timed region {timed_seconds:.2f} s",
                 "algorithmic_flops_per_step": FLOPS_PER_DTYPE, "avg_launch_us": round(ms_per_step * share_f32 * 1e3 / len(SHAPES), 2),
-                "note": "f32 accuracy costs three tf32 products per term, so this kernel's own ceiling is about frac = 0.333 (the peak is a measured cuBLAS rate, not a hard limit)",
-                "frac_of_3xtf32_ceiling": round(3 * f32_tf / tf32_peak, 4),
+                "note": "f32 accuracy costs three tf32 products per term: a third of the tf32 rate is what this kernel can reach; the peak is a measured cuBLAS rate, not a limit of the chip",
+                "frac_x3_products_vs_measured": round(3 * f32_tf / tf32_peak, 4),
+                "frac_of_nominal_tensor_peak": round(f32_tf / (NOMINAL_BF16_TFLOPS * TF32_OVER_BF16), 4),
                 "bf16_half": {"achieved": round(bf16_tf, 1), "peak": peaks[peak_kind], "frac": round(bf16_tf / peaks[peak_kind], 4),
+                              "frac_of_nominal_tensor_peak": round(bf16_tf / NOMINAL_BF16_TFLOPS, 4),
                               "share_of_step": round(1 - share_f32, 4)}}
 
-    line = {"metric": "matmul sweep GFLOP/s (and fraction of the tensor-core roofline) on B200", "value": round(value, 1),
-            "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
-            "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+    line = {"metric": METRIC, "value": round(value, 1),
+            "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+            "ms_per_step": round(ms_per_step, 5),
+            "ms_per_step_samples": {k: (round(v, 5) if k != "n" else v) for k, v in step_q.items()},
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16+f32", "data": "synthetic",
             "config": {"workload": WORKLOAD, "calls_per_step": 2 * len(SHAPES),
                        "launch": f"each step replays two CUDA graphs holding the step's 250 library calls on {max(1, args.streams)} parallel branches",
