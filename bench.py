@@ -522,7 +522,17 @@ def main():
         specs = op_specs(sg, seed, args.bw_rows)
         if args.op not in specs:
             raise SystemExit(f"--op must be one of {sorted(specs)}")
-        print(json.dumps(measure_op(sg, peaks, specs[args.op], samples=max(1, min(args.steps, 5)))), flush=True)
+        if args.steps == 0:
+            # a handful of plain launches over two buffer sets and nothing else: the command a profiler capture wraps
+            label, flops, bytes_, dtype, make, call = specs[args.op]
+            bufs = [make(s) for s in range(2)]
+            for i in range(4):
+                call(*bufs[i % 2])
+            torch.cuda.synchronize()
+            sg.sg_check()
+            print(json.dumps({"op": label, "kernel": sg.sg_last_kernel_name(), "launched": 4}), flush=True)
+            return
+        print(json.dumps(measure_op(sg, peaks, specs[args.op], samples=max(1, min(args.steps, SAMPLES)))), flush=True)
         return
 
     bufs = sweep_buffers(torch, seed)

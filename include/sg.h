@@ -266,17 +266,26 @@ sg_status sg_set_kernel_override(int kernel_family);
  */
 sg_status sg_set_tile_override(int tile_n, int ctas_per_tile, int k_splits);
 
-/* {tile width, CTAs per tile, k ranges} of the most recent tensor-core launch of the process. */
+/* {tile width, CTAs per tile, k ranges} of the most recent tensor-core launch made by this host thread. */
 void sg_last_tile_choice(int out[3]);
 
 /*
- * Stream-K tail of the most recent tensor-core launch of the process: when whole tiles are dealt out and the last
+ * Stream-K tail of the most recent tensor-core launch made by this host thread: when whole tiles are dealt out and the last
  * wave of tiles would be partly filled, the tiles of that wave are cut along the reduction instead (every CTA or CTA
  * pair gets an equal run of their k-blocks; the partial sums meet in the output by reduce-add).  out[0] = index of
  * the first tile of the tail in the tile order (-1: no tail), out[1] = k-blocks per run.  SG_TC_SK=0 in the
  * environment (read at the first call) turns the tail off.
  */
 void sg_last_stream_k(int out[2]);
+
+/*
+ * Tensor-map cache counters since the library was loaded: out[0] = look-ups answered from the
+ * cache, out[1] = look-ups that had to encode a map.  The cache is keyed by device, base pointer,
+ * element type, extents, byte strides, box and the other encode parameters, never by the
+ * memory's contents; it holds at most 2048 maps (about 0.7 MB of host memory), replacing the
+ * least recently used entry of a full bucket.
+ */
+void sg_tensor_map_cache_stats(int64_t out[2]);
 
 /*
  * Self-test of the device-side time-out path (the paper has no counterpart): launches one warp
@@ -294,6 +303,9 @@ sg_status sg_selftest_wait_timeout(int64_t budget_cycles, sg_stream_t stream);
  *   SG_TC_SK        0: never cut the last wave into a stream-K tail; 2: whenever the shape allows it
  *   SG_TC_KPS       1: one k-block per pipeline stage everywhere (bf16 matmuls normally move two)
  *   SG_TC_TA        0: keep the split f32 input tile in shared memory instead of tensor memory
+ *   SG_TC_PDL       0: tensor-core launches never start before the kernel ahead of them in the
+ *                   stream has finished (by default they set themselves up while it drains and
+ *                   wait for it before their first global read or write)
  *   SG_CONV_SINGLE  1: the stride-1 convolution kernel never uses CTA pairs
  */
 

@@ -26,6 +26,7 @@ EXPORTS = [
     "sg_depthwise_conv2d_nhwc_hwc", "sg_copy2d", "sg_transpose2d", "sg_colred2d", "sg_rowred2d", "sg_check", "sg_status_string",
     "sg_version", "sg_last_kernel", "sg_launch_count", "sg_set_kernel_override", "sg_set_tile_override",
     "sg_last_tile_choice", "sg_last_stream_k", "sg_shutdown", "sg_last_kernel_name", "sg_selftest_wait_timeout",
+    "sg_tensor_map_cache_stats",
 ]
 
 
@@ -80,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.sg_last_kernel_name.restype = ctypes.c_char_p
         L.sg_selftest_wait_timeout.argtypes = [i64, vp]
         L.sg_selftest_wait_timeout.restype = ci
+        L.sg_tensor_map_cache_stats.argtypes = [p64]
+        L.sg_tensor_map_cache_stats.restype = None
         _lib = L
     return _lib
 
@@ -288,3 +291,10 @@ def sg_selftest_wait_timeout(budget_cycles: int = 2_000_000, stream=None) -> Non
     rc = lib().sg_selftest_wait_timeout(int(budget_cycles), _stream(stream))
     if rc != SG_OK:
         raise SgError(rc, "sg_selftest_wait_timeout")
+
+
+def sg_tensor_map_cache_stats():
+    """(hits, misses) of the tensor-map cache since the library was loaded."""
+    out = (ctypes.c_int64 * 2)()
+    lib().sg_tensor_map_cache_stats(out)
+    return int(out[0]), int(out[1])

@@ -316,6 +316,13 @@ void sg_last_stream_k(int out[2]) {
     if (out) sg::tensor_last_stream_k(out);
 }
 
+void sg_tensor_map_cache_stats(int64_t out[2]) {
+    if (!out) return;
+    long long v[2];
+    tensor_map_cache_stats(v);
+    out[0] = v[0]; out[1] = v[1];
+}
+
 sg_status sg_selftest_wait_timeout(int64_t budget_cycles, sg_stream_t stream) {
     if (budget_cycles < 1000 || budget_cycles > 20000000) return SG_ERR_INVALID_ARG;    // at most ~10 ms of spinning
     return launch_wait_timeout_selftest((long long)budget_cycles, static_cast<cudaStream_t>(stream)) == cudaSuccess ? SG_OK : SG_ERR_CUDA;

@@ -1,25 +1,35 @@
-// Stride-1 bf16 convolutions on the tensor cores with every input pixel fetched once per tile
-// and the filter resident in shared memory.
+// Stride-1 convolutions on the tensor cores with every input pixel fetched once per tile and the
+// filter resident in shared memory; bf16 inputs directly, f32 inputs as three tf32 products per term.
 //
 // The im2col kernel fetches, for each of the KH*KW filter taps, a fresh 128-pixel input tile and
 // a fresh filter tile: on conv_2d 3x3 that is nine copies of nearly the same pixels and nine
 // filter tiles per output tile, and the TMA issue / L2 -> shared memory fill rate bounds it.
-// Here the iteration space is walked in "padded" output coordinates: q = (n*H_in + h)*W_in + w
-// counts output positions with the INPUT's row pitch, so the input pixel of tap (kh, kw) is row
-// q + kh*dh*W_in + kw*dw of the input seen as a [N*H_in*W_in, C] matrix.  A tile is 128
-// consecutive q (256 for a CTA pair).  Per block of 64 channels ONE TMA load brings, for every
-// filter row kh, the strip of 128 + (KW-1)*dw rows that the KW taps of that row need (a 3-D
-// box over an overlapping view of the input whose third dimension steps by dh*W_in rows), and
-// each tap's MMAs read its strip through a matrix descriptor whose start address is shifted by
-// kw*dw rows.  The filter (all taps, all channels, the tile's columns) is loaded once per CTA.
-// Positions whose (h, w) fall outside the output (the last KH-1 rows and KW-1 columns of every
-// image) are computed and dropped in the epilogue: (H_in*W_in)/(H_out*W_out) - 1 of the MMA
-// work, 7 % on 58x58 -> 56x56.
+// Here positions are counted with the INPUT's row pitch, q = (n*H_in + h)*W_in + w, so the input
+// pixel of tap (kh, kw) is row q + kh*dh*W_in + kw*dw of the input seen as a [N*H_in*W_in, C]
+// matrix.  A tile is 128 consecutive q that start at the beginning of an output row:
+//   * W_in <= 128: R whole image rows (R*W_in <= 128); positions with w >= W_out are computed and dropped;
+//   * W_in  > 128: a segment of 128 output positions of one image row.
+// Per block of channels (64 bf16 / 32 f32) ONE TMA load brings, for every filter row kh, the strip
+// of 128 + (KW-1)*dw rows that the KW taps of that row need (a 3-D box over an overlapping view of
+// the input whose third dimension steps by dh*W_in rows).  The filter (all taps, all channels, the
+// tile's columns) is loaded once per CTA and stays in shared memory.
+//   bf16: each tap's MMAs read its strip through a matrix descriptor whose start address is
+//         shifted by kw*dw rows.
+//   f32:  the filter is split once into hi = tf32(x) and lo = tf32(x - hi) (and transposed to
+//         K-major, which kind::tf32 needs); sixteen converter warps split the strip rows of each
+//         tap the same way into tensor memory (the tap's shift is a row offset of their reads)
+//         and the MMA warp accumulates lo*hi + hi*lo + hi*hi with the A operand in tensor memory.
 //
-// Warp roles: warp 0 producer (TMA), warp 1 MMA issuer and TMEM owner, warps 2-9 epilogue
-// (TMEM -> registers -> shared-memory transpose -> 128-byte row segments in global memory, rows
-// that are not outputs skipped).  Every wait is bounded.
-#include <mutex>
+// Because tiles start at row beginnings, the epilogue is TMA only: TMEM -> registers -> a swizzled
+// staging copy of the whole tile, laid out [image row][32-column chunk][w][32 f32] -> ONE tensor
+// store (or reduce-add) per tile through a 5-D map {f in chunk, w, chunk, h, n} of the output (a
+// TMA instruction costs its issuing thread about 0.3 us whatever it moves, so the number of
+// instructions is what counts); the TMA unit clips w >= W_out of a last segment and h >= H_out of
+// a last tile.  Outputs whose F is no multiple of 32 are stored chunk by chunk and row by row.
+//
+// Warp roles: warp 0 producer (TMA), warp 1 MMA issuer and TMEM owner, warps 2-5 epilogue,
+// warps 6-21 converters (f32 only).  Every wait is bounded.
+#include <algorithm>
 
 #include "sg_internal.cuh"
 #include "sg_tc_ptx.cuh"
@@ -28,81 +38,155 @@ namespace sg {
 namespace {
 
 constexpr int BM = 128;
-constexpr int SUB_BYTES = 64 * 128;          // filter sub-tile: 64 k-rows x 64 columns of bf16
 constexpr int MAX_KH = 8;
 constexpr int MAX_STAGES = 8;
-constexpr int EPI_WARPS = 8;                 // two per TMEM lane quarter, each takes half of the tile's columns
-constexpr int STAGING_BYTES = EPI_WARPS * 4096;   // one 32 x 32 f32 chunk per epilogue warp
-constexpr int CONV_THREADS = 64 + 32 * EPI_WARPS;
+constexpr int CONVERTER_WARPS = 16;
+constexpr int A_SLOTS = 4;                   // f32: split input k-blocks in flight in tensor memory (64 columns each)
 constexpr int SMEM_LIMIT = 232448 - 1024;    // opt-in maximum minus the alignment slack
 
 struct ConvParams {
-    int Q;                 // N * H_in * W_in padded output positions
-    int num_q_tiles, num_f_tiles, items_per_group;
-    int KH, KW, kbpt;      // filter rows, taps per row, 64-channel blocks per tap
-    int Hin, Win, Hout, Wout;
+    int Q;                 // N * H_in * W_in positions of the input matrix
+    int num_tiles;         // position tiles (one per CTA; a pair takes two neighbours)
+    int num_pos_items;     // ceil(num_tiles / CG)
+    int num_f_tiles;
+    int N, Hin, Win, Hout, Wout;
+    int KH, KW, kbpt;      // filter rows, taps per row, channel blocks per tap
     int dw;                // input rows between taps of a filter row
+    int rows_per_tile;     // R: image rows per tile (1 when a tile is a segment of a row)
+    int segs;              // segments of 128 positions per image row (1 when a tile holds whole rows)
+    int tiles_per_image;
+    int chunk_rows;        // staging rows of one 32-column chunk of one image row: W_out (128 for segments)
+    int staging_bytes;     // the staged tile (f32: at least the raw filter, which is staged there before it is split)
+    int blocked_store;     // 1: F is a multiple of 32, one 5-D store moves the tile; 0: one 4-D store per image row and chunk
     int strip_rows;        // 128 + (KW - 1) * dw
     int strip_stage_bytes; // KH strips of strip_rows x 128 B, rounded up to 1 KiB
     int stages;
-    int flt_bytes;         // resident filter: KH * kbpt * KW blocks of B_COLS x 128 B
-    int flt_blocked;       // 1: the filter map is blocked by 64 columns (one load per filter row and channel block)
+    int flt_bytes;         // resident filter
+    int flt_blocked;       // bf16: 1 = the filter map is blocked by 64 columns (one load per filter row and channel block)
     int F;
     int accumulate;
-    long long o_n, o_h, o_w;
-    float *O;
+    int wait_prior;        // 1: launched to overlap the kernel ahead of it: wait for it before touching global memory
 };
 
-// CG = 1: one CTA computes 128 positions x BN columns.  CG = 2: a CTA pair (one cluster)
-// computes 256 positions x BN columns with tcgen05.mma.cta_group::2: each CTA loads the strips
-// of its own 128 positions and keeps its own BN/2 columns of the filter, which halves the
-// resident filter and leaves room for a deeper ring of strips.
-template <int BN, int CG>
-__global__ void __launch_bounds__(CONV_THREADS, 1)
-conv_strip_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_flt, const ConvParams p) {
+template <int BN, int CG, bool F32>
+struct ConvCfg {
+    static constexpr int B_COLS = BN / CG;                           // filter columns resident in this CTA
+    static constexpr int BLOCK_BYTES = B_COLS * 128 * (F32 ? 2 : 1); // one (tap, channel block): [hi | lo] for f32
+    static constexpr int ACC_COLS = 2 * BN;
+    static constexpr int USED_COLS = ACC_COLS + (F32 ? A_SLOTS * 64 : 0);
+    static constexpr int TMEM_COLS = USED_COLS <= 128 ? 128 : USED_COLS <= 256 ? 256 : 512;
+    static constexpr int THREADS = 64 + 128 + (F32 ? 32 * CONVERTER_WARPS : 0);
+    static_assert(USED_COLS <= 512 && B_COLS % 64 == 0, "tile width");
+};
+
+// 3xTF32 split of four f32 words: hi = x rounded to the nearest tf32 value (on the bit pattern: add half an ulp, clear
+// the low 13 bits), lo = (x - hi) rounded the same way; x - hi is exact in f32, so x - hi - lo is below 2^-22 |x|.
+// Words of magnitude >= 2^127 (where rounding up could reach infinity), infinities and NaNs take a slow path:
+// hi truncated, lo = 0 unless finite.
+__device__ __forceinline__ void split4(const uint4 v, uint4 &h, uint4 &l) {
+    const float fx = __uint_as_float(v.x), fy = __uint_as_float(v.y), fz = __uint_as_float(v.z), fw = __uint_as_float(v.w);
+    const float big = fmaxf(fmaxf(fabsf(fx), fabsf(fy)), fmaxf(fabsf(fz), fabsf(fw)));
+    if (big < 1.7014118e38f) {
+        h.x = (v.x + 0x1000u) & 0xFFFFE000u; l.x = (__float_as_uint(fx - __uint_as_float(h.x)) + 0x1000u) & 0xFFFFE000u;
+        h.y = (v.y + 0x1000u) & 0xFFFFE000u; l.y = (__float_as_uint(fy - __uint_as_float(h.y)) + 0x1000u) & 0xFFFFE000u;
+        h.z = (v.z + 0x1000u) & 0xFFFFE000u; l.z = (__float_as_uint(fz - __uint_as_float(h.z)) + 0x1000u) & 0xFFFFE000u;
+        h.w = (v.w + 0x1000u) & 0xFFFFE000u; l.w = (__float_as_uint(fw - __uint_as_float(h.w)) + 0x1000u) & 0xFFFFE000u;
+    } else {
+        auto one = [](uint32_t x, uint32_t &hi, uint32_t &lo) {
+            hi = x & 0xFFFFE000u;
+            const float d = __uint_as_float(x) - __uint_as_float(hi);
+            lo = (x & 0x7F800000u) == 0x7F800000u ? 0u : __float_as_uint(d);
+        };
+        one(v.x, h.x, l.x); one(v.y, h.y, l.y); one(v.z, h.z, l.z); one(v.w, h.w, l.w);
+    }
+}
+
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, uint32_t src, int x, int y, int z, int w) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_4d(const CUtensorMap *map, uint32_t src, int x, int y, int z, int w) {
+    asm volatile("cp.reduce.async.bulk.tensor.4d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap *map, uint32_t src, int x, int y, int z, int w, int v) {
+    asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_5d(const CUtensorMap *map, uint32_t src, int x, int y, int z, int w, int v) {
+    asm volatile("cp.reduce.async.bulk.tensor.5d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v) : "memory");
+}
+// The four epilogue warps agree on one answer (all of them reach this barrier whatever they found).
+__device__ __forceinline__ bool epilogue_all(bool mine) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, 1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out) : "r"((uint32_t)mine) : "memory");
+    return out != 0;
+}
+
+// CG = 1: one CTA computes a tile of 128 positions x BN columns.  CG = 2: a CTA pair (one cluster) computes two
+// neighbouring tiles x BN columns with tcgen05.mma.cta_group::2: each CTA loads the strips of its own tile and keeps
+// its own BN/2 columns of the filter, which halves the resident filter and leaves room for a deeper ring of strips.
+template <int BN, int CG, bool F32>
+__global__ void __launch_bounds__(ConvCfg<BN, CG, F32>::THREADS, 1)
+conv_strip_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_flt,
+                  const __grid_constant__ CUtensorMap map_out, const ConvParams p) {
+    using C = ConvCfg<BN, CG, F32>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
 
     const uint32_t flt_addr = smem_base;
     const uint32_t strips_addr = flt_addr + p.flt_bytes;
-    const uint32_t staging_off = p.flt_bytes + p.stages * p.strip_stage_bytes;
+    const uint32_t ring_bytes = (uint32_t)(p.stages * p.strip_stage_bytes);
+    const uint32_t staging_off = p.flt_bytes + ring_bytes;
+    const uint32_t staging_addr = smem_base + staging_off;
     uint8_t *staging_gen = smem_gen + staging_off;
-    const uint32_t bars_addr = smem_base + staging_off + STAGING_BYTES;
-    uint8_t *bars_gen = staging_gen + STAGING_BYTES;
-    // barrier block: full[8] | empty[8] | flt_full[8] | flt_free | acc_full[2] | acc_empty[2] | tmem_ptr | abort
+    const uint32_t bars_addr = staging_addr + (uint32_t)p.staging_bytes;
+    uint8_t *bars_gen = staging_gen + p.staging_bytes;
+    // barrier block: full[8] | empty[8] | split_full[4] | split_empty[4] | acc_full[2] | acc_empty[2] | flt_full |
+    //                flt_free | (unused) | tmem_ptr | abort
     auto full_bar = [&](int s) { return bars_addr + 8u * s; };
     auto empty_bar = [&](int s) { return bars_addr + 8u * (8 + s); };
-    auto flt_full_bar = [&](int kh) { return bars_addr + 8u * (16 + kh); };
-    const uint32_t flt_free_bar = bars_addr + 8u * 24;
-    auto acc_full_bar = [&](int b) { return bars_addr + 8u * (25 + b); };
-    auto acc_empty_bar = [&](int b) { return bars_addr + 8u * (27 + b); };
-    volatile uint32_t *tmem_ptr_slot = reinterpret_cast<volatile uint32_t *>(bars_gen + 8 * 29);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_gen + 8 * 29 + 4);
-    constexpr uint32_t TMEM_COLS = 2 * BN;
-    constexpr int B_COLS = BN / CG;            // filter columns resident in this CTA
+    auto split_full_bar = [&](int s) { return bars_addr + 8u * (16 + s); };
+    auto split_empty_bar = [&](int s) { return bars_addr + 8u * (20 + s); };
+    auto acc_full_bar = [&](int b) { return bars_addr + 8u * (24 + b); };
+    auto acc_empty_bar = [&](int b) { return bars_addr + 8u * (26 + b); };
+    const uint32_t flt_full_bar = bars_addr + 8u * 28;
+    const uint32_t flt_free_bar = bars_addr + 8u * 29;
+    volatile uint32_t *tmem_ptr_slot = reinterpret_cast<volatile uint32_t *>(bars_gen + 8 * 31);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_gen + 8 * 31 + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) { prefetch_tensormap(&map_in); prefetch_tensormap(&map_flt); }
-    // In a pair, CTA 0 (the leader) issues the MMAs and owns the barriers the loads signal.
+    // a launch behind this one that asked for it may start to set itself up as our CTAs leave their SMs
+    asm volatile("griddepcontrol.launch_dependents;");
+    if (threadIdx.x == 0) { prefetch_tensormap(&map_in); prefetch_tensormap(&map_flt); prefetch_tensormap(&map_out); }
+    // In a pair, CTA 0 (the leader) issues the MMAs and owns the barriers the bf16 loads signal.
     const uint32_t cta_rank = CG == 2 ? cluster_ctarank() : 0u;
-    const int group_id = (int)blockIdx.x / CG;
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int k = 0; k < MAX_KH; ++k) mbar_init(flt_full_bar(k), 1);
-        mbar_init(flt_free_bar, 1);
-        for (int b = 0; b < 2; ++b) { mbar_init(acc_full_bar(b), 1); mbar_init(acc_empty_bar(b), EPI_WARPS * CG); }
-        *abort_flag = 0;
+    const int group_id = (int)blockIdx.x / CG, num_groups = (int)gridDim.x / CG;
+    if (warp == 0) {
+        // One barrier per lane.  full: one arrive.expect_tx by the producer.  empty: one tcgen05.commit (bf16) or one
+        // arrive per converter warp of this CTA (f32).  split_full / flt_ready: one arrive per converter warp of every
+        // CTA of the group.  acc_empty: one arrive per epilogue warp of every CTA of the group.
+        const uint32_t count = lane < 8 ? 1u : lane < 16 ? (F32 ? CONVERTER_WARPS : 1u) : lane < 20 ? (uint32_t)(CONVERTER_WARPS * CG)
+                             : lane < 26 ? 1u : lane < 28 ? (uint32_t)(4 * CG) : lane < 30 ? 1u : (uint32_t)(CONVERTER_WARPS * CG);
+        if (lane < 31) mbar_init(bars_addr + 8u * lane, count);
+        if (lane == 31) *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
         if constexpr (CG == 2) {
             asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                         ::"r"(smem_u32(const_cast<uint32_t *>(tmem_ptr_slot))), "r"(TMEM_COLS) : "memory");
+                         ::"r"(smem_u32(const_cast<uint32_t *>(tmem_ptr_slot))), "r"((uint32_t)C::TMEM_COLS) : "memory");
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
         } else {
             asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                         ::"r"(smem_u32(const_cast<uint32_t *>(tmem_ptr_slot))), "r"(TMEM_COLS) : "memory");
+                         ::"r"(smem_u32(const_cast<uint32_t *>(tmem_ptr_slot))), "r"((uint32_t)C::TMEM_COLS) : "memory");
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
         }
     }
@@ -112,67 +196,92 @@ conv_strip_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_const
     tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_slot;
 
-    // this group's items: a contiguous run of (column tile, q tile), q fastest, so that the resident
-    // filter changes as rarely as possible
-    const int total_items = p.num_q_tiles * p.num_f_tiles;
-    const int item0 = group_id * p.items_per_group;
-    const int item1 = item0 + p.items_per_group < total_items ? item0 + p.items_per_group : total_items;
-    const uint32_t flt_block_bytes = (uint32_t)B_COLS * 128u;   // one (tap, channel block): B_COLS/64 sub-tiles
+    // this group's items: a contiguous, balanced run of (column tile, position item), positions fastest, so that the
+    // resident filter changes as rarely as possible
+    const int total_items = p.num_pos_items * p.num_f_tiles;
+    const int item0 = (int)((long long)group_id * total_items / num_groups);
+    const int item1 = (int)((long long)(group_id + 1) * total_items / num_groups);
+    // tile -> first position, image, first row, first column
+    struct Tile { int q0, n, h0, w0; bool live; };
+    auto decode = [&](int pos_item) {
+        Tile t;
+        const int tile = pos_item * CG + (int)cta_rank;
+        t.live = tile < p.num_tiles;
+        t.n = tile / p.tiles_per_image;
+        const int r = tile - t.n * p.tiles_per_image;
+        if (p.segs == 1) { t.h0 = r * p.rows_per_tile; t.w0 = 0; }
+        else { t.h0 = r / p.segs; t.w0 = (r - t.h0 * p.segs) * BM; }
+        t.q0 = t.live ? (t.n * p.Hin + t.h0) * p.Win + t.w0 : p.Q;      // a dead tile reads zeros only
+        return t;
+    };
     const uint32_t strips_tx = (uint32_t)(p.KH * p.strip_rows) * 128u;
+    // bf16 pairs count both CTAs' strip bytes on the leader's barrier, which its MMA thread waits on; f32 pairs signal
+    // each CTA's own barrier (its converter warps wait there)
+    constexpr bool REMOTE_FULL = CG == 2 && !F32;
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
         if (lane == 0) {
+            if (p.wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");    // inputs may come from the kernel ahead
             int it = 0, cur_ft = -1, epochs = 0;
             bool ok = true;
             auto load_strips = [&](int q0, int cb) {       // one load: the strips of all filter rows
                 const int s = it % p.stages;
                 if (!mbar_wait(empty_bar(s), ((it / p.stages) & 1) ^ 1u, abort_flag)) return false;
-                // (a pair's loads all signal the leader's barriers, which the leader arms for both CTAs)
-                if (cta_rank == 0) mbar_expect_tx(full_bar(s), CG * strips_tx);
-                tma_tile_3d<CG == 2>(strips_addr + s * p.strip_stage_bytes, &map_in,
-                                     CG == 2 ? map_to_cta(full_bar(s), 0) : full_bar(s), cb * 64, q0, 0);
+                if (!REMOTE_FULL || cta_rank == 0) mbar_expect_tx(full_bar(s), (REMOTE_FULL ? CG : 1) * strips_tx);
+                tma_tile_3d<REMOTE_FULL>(strips_addr + s * p.strip_stage_bytes, &map_in,
+                                         REMOTE_FULL ? map_to_cta(full_bar(s), 0) : full_bar(s), cb * (F32 ? 32 : 64), q0, 0);
                 return true;
             };
             for (int item = item0; item < item1 && ok; ++item) {
-                const int ft = item / p.num_q_tiles, qt = item - ft * p.num_q_tiles;
-                const int q0 = (qt * CG + (int)cta_rank) * BM;
+                const int ft = item / p.num_pos_items;
+                const Tile t = decode(item - ft * p.num_pos_items);
                 int cb = 0;
                 if (ft != cur_ft) {
                     // the MMAs of the previous column tile must have finished reading the filter
                     if (epochs > 0 && !mbar_wait(flt_free_bar, (epochs - 1) & 1, abort_flag)) { ok = false; break; }
                     cur_ft = ft;
                     ++epochs;
-                    const int f0 = ft * BN + (int)cta_rank * B_COLS;
-                    for (int kh = 0; kh < p.KH && ok; ++kh) {
-                        const uint32_t fbar = CG == 2 ? map_to_cta(flt_full_bar(kh), 0) : flt_full_bar(kh);
-                        if (cta_rank == 0) mbar_expect_tx(flt_full_bar(kh), CG * p.kbpt * p.KW * flt_block_bytes);
+                    const int f0 = ft * BN + (int)cta_rank * C::B_COLS;
+                    // the first tile's first strips go out ahead of the filter (each TMA instruction costs this thread ~0.3 us)
+                    ok = load_strips(t.q0, 0); ++it; cb = 1;
+                    // one box per channel block: {columns of a sub-tile, channels of a block, B_COLS / sub-tile columns, KW, KH}
+                    const uint32_t load_bytes = (uint32_t)(p.KH * p.KW) * (uint32_t)C::B_COLS * 128u;
+                    if constexpr (F32) {
+                        // raw filter of this CTA's columns into the staging area, which is idle until the first epilogue
+                        // (there is one column tile only: the host side sees to it); the converter warps split it
+                        mbar_expect_tx(flt_full_bar, (uint32_t)p.kbpt * load_bytes);
+                        for (int c2 = 0; c2 < p.kbpt; ++c2)
+                            tma_tile_5d<false>(staging_addr + (uint32_t)c2 * load_bytes, &map_flt, flt_full_bar, 0, c2 * 32, f0 / 32, 0, 0);
+                    } else {
+                        const uint32_t fbar = CG == 2 ? map_to_cta(flt_full_bar, 0) : flt_full_bar;
+                        if (cta_rank == 0) mbar_expect_tx(flt_full_bar, CG * p.kbpt * load_bytes);
                         for (int c2 = 0; c2 < p.kbpt; ++c2) {
-                            const uint32_t dst = flt_addr + ((kh * p.kbpt + c2) * p.KW) * flt_block_bytes;
+                            const uint32_t dst = flt_addr + (uint32_t)c2 * load_bytes;
                             if (p.flt_blocked) {
-                                // box {64 columns, 64 channels, B_COLS/64 column blocks, KW taps, 1}
-                                tma_tile_5d<CG == 2>(dst, &map_flt, fbar, 0, c2 * 64, f0 / 64, 0, kh);
+                                tma_tile_5d<CG == 2>(dst, &map_flt, fbar, 0, c2 * 64, f0 / 64, 0, 0);
                             } else {
-                                for (int kw = 0; kw < p.KW; ++kw)
+                                for (int kh = 0; kh < p.KH; ++kh)
+                                    for (int kw = 0; kw < p.KW; ++kw)
 #pragma unroll
-                                    for (int j = 0; j < B_COLS / 64; ++j) {
-                                        if constexpr (CG == 2) tma_load_4d_cg2(dst + kw * flt_block_bytes + j * SUB_BYTES, &map_flt, fbar, f0 + j * 64, c2 * 64, kw, kh);
-                                        else tma_load_4d(dst + kw * flt_block_bytes + j * SUB_BYTES, &map_flt, fbar, f0 + j * 64, c2 * 64, kw, kh);
-                                    }
+                                        for (int j = 0; j < C::B_COLS / 64; ++j) {
+                                            const uint32_t d2 = dst + (uint32_t)(kh * p.KW + kw) * C::BLOCK_BYTES + j * 8192;
+                                            if constexpr (CG == 2) tma_load_4d_cg2(d2, &map_flt, fbar, f0 + j * 64, c2 * 64, kw, kh);
+                                            else tma_load_4d(d2, &map_flt, fbar, f0 + j * 64, c2 * 64, kw, kh);
+                                        }
                             }
                         }
-                        // the first tile's strips go out right behind the first filter row
-                        if (kh == 0) { ok = load_strips(q0, 0); ++it; cb = 1; }
                     }
                 }
-                for (; cb < p.kbpt && ok; ++cb, ++it) ok = load_strips(q0, cb);
+                for (; cb < p.kbpt && ok; ++cb, ++it) ok = load_strips(t.q0, cb);
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA).  The
         // whole warp walks the loop so that addresses stay warp-uniform; one elected lane issues.
         if (cta_rank == 0) {
-            constexpr uint32_t idesc = make_idesc(BN, CG * BM, false, false, true);   // filter read as stored: N-major
+            constexpr uint32_t idesc = F32 ? make_idesc(BN, CG * BM, true, false, false)     // split tiles are K-major
+                                           : make_idesc(BN, CG * BM, false, false, true);   // bf16 filter read as stored: N-major
             const bool issuer = elect_one();
             auto wait_all = [&](bool passed) { return __all_sync(0xffffffffu, passed) != 0; };
             // arrive, once the MMAs issued so far have finished, on the same barrier of every CTA of the group
@@ -185,123 +294,249 @@ conv_strip_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_const
                     umma_commit_cg2(map_to_cta(bar, 1));
                 }
             };
-            int it = 0, tl = 0, cur_ft = -1, epochs = 0;
-            unsigned flt_ready = 0;      // bit kh: this epoch's filter row kh has landed
+            int it = 0, kbi = 0, tl = 0, cur_ft = -1, epochs = 0;
+            bool flt_ready = false;      // this epoch's filter has landed (f32: has been split)
             bool ok = true;
             for (int item = item0; item < item1 && ok; ++item, ++tl) {
-                const int ft = item / p.num_q_tiles;
-                if (ft != cur_ft) { cur_ft = ft; ++epochs; flt_ready = 0; }
+                const int ft = item / p.num_pos_items;
+                if (ft != cur_ft) { cur_ft = ft; ++epochs; flt_ready = false; }
                 const int buf = tl & 1;
-                if (!wait_all(mbar_wait(acc_empty_bar(buf), ((tl >> 1) & 1) ^ 1u, abort_flag))) { ok = false; break; }
+                if (!wait_all(mbar_wait<CG == 2>(acc_empty_bar(buf), ((tl >> 1) & 1) ^ 1u, abort_flag))) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 uint32_t acc = 0;
                 for (int cb = 0; cb < p.kbpt && ok; ++cb, ++it) {
-                    const int s = it % p.stages;
-                    if (!wait_all(mbar_wait(full_bar(s), (it / p.stages) & 1, abort_flag))) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t strips = strips_addr + s * p.strip_stage_bytes;
-                    for (int kh = 0; kh < p.KH && ok; ++kh) {
-                        if (!(flt_ready >> kh & 1u)) {
-                            if (!wait_all(mbar_wait(flt_full_bar(kh), (epochs - 1) & 1, abort_flag))) { ok = false; break; }
-                            tc_fence_after();
-                            flt_ready |= 1u << kh;
-                        }
-                        for (int kw = 0; kw < p.KW; ++kw) {
-                            // the tap's 128 pixels start kw*dw rows into the strip of filter row kh: same
-                            // K-major layout, start address shifted by whole rows.  The 128-byte swizzle is
-                            // a function of the absolute shared-memory address, for the TMA that wrote the
-                            // strips and for the tensor core alike, so the shifted descriptor (base-offset
-                            // field clear) reads exactly the rows it names.
-                            const uint32_t a_addr = strips + (uint32_t)(kh * p.strip_rows + kw * p.dw) * 128u;
-                            const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024);
-                            const uint32_t b_addr = flt_addr + ((kh * p.kbpt + cb) * p.KW + kw) * flt_block_bytes;
-                            const uint64_t b_desc = make_smem_desc(b_addr, SUB_BYTES, 1024);
-                            if (issuer) {
+                    if constexpr (F32) {
+                        // (a slot's barrier also stands for the filter block its k-block uses: the converter warps split
+                        // that block, during this CTA's first tile, before they signal the slot)
+                        for (int kh = 0; kh < p.KH && ok; ++kh)
+                            for (int kw = 0; kw < p.KW; ++kw, ++kbi) {
+                                const int s = kbi & (A_SLOTS - 1);
+                                if (!wait_all(mbar_wait<CG == 2>(split_full_bar(s), (kbi / A_SLOTS) & 1, abort_flag))) { ok = false; break; }
+                                tc_fence_after();
+                                // filter block hi | lo (K-major, 8-column groups 1024 B apart); input hi | lo in tensor
+                                // memory, 32 columns (k) each, lane = position
+                                const uint32_t blk = flt_addr + (uint32_t)((cb * p.KH + kh) * p.KW + kw) * C::BLOCK_BYTES;
+                                const uint64_t bh = make_smem_desc(blk, 16, 1024);
+                                const uint64_t bl = make_smem_desc(blk + C::B_COLS * 128, 16, 1024);
+                                const uint32_t a_hi = tmem_base + (uint32_t)(C::ACC_COLS + s * 64), a_lo = a_hi + 32;
+                                if (issuer) {
 #pragma unroll
-                                for (int k = 0; k < 4; ++k) {
-                                    if constexpr (CG == 2) umma_bf16_cg2(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc, acc);
-                                    else umma_bf16(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc, acc);
-                                    acc = 1u;
+                                    for (int k = 0; k < 4; ++k) {
+                                        const uint64_t o = (uint64_t)(k * 2);
+                                        if constexpr (CG == 1) {
+                                            umma_tf32_ts(d_tmem, a_lo + k * 8, bh + o, idesc, acc);   // small terms first
+                                            umma_tf32_ts(d_tmem, a_hi + k * 8, bl + o, idesc, 1u);
+                                            umma_tf32_ts(d_tmem, a_hi + k * 8, bh + o, idesc, 1u);
+                                        } else {
+                                            umma_tf32_ts_cg2(d_tmem, a_lo + k * 8, bh + o, idesc, acc);
+                                            umma_tf32_ts_cg2(d_tmem, a_hi + k * 8, bl + o, idesc, 1u);
+                                            umma_tf32_ts_cg2(d_tmem, a_hi + k * 8, bh + o, idesc, 1u);
+                                        }
+                                        acc = 1u;
+                                    }
+                                }
+                                commit_all(split_empty_bar(s));
+                            }
+                    } else {
+                        const int s = it % p.stages;
+                        if (!wait_all(mbar_wait(full_bar(s), (it / p.stages) & 1, abort_flag))) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t strips = strips_addr + s * p.strip_stage_bytes;
+                        if (!flt_ready) {
+                            if (!wait_all(mbar_wait(flt_full_bar, (epochs - 1) & 1, abort_flag))) { ok = false; break; }
+                            tc_fence_after();
+                            flt_ready = true;
+                        }
+                        for (int kh = 0; kh < p.KH; ++kh) {
+                            for (int kw = 0; kw < p.KW; ++kw) {
+                                // the tap's 128 pixels start kw*dw rows into the strip of filter row kh: same
+                                // K-major layout, start address shifted by whole rows.  The 128-byte swizzle is
+                                // a function of the absolute shared-memory address, for the TMA that wrote the
+                                // strips and for the tensor core alike, so the shifted descriptor (base-offset
+                                // field clear) reads exactly the rows it names.
+                                const uint32_t a_addr = strips + (uint32_t)(kh * p.strip_rows + kw * p.dw) * 128u;
+                                const uint64_t a_desc = make_smem_desc(a_addr, 16, 1024);
+                                const uint32_t b_addr = flt_addr + ((cb * p.KH + kh) * p.KW + kw) * C::BLOCK_BYTES;
+                                const uint64_t b_desc = make_smem_desc(b_addr, 8192, 1024);
+                                if (issuer) {
+#pragma unroll
+                                    for (int k = 0; k < 4; ++k) {
+                                        if constexpr (CG == 2) umma_bf16_cg2(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc, acc);
+                                        else umma_bf16(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc, acc);
+                                        acc = 1u;
+                                    }
                                 }
                             }
                         }
+                        if (ok) commit_all(empty_bar(s));
                     }
-                    if (ok) commit_all(empty_bar(s));
                 }
                 if (ok) {
                     commit_all(acc_full_bar(buf));
-                    const bool last_of_ft = item + 1 >= item1 || (item + 1) / p.num_q_tiles != ft;
+                    const bool last_of_ft = item + 1 >= item1 || (item + 1) / p.num_pos_items != ft;
                     if (last_of_ft) commit_all(flt_free_bar);
                 }
             }
         }
+    } else if (warp >= 6) {
+        // ------------------------------------------------------------ converters (f32 only; warps 6 to 21)
+        if constexpr (F32) {
+            const int cw = warp - 6;
+            const int quarter = warp & 3, kpart = cw >> 2;     // TMEM lane quarter this warp may touch; its 8 of the 32 k columns
+            bool ok = item0 < item1;
+            // ---- the filter, once per CTA, block by block during the first tile: raw sub-tiles [32 k][32 columns] (128-byte
+            // rows, as stored) -> hi and lo tiles, K-major ([column][32 k] rows of 128 B in 8-row groups, 16-byte chunk c of
+            // row f at chunk c ^ (f & 7)).  A block (one tap, 32 channels, 64 columns) is sixteen units of an eighth of a
+            // sub-tile (4 k), one per converter warp: lane = column reads down its column (every load one 128-byte row across
+            // the warp) and writes one chunk of its row of both tiles.
+            static_assert(8 * C::B_COLS / 32 == CONVERTER_WARPS, "one filter unit per converter warp");
+            if (ok && !mbar_wait(flt_full_bar, 0, abort_flag)) ok = false;
+            auto split_filter_block = [&](int b) {
+                const int j = cw >> 3, eighth = cw & 7;
+                const float *col = reinterpret_cast<const float *>(staging_gen + (size_t)b * (C::B_COLS * 128) + j * 4096) + eighth * 4 * 32 + lane;
+                uint32_t x[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) x[k] = __float_as_uint(col[k * 32]);
+                const int f = j * 32 + lane;
+                const int off = (f >> 3) * 1024 + (f & 7) * 128 + ((eighth ^ (f & 7)) << 4);
+                uint4 h, l;
+                split4(make_uint4(x[0], x[1], x[2], x[3]), h, l);
+                uint8_t *blk = smem_gen + (size_t)b * C::BLOCK_BYTES;
+                *reinterpret_cast<uint4 *>(blk + off) = h;
+                *reinterpret_cast<uint4 *>(blk + C::B_COLS * 128 + off) = l;
+            };
+            // ---- the strips: per (channel block, tap) this warp's 32 positions x 8 channels -> tensor memory
+            int it = 0, kbi = 0;
+            for (int item = item0; item < item1 && ok; ++item) {
+                for (int cb = 0; cb < p.kbpt && ok; ++cb, ++it) {
+                    const int r = it % p.stages;
+                    if (!mbar_wait(full_bar(r), (it / p.stages) & 1, abort_flag)) { ok = false; break; }
+                    const uint8_t *stage = smem_gen + p.flt_bytes + (size_t)r * p.strip_stage_bytes;
+                    for (int kh = 0; kh < p.KH && ok; ++kh)
+                        for (int kw = 0; kw < p.KW; ++kw, ++kbi) {
+                            const int s = kbi & (A_SLOTS - 1);
+                            if (item == item0) {
+                                // first tile: this k-block's filter block (raw in the staging area) is split on the way
+                                split_filter_block((cb * p.KH + kh) * p.KW + kw);
+                                fence_async_smem();       // generic-proxy writes -> visible to the tensor core's reads
+                            }
+                            // row of the stage that holds this lane's position under tap (kh, kw); TMA wrote the stage
+                            // with the 128-byte swizzle (chunk c of row x at chunk c ^ (x & 7))
+                            const int row = kh * p.strip_rows + kw * p.dw + quarter * 32 + lane;
+                            const uint8_t *rp = stage + (size_t)row * 128;
+                            uint4 a_raw[2];
+#pragma unroll
+                            for (int i = 0; i < 2; ++i)
+                                a_raw[i] = *reinterpret_cast<const uint4 *>(rp + (((kpart * 2 + i) ^ (row & 7)) << 4));
+                            uint32_t hi[8], lo[8];
+#pragma unroll
+                            for (int i = 0; i < 2; ++i) {
+                                uint4 h, l;
+                                split4(a_raw[i], h, l);
+                                hi[4 * i] = h.x; hi[4 * i + 1] = h.y; hi[4 * i + 2] = h.z; hi[4 * i + 3] = h.w;
+                                lo[4 * i] = l.x; lo[4 * i + 1] = l.y; lo[4 * i + 2] = l.z; lo[4 * i + 3] = l.w;
+                            }
+                            // the MMAs that read this slot's tensor-memory columns four k-blocks ago are done
+                            if (!mbar_wait<CG == 2>(split_empty_bar(s), ((kbi / A_SLOTS) & 1) ^ 1u, abort_flag)) { ok = false; break; }
+                            tc_fence_after();
+                            const uint32_t t_hi = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(C::ACC_COLS + s * 64 + kpart * 8);
+                            tmem_st_32x8(t_hi, hi);
+                            tmem_st_32x8(t_hi + 32, lo);
+                            tmem_st_wait();
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) {
+                                if constexpr (CG == 1) mbar_arrive(split_full_bar(s));
+                                else mbar_arrive_cluster(map_to_cta(split_full_bar(s), 0));
+                            }
+                        }
+                    __syncwarp();
+                    if (ok && lane == 0) mbar_arrive(empty_bar(r));          // the raw stage may be refilled
+                }
+            }
+        }
     } else {
-        // ------------------------------------------------------------ epilogue
-        const int quarter = warp & 3;          // TMEM lane quarter this warp may access
-        const int half = (warp - 2) >> 2;      // which half of the tile's columns this warp writes
-        constexpr int CHUNKS = BN / 64;        // 32-column chunks per warp
-        uint8_t *stg = staging_gen + (warp - 2) * 4096;
-        const long long img = (long long)p.Hin * p.Win;
+        // ------------------------------------------------------------ epilogue (warps 2 to 5)
+        // The four warps stage the whole tile in shared memory the way one tensor store reads it: [image row i][32-column
+        // chunk j][w][32 f32], rows of 128 bytes with the 128-byte swizzle (a function of the row's absolute index, as the
+        // TMA unit applies it).  Each warp writes its TMEM lane quarter's positions; one thread then issues the store.
+        const int q = warp & 3;        // TMEM lane quarter this warp may access
+        const bool issuer = warp == 2 && lane == 0;
+        constexpr int CHUNKS = BN / 32;
         int tl = 0;
         bool ok = true;
+        if (p.wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");      // the output may still be in use by the kernel ahead
         for (int item = item0; item < item1 && ok; ++item, ++tl) {
-            const int ft = item / p.num_q_tiles, qt = item - ft * p.num_q_tiles;
-            // this lane's row: padded position q -> (n, h, w) -> its address in O, or null when the
-            // position is not an output
-            const long long q = ((long long)qt * CG + cta_rank) * BM + quarter * 32 + lane;
-            float *row_ptr = nullptr;
-            if (q < p.Q) {
-                const int n = (int)(q / img);
-                const int r = (int)(q - (long long)n * img);
-                const int h = r / p.Win, w = r - h * p.Win;
-                if (h < p.Hout && w < p.Wout) row_ptr = p.O + n * p.o_n + h * p.o_h + w * p.o_w;
+            const int ft = item / p.num_pos_items;
+            const Tile t = decode(item - ft * p.num_pos_items);
+            // this lane's position -> its staging row in chunk 0, or -1 when the position is no output
+            const int pos = q * 32 + lane;
+            int row0 = -1, rows_here = 0;
+            if (t.live) {
+                if (p.segs == 1) {
+                    const int i = pos / p.Win, w = pos - i * p.Win;
+                    rows_here = min(p.rows_per_tile, p.Hout - t.h0);
+                    if (i < rows_here && w < p.Wout) row0 = i * CHUNKS * p.chunk_rows + w;
+                } else {
+                    rows_here = 1;
+                    row0 = pos;          // (positions beyond W_out are clipped by the store)
+                }
             }
             const int buf = tl & 1;
-            if (!mbar_wait(acc_full_bar(buf), (tl >> 1) & 1, abort_flag)) { ok = false; break; }
+            if (!epilogue_all(mbar_wait(acc_full_bar(buf), (tl >> 1) & 1, abort_flag))) { ok = false; break; }
             tc_fence_after();
-            // all of this warp's columns leave TMEM at once; the accumulator buffer is handed back
-            // before the slow part (shared-memory transpose, global stores)
-            uint32_t r[CHUNKS][32];
+            if (issuer) bulk_wait_read<0>();          // the previous tile's store has read the staging area
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            // two chunks leave tensor memory per wait (64 registers in flight)
+#pragma unroll 1
+            for (int j = 0; j < CHUNKS; j += 2) {
+                uint32_t r[2][32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + j * 32), r[0]);
+                tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + (j + 1) * 32), r[1]);
+                tmem_ld_wait();
+                if (row0 >= 0) {
 #pragma unroll
-            for (int j = 0; j < CHUNKS; ++j)
-                tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + (half * CHUNKS + j) * 32), r[j]);
-            tmem_ld_wait();
+                    for (int jj = 0; jj < 2; ++jj) {
+                        const int row = row0 + (j + jj) * p.chunk_rows;
+                        uint8_t *dst = staging_gen + (size_t)row * 128;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)
+                            *reinterpret_cast<uint4 *>(dst + ((c ^ (row & 7)) << 4)) =
+                                make_uint4(r[jj][4 * c], r[jj][4 * c + 1], r[jj][4 * c + 2], r[jj][4 * c + 3]);
+                    }
+                }
+            }
+            // every tcgen05.ld of this buffer has completed: hand it back to the MMA thread
             tc_fence_before();
+            fence_async_smem();
             __syncwarp();
             if (lane == 0) {
                 if constexpr (CG == 1) mbar_arrive(acc_empty_bar(buf));
                 else mbar_arrive_cluster(map_to_cta(acc_empty_bar(buf), 0));
             }
-#pragma unroll
-            for (int j = 0; j < CHUNKS; ++j) {
-                // transpose through shared memory: lane = row writes its 8 chunks rotated by its row
-                // index (conflict-free), then 8 lanes read one row's 128 bytes
-                uint8_t *mine = stg + lane * 128;
-#pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4 *>(mine + (((c + lane) & 7) << 4)) =
-                        make_uint4(r[j][4 * c], r[j][4 * c + 1], r[j][4 * c + 2], r[j][4 * c + 3]);
-                __syncwarp();
-                const int cc = lane & 7;
-                const int col = ft * BN + (half * CHUNKS + j) * 32 + cc * 4;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int rr = 4 * i + (lane >> 3);
-                    float *dst = reinterpret_cast<float *>(__shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(row_ptr), rr));
-                    float4 v = *reinterpret_cast<const float4 *>(stg + rr * 128 + (((cc + rr) & 7) << 4));
-                    if (dst != nullptr && col < p.F) {
-                        float4 *o = reinterpret_cast<float4 *>(dst + col);
-                        if (p.accumulate) {
-                            const float4 old = *o;
-                            v.x += old.x; v.y += old.y; v.z += old.z; v.w += old.w;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (issuer && rows_here > 0) {
+                if (p.blocked_store) {
+                    // box {32 columns, chunk_rows positions, CHUNKS column chunks, R image rows, 1}
+                    if (p.accumulate) tma_reduce_add_5d(&map_out, staging_addr, 0, t.w0, ft * CHUNKS, t.h0, t.n);
+                    else tma_store_5d(&map_out, staging_addr, 0, t.w0, ft * CHUNKS, t.h0, t.n);
+                } else {
+                    for (int i = 0; i < rows_here; ++i)
+                        for (int j = 0; j < CHUNKS; ++j) {
+                            const int x = ft * BN + j * 32;
+                            if (x >= p.F) break;
+                            const uint32_t src = staging_addr + (uint32_t)((i * CHUNKS + j) * p.chunk_rows) * 128u;
+                            if (p.accumulate) tma_reduce_add_4d(&map_out, src, x, t.w0, t.h0 + i, t.n);
+                            else tma_store_4d(&map_out, src, x, t.w0, t.h0 + i, t.n);
                         }
-                        *o = v;
-                    }
                 }
-                __syncwarp();
+                bulk_commit();
             }
         }
+        // the staging area must stay until the last store has read it; the writes themselves are complete
+        // when the grid is
+        if (issuer) bulk_wait_read<0>();
     }
 
     // ---------------------------------------------------------------- teardown
@@ -316,28 +551,51 @@ conv_strip_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_const
     if (warp == 1) {
         tc_fence_after();
         if constexpr (CG == 2)
-            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS) : "memory");
         else
-            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS) : "memory");
     }
 }
 
-std::mutex g_conv_mu;
-bool g_attr_set[3] = {false, false, false};
-int g_attr_device = -1;
-int g_force_single = -1;       // SG_CONV_SINGLE=1 (testing): never use CTA pairs
-
 inline bool mult(int64_t v, int64_t q) { return v % q == 0; }
+
+template <int BN, int CG, bool F32>
+sg_status launch_kernel(const CUtensorMap &map_in, const CUtensorMap &map_flt, const CUtensorMap &map_out, const ConvParams &cp,
+                        int grid, int smem_bytes, int slot, cudaStream_t stream) {
+    using C = ConvCfg<BN, CG, F32>;
+    if (!tensor_ensure_smem_attr(144 + slot, reinterpret_cast<const void *>(conv_strip_kernel<BN, CG, F32>), SMEM_LIMIT + 1024))
+        return SG_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(C::THREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CG;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = cp.wait_prior ? 2 : 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, conv_strip_kernel<BN, CG, F32>, map_in, map_flt, map_out, cp);
+    count_launch();
+    note_kernel(F32 ? "conv_strip_kernel<f32>" : "conv_strip_kernel<bf16>");
+    return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
+}
 
 }  // namespace
 
 sg_status launch_conv_strip(const Problem &p, const void *In, const void *Flt, float *O, cudaStream_t stream) {
-    // ---- eligibility: bf16, unit conv strides, dense pixel pitch, TMA alignment rules ----
-    if (p.spatial_rank == 0 || !p.in_bf16) return SG_ERR_UNSUPPORTED;
+    // ---- eligibility: unit conv strides, dense pixel pitch, TMA alignment rules ----
+    if (p.spatial_rank == 0) return SG_ERR_UNSUPPORTED;
     if (p.sh != 1 || p.sw != 1) return SG_ERR_UNSUPPORTED;
     if (p.i_c != 1 || p.k_f != 1 || p.o_f != 1) return SG_ERR_UNSUPPORTED;
     if (p.KH > MAX_KH || p.KH < 1 || p.KW < 1 || p.KW > 256) return SG_ERR_UNSUPPORTED;
-    const int64_t es = 2;
+    const bool f32 = !p.in_bf16;
+    const int64_t es = f32 ? 4 : 2;
+    const int bkc = 128 / (int)es;                // channels per block
     // the input must be one [N*H_in*W_in, C] matrix with a uniform row pitch
     if (p.Hin > 1 && p.i_h != (int64_t)p.Win * p.i_w) return SG_ERR_UNSUPPORTED;
     if (p.batch > 1 && p.i_n != (int64_t)p.Hin * p.Win * p.i_w) return SG_ERR_UNSUPPORTED;
@@ -348,49 +606,65 @@ sg_status launch_conv_strip(const Problem &p, const void *In, const void *Flt, f
     if (!mult((int64_t)p.C * es, 16) || !mult((int64_t)p.N * es, 16)) return SG_ERR_UNSUPPORTED;   // TMA bounds work in 16-byte units
     if (p.KW > 1 && !mult(p.k_kw * es, 16)) return SG_ERR_UNSUPPORTED;
     if (p.KH > 1 && !mult(p.k_kh * es, 16)) return SG_ERR_UNSUPPORTED;
+    // the output as a 4-D tensor {f, w, h, n} for the tensor stores
     if (!mult(p.o_w, 4) || (p.Ho > 1 && !mult(p.o_h, 4)) || (p.batch > 1 && !mult(p.o_n, 4)) || !mult(p.N, 4)) return SG_ERR_UNSUPPORTED;
+    if (p.o_w < p.N) return SG_ERR_UNSUPPORTED;
     const int64_t pitch_limit = (int64_t)1 << 40;
     if (p.i_w * es >= pitch_limit || p.k_c * es >= pitch_limit) return SG_ERR_UNSUPPORTED;
     const int64_t Q = (int64_t)p.batch * p.Hin * p.Win;
     if (Q > 0x7fffffff - 4096) return SG_ERR_UNSUPPORTED;
-    const int64_t strip_rows = BM + (int64_t)(p.KW - 1) * p.dw;
-    if (strip_rows > 256) return SG_ERR_UNSUPPORTED;
+    if (BM + (int64_t)(p.KW - 1) * p.dw > 256) return SG_ERR_UNSUPPORTED;
     const int64_t shift_rows = (int64_t)p.dh * p.Win;              // input rows between filter rows
     const int64_t q_extent = Q - (int64_t)(p.KH - 1) * shift_rows;
     if (q_extent < 1 || shift_rows * p.i_w * es >= pitch_limit) return SG_ERR_UNSUPPORTED;
-    // wasted positions: the padded domain against the true one
-    if ((double)Q > 1.35 * (double)p.M) return SG_ERR_UNSUPPORTED;
 
-    if (g_force_single < 0) {
-        const char *e = getenv("SG_CONV_SINGLE");
-        g_force_single = e ? atoi(e) : 0;
+    // ---- tiles: whole image rows (W_in <= 128) or segments of a row ----
+    int rows_per_tile = 1, segs = 1, chunk_rows = BM;
+    if (p.Win <= BM) {
+        rows_per_tile = std::min(BM / p.Win, p.Ho);
+        chunk_rows = p.Wo;
+    } else {
+        segs = (p.Wo + BM - 1) / BM;
     }
-    // 128 columns on a CTA pair when there are more than 64 columns and at least two 128-position
-    // tiles (each CTA keeps 64 columns of the filter); otherwise one CTA with 64 or 128 columns
+    // rows of a strip that feed outputs (the tensor core reads 128 rows per tap whatever lies behind them in shared
+    // memory; what it makes of the rest lands in positions that are dropped)
+    const int64_t strip_rows = (p.Win <= BM ? (int64_t)rows_per_tile * p.Win : BM) + (int64_t)(p.KW - 1) * p.dw;
+    const int64_t tiles_per_image = p.Win <= BM ? (p.Ho + rows_per_tile - 1) / rows_per_tile : (int64_t)p.Ho * segs;
+    const int64_t num_tiles = (int64_t)p.batch * tiles_per_image;
+    if (num_tiles > 0x3fffffff) return SG_ERR_UNSUPPORTED;
+    // tensor-core rows that compute outputs: below half, the im2col kernel (whose tile rows are all outputs) is the better one
+    if ((double)p.M < 0.5 * (double)num_tiles * BM) return SG_ERR_UNSUPPORTED;
+
+    int dev = 0, num_sms = 0, pdl = -1, single = 0;
+    if (!tensor_device_info(&dev, &num_sms, &pdl, &single)) return SG_ERR_CUDA;
+
+    // 128 columns on a CTA pair when there are more than 64 columns and at least two tiles (each CTA keeps 64 columns of
+    // the filter); otherwise one CTA with 64 or 128 columns.  f32: the split filter (hi and lo) of the one column tile
+    // must fit beside a ring whose top can stage the raw filter.
     const int BN = p.N > 64 ? 128 : 64;
-    const int kbpt = (p.C + 63) / 64;
+    const int kbpt = (p.C + bkc - 1) / bkc;
     const int strip_stage_bytes = (int)(((int64_t)p.KH * strip_rows * 128 + 1023) / 1024) * 1024;   // KH strips per stage
-    int CG = (BN == 128 && Q > BM && g_force_single == 0) ? 2 : 1;
-    int64_t flt_bytes = 0, fixed = 0;
+    int CG = (BN == 128 && num_tiles > 1 && single == 0) ? 2 : 1;
+    if (f32 && (p.N > BN || (BN == 128 && CG == 1))) return SG_ERR_UNSUPPORTED;
+    int64_t flt_bytes = 0, fixed = 0, staging_bytes = 0;
     int stages = 0;
     for (;; CG = 1) {
-        flt_bytes = (int64_t)p.KH * p.KW * kbpt * (BN / CG) * 128;
-        fixed = flt_bytes + STAGING_BYTES + 256;
+        flt_bytes = (int64_t)p.KH * p.KW * kbpt * (BN / CG) * 128 * (f32 ? 2 : 1);
+        // the staged output tile: [image row][32-column chunk][position][32 f32]; f32: the raw filter (half the size of
+        // the split one) waits there to be split
+        staging_bytes = (int64_t)rows_per_tile * (BN / 32) * chunk_rows * 128;
+        if (f32 && staging_bytes < flt_bytes / 2) staging_bytes = flt_bytes / 2;
+        staging_bytes = (staging_bytes + 1023) / 1024 * 1024;
+        fixed = flt_bytes + staging_bytes + 512;
         stages = (int)((SMEM_LIMIT - fixed) / strip_stage_bytes);
         if (stages > MAX_STAGES) stages = MAX_STAGES;
-        if (stages >= 2 || CG == 1) break;
+        if (stages >= 2 || CG == 1 || f32) break;
     }
     if (stages < 2) return SG_ERR_UNSUPPORTED;
     const int smem_bytes = (int)(fixed + (int64_t)stages * strip_stage_bytes + 1024);
 
-    std::lock_guard<std::mutex> lock(g_conv_mu);
-    int num_sms = 0;
-    if (!tensor_driver_ready(&num_sms)) return SG_ERR_CUDA;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev != g_attr_device) { g_attr_set[0] = g_attr_set[1] = g_attr_set[2] = false; g_attr_device = dev; }
-
-    alignas(64) CUtensorMap map_in, map_flt;
+    alignas(64) CUtensorMap map_in, map_flt, map_out;
+    const CUtensorMapDataType in_type = f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     {
         // overlapping 3-D view: {channel, position, filter row}; a step in the third dimension is
         // dh*W_in positions.  The position extent stops (KH-1)*dh*W_in short of the end so that no
@@ -398,71 +672,84 @@ sg_status launch_conv_strip(const Problem &p, const void *In, const void *Flt, f
         // with h >= H_out of the last image, which are not outputs.
         cuuint64_t dims[3] = {(cuuint64_t)p.C, (cuuint64_t)q_extent, (cuuint64_t)p.KH};
         cuuint64_t strides[2] = {(cuuint64_t)(p.i_w * es), (cuuint64_t)((p.KH > 1 ? shift_rows : Q) * p.i_w * es)};
-        cuuint32_t box[3] = {64, (cuuint32_t)strip_rows, (cuuint32_t)p.KH};
+        cuuint32_t box[3] = {(cuuint32_t)bkc, (cuuint32_t)strip_rows, (cuuint32_t)p.KH};
         if (strides[1] >= ((cuuint64_t)1 << 40)) return SG_ERR_UNSUPPORTED;
-        if (!tensor_encode_tiled(&map_in, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(In), dims, strides, box,
+        if (!tensor_encode_tiled(&map_in, in_type, 3, const_cast<void *>(In), dims, strides, box,
                                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B)) return SG_ERR_UNSUPPORTED;
     }
     const int64_t s_kw = p.KW > 1 ? p.k_kw : (int64_t)p.C * p.k_c;
     const int64_t s_kh = p.KH > 1 ? p.k_kh : (int64_t)p.KW * s_kw;
-    const bool flt_blocked = p.N % 64 == 0;     // whole 64-column blocks: one box per filter row and channel block
+    const int sub = f32 ? 32 : 64;               // filter columns per 128-byte row
+    const bool flt_blocked = p.N % sub == 0;     // whole column blocks: one box per filter row and channel block
+    if (f32 && !flt_blocked) return SG_ERR_UNSUPPORTED;
     if (flt_blocked) {
-        // {column in block, channel, column block, kw, kh}, box {64, 64, B_COLS/64, KW, 1}
-        cuuint64_t dims[5] = {64, (cuuint64_t)p.C, (cuuint64_t)(p.N / 64), (cuuint64_t)p.KW, (cuuint64_t)p.KH};
+        // {column in block, channel, column block, kw, kh}, box {sub, channels per block, B_COLS/sub, KW, KH}; bf16 lands as
+        // the tensor core reads it (128-byte swizzle), f32 as stored (the converter warps transpose it)
+        cuuint64_t dims[5] = {(cuuint64_t)sub, (cuuint64_t)p.C, (cuuint64_t)(p.N / sub), (cuuint64_t)p.KW, (cuuint64_t)p.KH};
         cuuint64_t strides[4] = {(cuuint64_t)(p.k_c * es), 128, (cuuint64_t)(s_kw * es), (cuuint64_t)(s_kh * es)};
-        cuuint32_t box[5] = {64, 64, (cuuint32_t)(BN / CG / 64), (cuuint32_t)p.KW, 1};
-        if (!tensor_encode_tiled(&map_flt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(Flt), dims, strides, box,
-                                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B)) return SG_ERR_UNSUPPORTED;
+        cuuint32_t box[5] = {(cuuint32_t)sub, (cuuint32_t)bkc, (cuuint32_t)(BN / CG / sub), (cuuint32_t)p.KW, (cuuint32_t)p.KH};
+        if (!tensor_encode_tiled(&map_flt, in_type, 5, const_cast<void *>(Flt), dims, strides, box,
+                                 f32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B))
+            return SG_ERR_UNSUPPORTED;
     } else {
         cuuint64_t dims[4] = {(cuuint64_t)p.N, (cuuint64_t)p.C, (cuuint64_t)p.KW, (cuuint64_t)p.KH};
         cuuint64_t strides[3] = {(cuuint64_t)(p.k_c * es), (cuuint64_t)(s_kw * es), (cuuint64_t)(s_kh * es)};
         cuuint32_t box[4] = {64, 64, 1, 1};
-        if (!tensor_encode_tiled(&map_flt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(Flt), dims, strides, box,
+        if (!tensor_encode_tiled(&map_flt, in_type, 4, const_cast<void *>(Flt), dims, strides, box,
                                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B)) return SG_ERR_UNSUPPORTED;
+    }
+    const bool blocked_store = p.N % 32 == 0;
+    {
+        // A dimension of extent 1 gets the dense stride (its own is not used and may be 0).
+        const int64_t s_w = p.o_w, s_h = p.Ho > 1 ? p.o_h : (int64_t)p.Wo * s_w, s_n = p.batch > 1 ? p.o_n : (int64_t)p.Ho * s_h;
+        if (s_w * 4 >= pitch_limit || s_h * 4 >= pitch_limit || s_n * 4 >= pitch_limit || s_h % 4 != 0 || s_n % 4 != 0) return SG_ERR_UNSUPPORTED;
+        bool ok;
+        if (blocked_store) {
+            // {f in chunk, w, chunk, h, n}: one box {32, positions of a row (segment), chunks of the tile, rows of the tile, 1}
+            // is the whole tile
+            cuuint64_t dims[5] = {32, (cuuint64_t)p.Wo, (cuuint64_t)(p.N / 32), (cuuint64_t)p.Ho, (cuuint64_t)p.batch};
+            cuuint64_t strides[4] = {(cuuint64_t)(s_w * 4), 128, (cuuint64_t)(s_h * 4), (cuuint64_t)(s_n * 4)};
+            cuuint32_t box[5] = {32, (cuuint32_t)chunk_rows, (cuuint32_t)(BN / 32), (cuuint32_t)rows_per_tile, 1};
+            ok = tensor_encode_tiled(&map_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, O, dims, strides, box,
+                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE);
+        } else {
+            // {f, w, h, n}; one store = 32 columns x the positions of one image row (or one 128-position segment)
+            cuuint64_t dims[4] = {(cuuint64_t)p.N, (cuuint64_t)p.Wo, (cuuint64_t)p.Ho, (cuuint64_t)p.batch};
+            cuuint64_t strides[3] = {(cuuint64_t)(s_w * 4), (cuuint64_t)(s_h * 4), (cuuint64_t)(s_n * 4)};
+            cuuint32_t box[4] = {32, (cuuint32_t)chunk_rows, 1, 1};
+            ok = tensor_encode_tiled(&map_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, O, dims, strides, box,
+                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE);
+        }
+        if (!ok) return SG_ERR_UNSUPPORTED;
     }
 
     ConvParams cp{};
     cp.Q = (int)Q;
-    cp.num_q_tiles = (int)((Q + CG * BM - 1) / (CG * BM));
+    cp.num_tiles = (int)num_tiles;
+    cp.num_pos_items = (int)((num_tiles + CG - 1) / CG);
     cp.num_f_tiles = (p.N + BN - 1) / BN;
-    const int total = cp.num_q_tiles * cp.num_f_tiles;
+    const int total = cp.num_pos_items * cp.num_f_tiles;
     const int groups_max = num_sms / CG;
     const int groups = total < groups_max ? total : groups_max;
-    cp.items_per_group = (total + groups - 1) / groups;
-    const int grid = CG * ((total + cp.items_per_group - 1) / cp.items_per_group);
+    const int grid = CG * groups;
+    cp.N = p.batch; cp.Hin = p.Hin; cp.Win = p.Win; cp.Hout = p.Ho; cp.Wout = p.Wo;
     cp.KH = p.KH; cp.KW = p.KW; cp.kbpt = kbpt;
-    cp.Hin = p.Hin; cp.Win = p.Win; cp.Hout = p.Ho; cp.Wout = p.Wo;
     cp.dw = p.dw;
+    cp.rows_per_tile = rows_per_tile; cp.segs = segs; cp.tiles_per_image = (int)tiles_per_image;
+    cp.chunk_rows = chunk_rows; cp.staging_bytes = (int)staging_bytes; cp.blocked_store = blocked_store ? 1 : 0;
     cp.strip_rows = (int)strip_rows; cp.strip_stage_bytes = strip_stage_bytes; cp.stages = stages;
     cp.flt_bytes = (int)flt_bytes;
     cp.flt_blocked = flt_blocked ? 1 : 0;
     cp.F = p.N; cp.accumulate = p.accumulate;
-    cp.o_n = p.o_n; cp.o_h = p.o_h; cp.o_w = p.o_w; cp.O = O;
+    cp.wait_prior = pdl == 0 ? 0 : 1;
 
-    void (*kernel)(const CUtensorMap, const CUtensorMap, const ConvParams) =
-        BN == 64 ? conv_strip_kernel<64, 1> : (CG == 2 ? conv_strip_kernel<128, 2> : conv_strip_kernel<128, 1>);
-    const int slot = BN == 64 ? 0 : (CG == 2 ? 2 : 1);
-    if (!g_attr_set[slot]) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT + 1024) != cudaSuccess)
-            return SG_ERR_CUDA;
-        g_attr_set[slot] = true;
+    if (f32) {
+        if (BN == 64) return launch_kernel<64, 1, true>(map_in, map_flt, map_out, cp, grid, smem_bytes, 3, stream);
+        return launch_kernel<128, 2, true>(map_in, map_flt, map_out, cp, grid, smem_bytes, 4, stream);
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid, 1, 1);
-    cfg.blockDim = dim3(CONV_THREADS, 1, 1);
-    cfg.dynamicSmemBytes = smem_bytes;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = CG;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, map_in, map_flt, cp);
-    count_launch();
-    note_kernel("conv_strip_kernel");
-    return e == cudaSuccess ? SG_OK : SG_ERR_CUDA;
+    if (BN == 64) return launch_kernel<64, 1, false>(map_in, map_flt, map_out, cp, grid, smem_bytes, 0, stream);
+    if (CG == 2) return launch_kernel<128, 2, false>(map_in, map_flt, map_out, cp, grid, smem_bytes, 2, stream);
+    return launch_kernel<128, 1, false>(map_in, map_flt, map_out, cp, grid, smem_bytes, 1, stream);
 }
 
 sg_status conv_read_status(cudaStream_t stream) { return read_status_word(stream); }

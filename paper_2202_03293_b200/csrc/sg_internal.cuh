@@ -47,6 +47,11 @@ cudaError_t launch_wait_timeout_selftest(long long budget_cycles, cudaStream_t s
 // current device is usable (and its SM count), and a tiled tensor-map encoder (interleave none,
 // element strides 1, out-of-bounds elements read as zero).  Call with no library lock held.
 bool tensor_driver_ready(int *num_sms);
+// The current device's index and SM count plus two test switches (SG_TC_PDL, SG_CONV_SINGLE); false when the device is unusable.
+bool tensor_device_info(int *device, int *num_sms, int *pdl, int *conv_single);
+// Raises a kernel's dynamic shared-memory limit once per device; `slot` (144..159 for callers outside the GEMM file)
+// names the kernel instantiation.
+bool tensor_ensure_smem_attr(int slot, const void *kernel, int bytes);
 bool tensor_encode_tiled(CUtensorMap *map, CUtensorMapDataType type, int rank, void *base, const cuuint64_t *dims,
                          const cuuint64_t *strides, const cuuint32_t *box, CUtensorMapSwizzle swizzle,
                          CUtensorMapL2promotion promotion);
@@ -56,6 +61,7 @@ sg_status launch_conv_strip(const Problem &p, const void *In, const void *Flt, f
 sg_status conv_read_status(cudaStream_t stream);
 void tensor_set_tile_override(int bn, int cg, int splits);
 void tensor_last_choice(int out[3]);
+void tensor_map_cache_stats(long long out[2]);     // {hits, misses} since the library was loaded
 void tensor_last_stream_k(int out[2]);
 // Reads and clears the current device's status word (written by kernels whose bounded
 // waits expire); the caller has already synchronised the stream.

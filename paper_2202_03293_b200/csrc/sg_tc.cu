@@ -36,6 +36,9 @@
 // drains its copies, frees its TMEM and returns.
 #include <cuda.h>
 
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
 #include <mutex>
 #include <type_traits>
 
@@ -68,8 +71,10 @@ struct TcParams {
     int b_blocked;       // 1: the filter map is blocked by sub-tile columns: one TMA load fetches the whole filter tile
     int sk_first_tile;   // stream-K tail: tiles from this one on are not dealt out whole; their k-blocks, taken as one
     int sk_units;        //   sequence, are cut into equal runs of `sk_units` k-blocks, one run per CTA (or pair); 0 = no tail
-    int wait_prior;      // 1: the launch may start before the clearing kernel ahead of it has finished (programmatic
-                         //    dependent launch): nothing may be added into the output before griddepcontrol.wait
+    int wait_prior;      // the launch may start before the kernel ahead of it in the stream has finished (programmatic
+                         // dependent launch).  1: that kernel is this library's clearing kernel, which touches only the
+                         // output: the stores wait for it (griddepcontrol.wait), the loads need not.  2: it is any
+                         // kernel: loads and stores both wait.  0: an ordinary launch.
 };
 
 // 3xTF32 split of four f32 words.  hi = x rounded to the nearest tf32 value (10 mantissa bits;
@@ -198,6 +203,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_gen + 8 * 24 + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // A launch behind this one that asked for it may start now: its CTAs take an SM as soon as one of ours leaves it
+    // and set themselves up while the rest of this grid drains; they touch global memory only after this grid is done.
+    asm volatile("griddepcontrol.launch_dependents;");
     if (threadIdx.x == 0) { prefetch_tensormap(&map_in); prefetch_tensormap(&map_flt); prefetch_tensormap(&map_out); }
     // In a pair, CTA 0 (the leader) issues the MMAs; both CTAs produce and both run epilogues.
     const uint32_t cta_rank = CG == 2 ? cluster_ctarank() : 0u;
@@ -278,6 +286,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         // input tiles, the last warp the filter tiles; both arm the stage's barrier for their bytes
         if (lane == 0) {
             const bool input_side = warp == 0;
+            // the operands may be the output of the kernel ahead of this one
+            if (p.wait_prior == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
             int it = 0;   // k-block counter across all of this CTA's tiles
             bool ok = true;
             Cursor cur{0, sk_u0};
@@ -603,8 +613,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         auto epi_sync = [] { asm volatile("bar.sync 1, 128;" ::: "memory"); };
         int tl = 0, chunk_count = 0;
         bool ok = true;
-        // a split reduction that overwrites follows a kernel that clears the output: this grid was allowed to start (and
-        // to run its whole first reduction) beside it, but the first reduce-add must see the cleared output
+        // This grid may have started beside the kernel ahead of it.  Behind a clearing kernel the whole first reduction
+        // runs meanwhile, but the first reduce-add must see the cleared output; behind any other kernel the output may
+        // still be in use (read or written) until that kernel has finished.
         if (p.wait_prior) asm volatile("griddepcontrol.wait;" ::: "memory");
         Cursor cur{0, sk_u0};
         int tile, kb0, kb1, add;
@@ -700,44 +711,193 @@ typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_
                                    const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-struct Driver {
-    EncodeTiledFn tiled = nullptr;
-    EncodeIm2colFn im2col = nullptr;
+// ---- process-wide host state -----------------------------------------------------------------
+// g_mu guards the driver entry points, the per-device records and the overrides; it is held for a few loads and stores,
+// never across a tensor-map encode or a launch.  The tensor-map cache has a lock of its own.
+constexpr int kMaxDevices = 64;
+constexpr int kAttrSlots = 160;
+struct DeviceState {
+    bool ready = false;
     int num_sms = 0;
-    int device = -1;
-    bool attr_set[128] = {};
-    bool ok = false;
+    bool attr_set[kAttrSlots] = {};      // shared-memory limit raised for kernel instantiation `slot` on this device
+};
+struct Overrides {
+    bool env_read = false;
+    int bn = 0;      // tile width forced by SG_TC_BN or sg_set_tile_override (0: automatic)
+    int cg = 0;      // CTAs per tile (0: automatic)
+    int split = 0;   // k ranges per tile (0: automatic)
+    int kps = 0;     // SG_TC_KPS=1 (testing): one k-block per stage everywhere
+    int sk = -1;     // SG_TC_SK (testing): 0 = never cut the last wave into a stream-K tail, 2 = whenever it is possible
+    int ta = -1;     // SG_TC_TA (testing): 0 never, 1 always keep the split f32 input tile in tensor memory
+    int pdl = -1;    // SG_TC_PDL (testing): 0 = launches never overlap the tail of the kernel ahead of them
+    int conv_single = 0;   // SG_CONV_SINGLE=1 (testing): the stride-1 convolution kernel never uses CTA pairs
 };
 std::mutex g_mu;
-Driver g_drv;
-int g_bn_override = -1;   // tile width forced by SG_TC_BN or sg_set_tile_override (-1: not read yet; 0: automatic)
-int g_cg_override = 0;    // CTAs per tile (0: automatic)
-int g_split_override = 0; // k ranges per tile (0: automatic)
-int g_kps_override = 0;   // SG_TC_KPS=1 (testing): one k-block per stage everywhere
-int g_last_sk[2] = {-1, 0};
-int g_sk_override = -1;   // SG_TC_SK (testing): 0 = never cut the last wave into a stream-K tail, 2 = whenever it is possible
-int g_ta_override = -1;   // SG_TC_TA (testing): 0 never, 1 always keep the split f32 input tile in tensor memory
-int g_last_choice[3] = {0, 0, 0};
+EncodeTiledFn g_encode_tiled = nullptr;
+EncodeIm2colFn g_encode_im2col = nullptr;
+DeviceState g_dev[kMaxDevices];
+Overrides g_ov;
+thread_local int t_last_sk[2] = {-1, 0};
+thread_local int t_last_choice[3] = {0, 0, 0};
 
-bool init_driver() {
+// The environment switches are read once per process (caller holds g_mu).
+void read_env_locked() {
+    if (g_ov.env_read) return;
+    auto env = [](const char *name, int dflt) { const char *e = getenv(name); return e ? atoi(e) : dflt; };
+    g_ov.bn = env("SG_TC_BN", 0); g_ov.cg = env("SG_TC_CG", 0); g_ov.split = env("SG_TC_SPLIT", 0);
+    g_ov.kps = env("SG_TC_KPS", 0); g_ov.ta = env("SG_TC_TA", -1); g_ov.sk = env("SG_TC_SK", -1);
+    g_ov.pdl = env("SG_TC_PDL", -1);
+    g_ov.conv_single = env("SG_CONV_SINGLE", 0);
+    g_ov.env_read = true;
+}
+
+// The current device's record (created at the first call on that device), or nullptr when the device is unusable.
+// Fills a snapshot of the overrides when asked for.
+const DeviceState *device_state(int *device_out, Overrides *ov_out) {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return false;
-    if (g_drv.ok && g_drv.device == dev) return true;
-    g_drv = Driver{};   // first use, or the caller switched devices: per-device state starts over
-    void *fn = nullptr;
-    cudaDriverEntryPointQueryResult qr;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess || !fn) return false;
-    g_drv.tiled = reinterpret_cast<EncodeTiledFn>(fn);
-    fn = nullptr;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn, cudaEnableDefault, &qr) != cudaSuccess || !fn) return false;
-    g_drv.im2col = reinterpret_cast<EncodeIm2colFn>(fn);
-    if (cudaDeviceGetAttribute(&g_drv.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
-    int major = 0;
-    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
-    if (major != 10) return false;
-    g_drv.device = dev;
-    g_drv.ok = true;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_encode_tiled || !g_encode_im2col) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess || !fn) return nullptr;
+        g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+        fn = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn, cudaEnableDefault, &qr) != cudaSuccess || !fn) return nullptr;
+        g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(fn);
+    }
+    DeviceState &d = g_dev[dev];
+    if (!d.ready) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess || major != 10) return nullptr;
+        d.ready = true;
+    }
+    read_env_locked();
+    if (device_out) *device_out = dev;
+    if (ov_out) *ov_out = g_ov;
+    return &d;
+}
+
+// Raises a kernel's dynamic shared-memory limit once per device and instantiation.
+template <typename Kernel>
+bool ensure_smem_attr(int dev, int slot, Kernel kernel, int bytes) {
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (g_dev[dev].attr_set[slot]) return true;
+    }
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    std::lock_guard<std::mutex> lock(g_mu);
+    g_dev[dev].attr_set[slot] = true;
     return true;
+}
+
+// ---- tensor-map cache -------------------------------------------------------------------------
+// Encoding a tensor map is a driver call of about a microsecond, and a call needs three.  A map depends only on the
+// address and geometry it describes (never on the memory's contents), so encoded maps are kept in a bounded,
+// process-wide table keyed by everything that goes into the encode: device, base pointer, element type, extents, byte
+// strides, box, traversal strides, im2col corners, swizzle and L2 promotion.  4-way buckets, oldest entry of a full bucket
+// replaced; sg_shutdown drops the table.
+struct MapKey {
+    uint64_t base;
+    uint64_t dims[5];
+    uint64_t strides[4];
+    uint32_t box[5];
+    uint32_t trav[5];
+    int32_t lower[3], upper[3];
+    uint32_t rank, type, swizzle, promotion, im2col, channels_per_pixel, pixels_per_column, device;
+};
+struct MapSlot {
+    MapKey key;
+    CUtensorMap map;
+    uint32_t used, age;
+};
+constexpr uint32_t kCacheBuckets = 512, kCacheWays = 4;
+std::mutex g_cache_mu;
+MapSlot *g_cache = nullptr;
+uint32_t g_cache_clock = 0;
+std::atomic<long long> g_cache_hits{0}, g_cache_misses{0};
+
+inline uint64_t hash_key(const MapKey &k) {
+    const uint64_t *w = reinterpret_cast<const uint64_t *>(&k);
+    uint64_t h = 0x9E3779B97F4A7C15ull;
+    for (size_t i = 0; i < sizeof(MapKey) / 8; ++i) { h ^= w[i]; h *= 0xff51afd7ed558ccdull; h ^= h >> 32; }
+    return h;
+}
+static_assert(sizeof(MapKey) % 8 == 0, "MapKey is hashed in 64-bit words");
+
+// Looks the key up; on a miss calls `encode` (outside the lock) and stores the result.
+template <typename Encode>
+bool cached_map(const MapKey &key, CUtensorMap *out, Encode encode) {
+    const uint32_t bucket = (uint32_t)(hash_key(key) % kCacheBuckets) * kCacheWays;
+    {
+        std::lock_guard<std::mutex> lock(g_cache_mu);
+        if (g_cache) {
+            for (uint32_t w = 0; w < kCacheWays; ++w) {
+                MapSlot &sl = g_cache[bucket + w];
+                if (sl.used && memcmp(&sl.key, &key, sizeof(MapKey)) == 0) {
+                    *out = sl.map;
+                    sl.age = ++g_cache_clock;
+                    g_cache_hits.fetch_add(1, std::memory_order_relaxed);
+                    return true;
+                }
+            }
+        }
+    }
+    if (!encode(out)) return false;
+    g_cache_misses.fetch_add(1, std::memory_order_relaxed);
+    std::lock_guard<std::mutex> lock(g_cache_mu);
+    if (!g_cache) {
+        g_cache = static_cast<MapSlot *>(calloc((size_t)kCacheBuckets * kCacheWays, sizeof(MapSlot)));
+        if (!g_cache) return true;      // no table: the map is still good
+    }
+    uint32_t victim = 0, oldest = 0xffffffffu;
+    for (uint32_t w = 0; w < kCacheWays; ++w) {
+        const MapSlot &sl = g_cache[bucket + w];
+        if (!sl.used) { victim = w; break; }
+        if (sl.age < oldest) { oldest = sl.age; victim = w; }
+    }
+    MapSlot &sl = g_cache[bucket + victim];
+    sl.key = key; sl.map = *out; sl.used = 1; sl.age = ++g_cache_clock;
+    return true;
+}
+
+bool encode_tiled_cached(CUtensorMap *map, int device, CUtensorMapDataType type, int rank, const void *base, const cuuint64_t *dims,
+                         const cuuint64_t *strides, const cuuint32_t *box, CUtensorMapSwizzle swizzle,
+                         CUtensorMapL2promotion promotion) {
+    MapKey k;
+    memset(&k, 0, sizeof(k));
+    k.base = reinterpret_cast<uint64_t>(base);
+    for (int i = 0; i < rank; ++i) { k.dims[i] = dims[i]; k.box[i] = box[i]; k.trav[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) k.strides[i] = strides[i];
+    k.rank = (uint32_t)rank; k.type = (uint32_t)type; k.swizzle = (uint32_t)swizzle; k.promotion = (uint32_t)promotion;
+    k.device = (uint32_t)device;
+    EncodeTiledFn fn = g_encode_tiled;      // set before any caller gets here (device_state)
+    return cached_map(k, map, [&](CUtensorMap *m) {
+        const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+        return fn(m, type, (cuuint32_t)rank, const_cast<void *>(base), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
+                  promotion, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
+}
+
+bool encode_im2col_cached(CUtensorMap *map, int device, CUtensorMapDataType type, int rank, const void *base, const cuuint64_t *dims,
+                          const cuuint64_t *strides, const int *lower, const int *upper, cuuint32_t channels_per_pixel,
+                          cuuint32_t pixels_per_column, const cuuint32_t *trav) {
+    MapKey k;
+    memset(&k, 0, sizeof(k));
+    k.base = reinterpret_cast<uint64_t>(base);
+    for (int i = 0; i < rank; ++i) { k.dims[i] = dims[i]; k.trav[i] = trav[i]; }
+    for (int i = 0; i + 1 < rank; ++i) k.strides[i] = strides[i];
+    for (int i = 0; i + 2 < rank; ++i) { k.lower[i] = lower[i]; k.upper[i] = upper[i]; }
+    k.rank = (uint32_t)rank; k.type = (uint32_t)type; k.swizzle = (uint32_t)CU_TENSOR_MAP_SWIZZLE_128B;
+    k.promotion = (uint32_t)CU_TENSOR_MAP_L2_PROMOTION_L2_128B; k.im2col = 1;
+    k.channels_per_pixel = channels_per_pixel; k.pixels_per_column = pixels_per_column; k.device = (uint32_t)device;
+    EncodeIm2colFn fn = g_encode_im2col;
+    return cached_map(k, map, [&](CUtensorMap *m) {
+        return fn(m, type, (cuuint32_t)rank, const_cast<void *>(base), dims, strides, lower, upper, channels_per_pixel, pixels_per_column,
+                  trav, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    });
 }
 
 inline bool mult(int64_t v, int64_t q) { return v % q == 0; }
@@ -773,31 +933,34 @@ double estimate_ns(const Variant &v, bool f32, int64_t tiles, int64_t groups, in
     return t;
 }
 
+struct LaunchCtx {
+    const DeviceState *dev;
+    int device;
+    cudaStream_t stream;
+};
+
 template <int BN, int CG, bool F32, int KPS, int LAY = 0>
 sg_status launch_variant(const CUtensorMap &mi, const CUtensorMap &mf, const CUtensorMap &mo, TcParams tp, int M, int N,
-                         int slot, cudaStream_t stream) {
+                         int slot, const LaunchCtx &ctx) {
   if constexpr ((F32 && BN == 256 && CG == 1) || (KPS == 2 && (F32 || (BN == 256 && CG == 1))) ||
                 ((LAY & 3) != 0 && (KPS != 1 || (BN == 256 && CG == 1) || (BN == 128 && CG == 2))) ||
                 ((LAY & 4) != 0 && !F32)) {
     return SG_ERR_INTERNAL;   // the split slots of a 128 x 256 f32 tile do not fit beside a TMA ring
   } else {
     using C = Cfg<BN, CG, F32, KPS, (LAY & 4) != 0>;
-    if (!g_drv.attr_set[slot]) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, CG, F32, KPS, LAY>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
-            return SG_ERR_CUDA;
-        g_drv.attr_set[slot] = true;
-    }
+    static_assert(5 * 3 * 8 <= kAttrSlots, "attribute slots");
+    if (!ensure_smem_attr(ctx.device, slot, tc_gemm_kernel<BN, CG, F32, KPS, LAY>, C::SMEM_BYTES)) return SG_ERR_CUDA;
     tp.num_m_tiles = (M + CG * BM - 1) / (CG * BM);
     tp.num_n_tiles = (N + BN - 1) / BN;
     const int tiles = tp.num_m_tiles * tp.num_n_tiles * tp.splits;
-    const int groups = g_drv.num_sms / CG;
+    const int groups = ctx.dev->num_sms / CG;
     // (a stream-K tail deals its runs to every group, also when there are fewer tiles than groups)
     const int grid = CG * ((tiles < groups && tp.sk_units == 0) ? tiles : groups);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
     cfg.blockDim = dim3(C::THREADS, 1, 1);
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
-    cfg.stream = stream;
+    cfg.stream = ctx.stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = CG;
@@ -847,22 +1010,11 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     const int64_t pitch_limit = (int64_t)1 << 40;
     if (a_pitch * es >= pitch_limit || b_pitch * es >= pitch_limit || p.o_w * 4 >= pitch_limit) return SG_ERR_UNSUPPORTED;
 
-    std::lock_guard<std::mutex> lock(g_mu);
-    if (!init_driver()) return SG_ERR_CUDA;
-    if (g_bn_override < 0) {
-        const char *e = getenv("SG_TC_BN");
-        g_bn_override = e ? atoi(e) : 0;
-        e = getenv("SG_TC_CG");
-        g_cg_override = e ? atoi(e) : 0;
-        e = getenv("SG_TC_SPLIT");
-        g_split_override = e ? atoi(e) : 0;
-        e = getenv("SG_TC_KPS");
-        g_kps_override = e ? atoi(e) : 0;
-        e = getenv("SG_TC_TA");
-        g_ta_override = e ? atoi(e) : -1;
-        e = getenv("SG_TC_SK");
-        g_sk_override = e ? atoi(e) : -1;
-    }
+    LaunchCtx ctx{nullptr, 0, stream};
+    Overrides ov;
+    ctx.dev = device_state(&ctx.device, &ov);
+    if (!ctx.dev) return SG_ERR_CUDA;
+    const int num_sms = ctx.dev->num_sms;
 
     alignas(64) CUtensorMap map_in, map_flt, map_out;
     TcParams tp{};
@@ -873,8 +1025,6 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     tp.Ho = p.Ho; tp.Wo = p.Wo; tp.sh = p.sh; tp.sw = p.sw; tp.dh = p.dh; tp.dw = p.dw;
     tp.accumulate = p.accumulate;
 
-    const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-    CUresult r;
     // ---- input operand ----
     if (p.spatial_rank == 0) {
         tp.a_mode = 0;      // the map is encoded below, once the tile variant is known
@@ -889,6 +1039,7 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         // Tensors below 128 KiB are kept off the im2col path.
         int64_t in_bytes = (int64_t)p.batch * (p.spatial_rank == 2 ? used_h : 1) * used_w * p.C * es;
         if (in_bytes < 131072) return SG_ERR_UNSUPPORTED;
+        bool ok;
         if (p.spatial_rank == 1) {
             if (span_w > 32767) return SG_ERR_UNSUPPORTED;
             if (p.batch > 1 && !mult(p.i_n * es, 16)) return SG_ERR_UNSUPPORTED;
@@ -897,9 +1048,7 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
             cuuint64_t strides[2] = {(cuuint64_t)(p.i_w * es), (cuuint64_t)((p.batch > 1 ? p.i_n : used_w * p.i_w) * es)};
             int lower[1] = {0}, upper[1] = {(int)-span_w};
             cuuint32_t trav[3] = {1, (cuuint32_t)p.sw, 1};
-            r = g_drv.im2col(&map_in, in_type, 3, const_cast<void *>(In), dims, strides, lower,
-                             upper, BK, BM, trav, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            ok = encode_im2col_cached(&map_in, ctx.device, in_type, 3, In, dims, strides, lower, upper, BK, BM, trav);
         } else {
             if (span_w > 127 || span_h > 127) return SG_ERR_UNSUPPORTED;
             if (!mult(p.i_h * es, 16) || (p.batch > 1 && !mult(p.i_n * es, 16))) return SG_ERR_UNSUPPORTED;
@@ -909,28 +1058,24 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
                                      (cuuint64_t)((p.batch > 1 ? p.i_n : used_h * p.i_h) * es)};
             int lower[2] = {0, 0}, upper[2] = {(int)-span_w, (int)-span_h};
             cuuint32_t trav[4] = {1, (cuuint32_t)p.sw, (cuuint32_t)p.sh, 1};
-            r = g_drv.im2col(&map_in, in_type, 4, const_cast<void *>(In), dims, strides, lower,
-                             upper, BK, BM, trav, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            ok = encode_im2col_cached(&map_in, ctx.device, in_type, 4, In, dims, strides, lower, upper, BK, BM, trav);
         }
-        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
+        if (!ok) return SG_ERR_UNSUPPORTED;
     }
     // ---- output: 2-D {f, m} f32, stored in boxes of 32 columns x 128 rows ----
     {
         cuuint64_t dims[2] = {(cuuint64_t)p.N, (cuuint64_t)p.M};
         cuuint64_t strides[1] = {(cuuint64_t)(p.o_w * 4)};
         cuuint32_t box[2] = {32, BM};     // one store moves a chunk of 128 rows x 32 columns
-        r = g_drv.tiled(&map_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, O, dims, strides, box, ones,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
+        if (!encode_tiled_cached(&map_out, ctx.device, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, O, dims, strides, box,
+                                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE)) return SG_ERR_UNSUPPORTED;
     }
 
     // ---- tile variant and k split: lowest estimated time ----
     int pick = -1, splits = 1;
-    if (g_bn_override > 0) {
+    if (ov.bn > 0) {
         for (int i = 0; i < kNumVariants; ++i)
-            if (kVariants[i].bn == g_bn_override && kVariants[i].cg == (g_cg_override > 0 ? g_cg_override : 1) &&
+            if (kVariants[i].bn == ov.bn && kVariants[i].cg == (ov.cg > 0 ? ov.cg : 1) &&
                 !(f32 && kVariants[i].bn == 256 && kVariants[i].cg == 1) &&
                 !(lay != 0 && ((kVariants[i].bn == 256 && kVariants[i].cg == 1) || (kVariants[i].bn == 128 && kVariants[i].cg == 2)))) pick = i;
     }
@@ -939,23 +1084,23 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         return s >= 1 && (s - 1) * per < tp.num_kb;
     };
     if (pick >= 0) {
-        splits = g_split_override > 0 && valid_split(g_split_override) ? g_split_override : 1;
+        splits = ov.split > 0 && valid_split(ov.split) ? ov.split : 1;
     } else {
         // A forced split is taken as given when it fits the reduction (every range non-empty), with the variant that
         // is cheapest for it; one that does not fit is ignored and the estimate chooses the split as well.
-        const int forced = g_split_override > 0 && valid_split(g_split_override) ? g_split_override : 0;
+        const int forced = ov.split > 0 && valid_split(ov.split) ? ov.split : 0;
         double best = 1e300;
         // (a forced pair count that no variant can honour on this shape is dropped in a second pass)
         for (int pass = 0; pass < 2 && pick < 0; ++pass)
         for (int i = 0; i < kNumVariants; ++i) {
             const Variant &v = kVariants[i];
-            if (pass == 0 && g_cg_override > 0 && v.cg != g_cg_override && !(v.cg == 1 && p.M <= BM)) continue;
+            if (pass == 0 && ov.cg > 0 && v.cg != ov.cg && !(v.cg == 1 && p.M <= BM)) continue;
             if (f32 && v.bn == 256 && v.cg == 1) continue;       // not built (shared-memory budget)
             if (lay != 0 && ((v.bn == 256 && v.cg == 1) || (v.bn == 128 && v.cg == 2))) continue;   // not built for transposed operands
             if (v.bn > 64 && v.bn / 2 >= p.N) continue;          // at most half of the tile would be used
             if (v.cg == 2 && p.M <= BM) continue;                // the second CTA would have no rows
             const int64_t tiles = (int64_t)((p.M + v.cg * BM - 1) / (v.cg * BM)) * ((p.N + v.bn - 1) / v.bn);
-            const int64_t groups = g_drv.num_sms / v.cg;
+            const int64_t groups = num_sms / v.cg;
             if (forced) {
                 const double c = estimate_ns(v, f32, tiles, groups, tp.num_kb, forced, p.accumulate != 0);
                 if (c < best) { best = c; pick = i; splits = forced; }
@@ -970,6 +1115,11 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         }
     }
     if (pick < 0) return SG_ERR_INTERNAL;
+    const Variant &var = kVariants[pick];
+    // bf16 matmuls with whole k-blocks move two k-blocks per stage and per TMA load
+    const bool b_blocked = p.N % BK == 0 && !b_km;
+    const int kps = (!f32 && lay == 0 && p.spatial_rank == 0 && p.K % BK == 0 && b_blocked &&
+                     !(var.bn == 256 && var.cg == 1) && ov.kps != 1) ? 2 : 1;
     // ---- filter operand ----
     {
         const int64_t s_kw = p.KW > 1 ? p.k_kw : (int64_t)p.C * p.k_c;
@@ -978,38 +1128,34 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         // sub-tiles are read by the converter warps, one 128-byte row per load: no swizzle
         const CUtensorMapSwizzle swz = f32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B;
         const int sub_cols = BK;      // columns of one sub-tile: a 128-byte row
-        tp.b_blocked = p.N % sub_cols == 0 && !b_km;
+        tp.b_blocked = b_blocked;
+        bool ok;
         if (b_km) {
             // stored [n][k], k contiguous: 2-D {k, n}, box {BK, columns of this CTA} lands K-major
             cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)p.N};
             cuuint64_t strides[1] = {(cuuint64_t)(b_pitch * es)};
-            cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)(kVariants[pick].bn / kVariants[pick].cg)};
-            r = g_drv.tiled(&map_flt, in_type, 2, const_cast<void *>(Flt), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)(var.bn / var.cg)};
+            ok = encode_tiled_cached(&map_flt, ctx.device, in_type, 2, Flt, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B,
+                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
         } else if (tp.b_blocked) {
             // whole sub-tile column blocks: 5-D {column in block, c, column block, kw, kh}; one box
-            // {sub_cols, BK, blocks of this CTA, 1, 1} is the CTA's whole filter tile of a k-block
+            // {sub_cols, BK (two k-blocks: 2 BK), blocks of this CTA, 1, 1} is the CTA's whole filter tile of a stage
             cuuint64_t dims[5] = {(cuuint64_t)sub_cols, (cuuint64_t)p.C, (cuuint64_t)(p.N / sub_cols), (cuuint64_t)p.KW, (cuuint64_t)p.KH};
             cuuint64_t strides[4] = {(cuuint64_t)(p.k_c * es), (cuuint64_t)ROW_BYTES, (cuuint64_t)(s_kw * es), (cuuint64_t)(s_kh * es)};
-            // (bf16 matmuls with whole k-blocks fetch two k-blocks per load, see below)
-            const bool two = !f32 && lay == 0 && p.spatial_rank == 0 && p.K % BK == 0 && !(kVariants[pick].bn == 256 && kVariants[pick].cg == 1) && g_kps_override != 1;
-            cuuint32_t box[5] = {(cuuint32_t)sub_cols, (cuuint32_t)(two ? 2 * BK : BK), (cuuint32_t)(kVariants[pick].bn / kVariants[pick].cg / sub_cols), 1, 1};
-            r = g_drv.tiled(&map_flt, in_type, 5, const_cast<void *>(Flt), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            cuuint32_t box[5] = {(cuuint32_t)sub_cols, (cuuint32_t)(kps * BK), (cuuint32_t)(var.bn / var.cg / sub_cols), 1, 1};
+            ok = encode_tiled_cached(&map_flt, ctx.device, in_type, 5, Flt, dims, strides, box, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
         } else {
             // 4-D {f, c, kw, kh}, one sub-tile per load
             cuuint64_t dims[4] = {(cuuint64_t)p.N, (cuuint64_t)p.C, (cuuint64_t)p.KW, (cuuint64_t)p.KH};
             cuuint64_t strides[3] = {(cuuint64_t)(p.k_c * es), (cuuint64_t)(s_kw * es), (cuuint64_t)(s_kh * es)};
             cuuint32_t box[4] = {(cuuint32_t)sub_cols, (cuuint32_t)BK, 1, 1};
-            r = g_drv.tiled(&map_flt, in_type, 4, const_cast<void *>(Flt), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            ok = encode_tiled_cached(&map_flt, ctx.device, in_type, 4, Flt, dims, strides, box, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
         }
-        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
+        if (!ok) return SG_ERR_UNSUPPORTED;
     }
-    // bf16 matmuls with whole k-blocks move two k-blocks per stage and per TMA load
-    const int kps = (!f32 && lay == 0 && p.spatial_rank == 0 && p.K % BK == 0 && tp.b_blocked &&
-                     !(kVariants[pick].bn == 256 && kVariants[pick].cg == 1) && g_kps_override != 1) ? 2 : 1;
     if (p.spatial_rank == 0) {
+        const CUtensorMapSwizzle swz_a = (a_mn && f32) ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B;
+        bool ok;
         if (a_mn) {
             // stored [k][m], m contiguous, blocked by sub-tile rows of m (a 128-byte row: BK elements):
             // {m in block, k, m block}, box {BK, BK, 128 / BK}.  bf16 lands as an M-major operand
@@ -1017,24 +1163,20 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
             cuuint64_t dims[3] = {(cuuint64_t)BK, (cuuint64_t)p.K, (cuuint64_t)(p.M / BK)};
             cuuint64_t strides[2] = {(cuuint64_t)(a_pitch * es), (cuuint64_t)ROW_BYTES};
             cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BK, (cuuint32_t)(BM / BK)};
-            r = g_drv.tiled(&map_in, in_type, 3, const_cast<void *>(In), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                            f32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            ok = encode_tiled_cached(&map_in, ctx.device, in_type, 3, In, dims, strides, box, swz_a, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
         } else if (kps == 2) {
             // blocked by k-blocks: {k in block, m, k-block}, box {BK, 128, 2}
             cuuint64_t dims[3] = {(cuuint64_t)BK, (cuuint64_t)p.M, (cuuint64_t)(p.K / BK)};
             cuuint64_t strides[2] = {(cuuint64_t)(p.i_w * es), (cuuint64_t)ROW_BYTES};
             cuuint32_t box[3] = {(cuuint32_t)BK, BM, 2};
-            r = g_drv.tiled(&map_in, in_type, 3, const_cast<void *>(In), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            ok = encode_tiled_cached(&map_in, ctx.device, in_type, 3, In, dims, strides, box, swz_a, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
         } else {
             cuuint64_t dims[2] = {(cuuint64_t)p.K, (cuuint64_t)p.M};
             cuuint64_t strides[1] = {(cuuint64_t)(p.i_w * es)};
             cuuint32_t box[2] = {(cuuint32_t)BK, BM};
-            r = g_drv.tiled(&map_in, in_type, 2, const_cast<void *>(In), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            ok = encode_tiled_cached(&map_in, ctx.device, in_type, 2, In, dims, strides, box, swz_a, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
         }
-        if (r != CUDA_SUCCESS) return SG_ERR_UNSUPPORTED;
+        if (!ok) return SG_ERR_UNSUPPORTED;
     }
     // k ranges are whole stages; every range keeps at least one k-block
     int per = (tp.num_kb + splits - 1) / splits;
@@ -1042,11 +1184,15 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     splits = (tp.num_kb + per - 1) / per;
     tp.splits = splits;
     tp.kb_per_split = per;
+    // Unless something below says otherwise the kernel may start while the kernel ahead of it in the stream drains
+    // (programmatic dependent launch): it sets up its barriers and tensor memory, then waits for that kernel to finish
+    // before its first global read or write.
+    tp.wait_prior = ov.pdl == 0 ? 0 : 2;
     if (splits > 1) {
         // partial sums meet in the output by TMA reduce-add: an overwriting call clears it first
         if (!p.accumulate) {
             if (launch_zero_fill(p, O, stream) != cudaSuccess) return SG_ERR_CUDA;
-            tp.wait_prior = 1;      // the clearing kernel lets its dependents start at once
+            tp.wait_prior = 1;      // the clearing kernel lets its dependents start at once: only the stores wait for it
         }
         tp.accumulate = 1;
     }
@@ -1057,23 +1203,22 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     // outweigh the extra epilogues and the clearing launch (4096^3 f32 alone on the GPU: 498 -> 468 us; inside a step
     // of concurrent launches the other launches fill the last wave anyway and nothing changes).
     {
-        const Variant &v = kVariants[pick];
-        const int groups = g_drv.num_sms / v.cg;
-        const int num_m_tiles = (p.M + v.cg * BM - 1) / (v.cg * BM), num_n_tiles = (p.N + v.bn - 1) / v.bn;
+        const int groups = num_sms / var.cg;
+        const int num_m_tiles = (p.M + var.cg * BM - 1) / (var.cg * BM), num_n_tiles = (p.N + var.bn - 1) / var.bn;
         const int64_t tiles = (int64_t)num_m_tiles * num_n_tiles;
         const int left = (int)(tiles % groups);
-        if (g_sk_override != 0 && splits == 1 && tiles > groups && left != 0 && tp.num_kb % kps == 0) {
+        if (ov.sk != 0 && splits == 1 && tiles > groups && left != 0 && tp.num_kb % kps == 0) {
             const int64_t units = (int64_t)left * tp.num_kb;
             int run = (int)((units + groups - 1) / groups);
             run = (run + kps - 1) / kps * kps;
-            const double kb_ns = f32 ? v.mma_ns_f32 : v.mma_ns;
+            const double kb_ns = f32 ? var.mma_ns_f32 : var.mma_ns;
             const double saved = (double)(tp.num_kb - run) * kb_ns;
-            const double extra = 2.0 * (1500.0 + (double)v.bn * (f32 ? 24.0 : 12.0)) + 2500.0;
-            if (run >= 4 * kps && (saved > 2.0 * extra || g_sk_override == 2)) {
+            const double extra = 2.0 * (1500.0 + (double)var.bn * (f32 ? 24.0 : 12.0)) + 2500.0;
+            if (run >= 4 * kps && (saved > 2.0 * extra || ov.sk == 2)) {
                 tp.sk_first_tile = (int)(tiles - left);
                 tp.sk_units = run;
                 if (!p.accumulate) {
-                    zero_tiles_kernel<<<left, 256, 0, stream>>>(O, p.o_w, p.M, p.N, v.cg * BM, v.bn, num_m_tiles, num_n_tiles, tp.sk_first_tile);
+                    zero_tiles_kernel<<<left, 256, 0, stream>>>(O, p.o_w, p.M, p.N, var.cg * BM, var.bn, num_m_tiles, num_n_tiles, tp.sk_first_tile);
                     count_launch();
                     if (cudaGetLastError() != cudaSuccess) return SG_ERR_CUDA;
                     tp.wait_prior = 1;
@@ -1081,28 +1226,28 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
             }
         }
     }
-    g_last_choice[0] = kVariants[pick].bn; g_last_choice[1] = kVariants[pick].cg; g_last_choice[2] = splits;
-    g_last_sk[0] = tp.sk_units > 0 ? tp.sk_first_tile : -1; g_last_sk[1] = tp.sk_units;
+    t_last_choice[0] = var.bn; t_last_choice[1] = var.cg; t_last_choice[2] = splits;
+    t_last_sk[0] = tp.sk_units > 0 ? tp.sk_first_tile : -1; t_last_sk[1] = tp.sk_units;
     // f32 (either operand stored either way): the split input tile goes to tensor memory.  With
     // 256-column tiles that costs the second accumulator buffer, which short reductions used to feel; since the
     // converters stopped being the bottleneck the sweep is no slower with it everywhere (5.72 to 5.79 ms per step
     // either way), so there is one rule.
-    const int lay_k = (f32 && g_ta_override != 0) ? (lay | 4) : lay;
+    const int lay_k = (f32 && ov.ta != 0) ? (lay | 4) : lay;
     const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0) + lay_k * 3 * kNumVariants;
 #define SG_LAUNCH(BN_, CG_)                                                                                \
-    (f32 ? (lay_k == 4 ? launch_variant<BN_, CG_, true, 1, 4>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)     \
-            : lay_k == 6 ? launch_variant<BN_, CG_, true, 1, 6>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)   \
-            : lay_k == 5 ? launch_variant<BN_, CG_, true, 1, 5>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)   \
-            : lay_k == 7 ? launch_variant<BN_, CG_, true, 1, 7>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)   \
-            : lay == 0 ? launch_variant<BN_, CG_, true, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)         \
-            : lay == 1 ? launch_variant<BN_, CG_, true, 1, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
-            : lay == 2 ? launch_variant<BN_, CG_, true, 1, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
-                       : launch_variant<BN_, CG_, true, 1, 3>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream))   \
-     : lay == 1 ? launch_variant<BN_, CG_, false, 1, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
-     : lay == 2 ? launch_variant<BN_, CG_, false, 1, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
-     : lay == 3 ? launch_variant<BN_, CG_, false, 1, 3>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream)    \
-     : kps == 2 ? launch_variant<BN_, CG_, false, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream) \
-                : launch_variant<BN_, CG_, false, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, stream))
+    (f32 ? (lay_k == 4 ? launch_variant<BN_, CG_, true, 1, 4>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)     \
+            : lay_k == 6 ? launch_variant<BN_, CG_, true, 1, 6>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)   \
+            : lay_k == 5 ? launch_variant<BN_, CG_, true, 1, 5>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)   \
+            : lay_k == 7 ? launch_variant<BN_, CG_, true, 1, 7>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)   \
+            : lay == 0 ? launch_variant<BN_, CG_, true, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)         \
+            : lay == 1 ? launch_variant<BN_, CG_, true, 1, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)    \
+            : lay == 2 ? launch_variant<BN_, CG_, true, 1, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)    \
+                       : launch_variant<BN_, CG_, true, 1, 3>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx))   \
+     : lay == 1 ? launch_variant<BN_, CG_, false, 1, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)    \
+     : lay == 2 ? launch_variant<BN_, CG_, false, 1, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)    \
+     : lay == 3 ? launch_variant<BN_, CG_, false, 1, 3>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)    \
+     : kps == 2 ? launch_variant<BN_, CG_, false, 2>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx) \
+                : launch_variant<BN_, CG_, false, 1>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx))
     switch (pick) {
         case 0: return SG_LAUNCH(64, 1);
         case 1: return SG_LAUNCH(128, 1);
@@ -1128,44 +1273,63 @@ cudaError_t launch_wait_timeout_selftest(long long budget_cycles, cudaStream_t s
 }
 
 bool tensor_driver_ready(int *num_sms) {
+    const DeviceState *d = device_state(nullptr, nullptr);
+    if (!d) return false;
+    if (num_sms) *num_sms = d->num_sms;
+    return true;
+}
+
+bool tensor_device_info(int *device, int *num_sms, int *pdl, int *conv_single) {
+    Overrides ov;
+    const DeviceState *d = device_state(device, &ov);
+    if (!d) return false;
+    *num_sms = d->num_sms;
+    *pdl = ov.pdl;
+    *conv_single = ov.conv_single;
+    return true;
+}
+
+bool tensor_ensure_smem_attr(int slot, const void *kernel, int bytes) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices || slot < 0 || slot >= kAttrSlots) return false;
+    {
+        std::lock_guard<std::mutex> lock(g_mu);
+        if (g_dev[dev].attr_set[slot]) return true;
+    }
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
     std::lock_guard<std::mutex> lock(g_mu);
-    if (!init_driver()) return false;
-    if (num_sms) *num_sms = g_drv.num_sms;
+    g_dev[dev].attr_set[slot] = true;
     return true;
 }
 
 bool tensor_encode_tiled(CUtensorMap *map, CUtensorMapDataType type, int rank, void *base, const cuuint64_t *dims,
                          const cuuint64_t *strides, const cuuint32_t *box, CUtensorMapSwizzle swizzle,
                          CUtensorMapL2promotion promotion) {
-    const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-    EncodeTiledFn fn;
-    {
-        std::lock_guard<std::mutex> lock(g_mu);
-        if (!init_driver()) return false;
-        fn = g_drv.tiled;
-    }
-    return fn(map, type, (cuuint32_t)rank, base, dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, promotion,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    int dev = 0;
+    if (!device_state(&dev, nullptr)) return false;
+    return encode_tiled_cached(map, dev, type, rank, base, dims, strides, box, swizzle, promotion);
 }
 
 void tensor_set_tile_override(int bn, int cg, int splits) {
     std::lock_guard<std::mutex> lock(g_mu);
-    g_bn_override = bn; g_cg_override = cg; g_split_override = splits;
+    read_env_locked();
+    g_ov.bn = bn; g_ov.cg = cg; g_ov.split = splits;
 }
 
-void tensor_last_stream_k(int out[2]) {
-    std::lock_guard<std::mutex> lock(g_mu);
-    out[0] = g_last_sk[0]; out[1] = g_last_sk[1];
-}
+void tensor_last_stream_k(int out[2]) { out[0] = t_last_sk[0]; out[1] = t_last_sk[1]; }
 
-void tensor_last_choice(int out[3]) {
-    std::lock_guard<std::mutex> lock(g_mu);
-    out[0] = g_last_choice[0]; out[1] = g_last_choice[1]; out[2] = g_last_choice[2];
-}
+void tensor_last_choice(int out[3]) { out[0] = t_last_choice[0]; out[1] = t_last_choice[1]; out[2] = t_last_choice[2]; }
+
+void tensor_map_cache_stats(long long out[2]) { out[0] = g_cache_hits.load(); out[1] = g_cache_misses.load(); }
 
 void tensor_shutdown() {
+    {
+        std::lock_guard<std::mutex> lock(g_cache_mu);
+        free(g_cache);
+        g_cache = nullptr;
+    }
     std::lock_guard<std::mutex> lock(g_mu);
-    g_drv = Driver{};
+    for (DeviceState &d : g_dev) d = DeviceState{};
 }
 
 }  // namespace sg

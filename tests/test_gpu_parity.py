@@ -381,6 +381,37 @@ def test_conv1d_strip_kernel(N, Wo, C, KW, F, dw):
     assert_within_bound(O, want, S, "conv1d strip kernel")
 
 
+# f32 inputs on the same kernel: the filter split once into hi and lo and kept resident, the strips split per tap into
+# tensor memory.  Config 3 at full size in both modes, dilations, ragged channel blocks, 2-D windows, integer inputs.
+@pytest.mark.parametrize("accumulate", [False, True])
+def test_c3_conv1d_f32_strip_kernel_full(accumulate):
+    O, want, S = run_conv1d(32, 1024, 64, 3, 128, 1, 1, "f32", family=STRIP, accumulate=accumulate, seed=SEED + 2)
+    assert sg.sg_last_kernel_name() == "conv_strip_kernel<f32>"
+    assert assert_within_bound(O, want, S, "conv1d config 3, strip kernel") < F32_TENSOR_RATIO
+    O, want, S = run_conv1d(32, 1024, 64, 3, 128, 1, 1, "f32", seed=SEED + 2)      # and it is the default choice
+    assert sg.sg_last_kernel_name() == "conv_strip_kernel<f32>"
+    assert assert_within_bound(O, want, S, "conv1d config 3, default") < F32_TENSOR_RATIO
+
+
+@pytest.mark.parametrize("N,Wo,C,KW,F,dw", [(4, 300, 64, 3, 128, 1), (3, 333, 40, 3, 64, 1), (2, 411, 64, 3, 96, 2), (1, 5000, 64, 3, 64, 4),
+                                            (5, 97, 32, 2, 32, 3)])
+def test_conv1d_f32_strip_kernel(N, Wo, C, KW, F, dw):
+    O, want, S = run_conv1d(N, Wo, C, KW, F, 1, dw, "f32", family=STRIP, seed=SEED + 17, extra_w=3)
+    assert sg.sg_last_kernel_name() == "conv_strip_kernel<f32>"
+    assert assert_within_bound(O, want, S, "conv1d f32 strip kernel") < F32_TENSOR_RATIO
+    O, want, S = run_conv1d(N, Wo, C, KW, F, 1, dw, "f32", family=STRIP, dist="ints", seed=SEED + 17)
+    assert np.array_equal(O.cpu().numpy().astype(np.float64), want)
+
+
+@pytest.mark.parametrize("N,Ho,Wo,C,KH,KW,F,dl", [(3, 20, 20, 32, 2, 2, 64, (1, 1)), (2, 30, 40, 40, 1, 3, 128, (1, 3)),
+                                                   (4, 13, 17, 16, 2, 3, 32, (1, 1)), (2, 9, 150, 32, 2, 2, 64, (2, 1))])
+@pytest.mark.parametrize("accumulate", [False, True])
+def test_conv2d_f32_strip_kernel(N, Ho, Wo, C, KH, KW, F, dl, accumulate):
+    O, want, S = run_conv2d(N, Ho, Wo, C, KH, KW, F, (1, 1), dl, "f32", family=STRIP, accumulate=accumulate, seed=SEED + 18)
+    assert sg.sg_last_kernel_name() == "conv_strip_kernel<f32>"
+    assert assert_within_bound(O, want, S, "conv2d f32 strip kernel") < F32_TENSOR_RATIO
+
+
 def test_conv_strip_kernel_changes_filter_inside_a_cta():
     # two column tiles and an odd number of position tiles, more items than CTA groups: some
     # group's run of items straddles the column tiles, so it reloads its resident filter
@@ -392,7 +423,8 @@ def test_conv_strip_kernel_changes_filter_inside_a_cta():
 def test_conv_strip_kernel_exact_and_rejections():
     O, want, S = run_conv2d(2, 24, 24, 64, 3, 3, 64, (1, 1), (1, 1), "bf16", family=STRIP, dist="ints", seed=SEED + 7)
     assert np.array_equal(O.cpu().numpy().astype(np.float64), want)
-    # strided convolutions, f32 inputs and filters beyond shared memory are not this kernel's
+    # strided convolutions and filters beyond shared memory (here also: 3 x 3 x 64 x 64 in f32, split into hi and lo) are
+    # not this kernel's
     I = torch.zeros(1, 40, 40, 64, device="cuda", dtype=torch.bfloat16)
     Kf = torch.zeros(3, 3, 64, 64, device="cuda", dtype=torch.bfloat16)
     sg.sg_set_kernel_override(STRIP)
@@ -875,4 +907,79 @@ def test_device_timeout_is_reported_once_and_cleared():
     sg.sg_check()                                   # cleared by the read
     C, want, S = run_matmul(256, 256, 256, "bf16", family=TENSOR, seed=SEED + 41)
     assert_within_bound(C, want, S, "after a reported time-out")
+    sg.sg_check()
+
+
+# ------------------------------------------------------------------ host-side state: tensor-map cache, overlapped launches
+
+def test_tensor_map_cache_hits_and_never_serves_a_stale_map():
+    A = torch.randint(-2, 3, (512, 256), device="cuda").to(torch.bfloat16)
+    B = torch.randint(-2, 3, (256, 384), device="cuda").to(torch.bfloat16)
+    C = torch.empty(512, 384, device="cuda")
+    sg.sg_set_kernel_override(TENSOR)
+    h0, m0 = sg.sg_tensor_map_cache_stats()
+    sg.sg_matmul(A, B, C)
+    h1, m1 = sg.sg_tensor_map_cache_stats()
+    sg.sg_matmul(A, B, C)
+    h2, m2 = sg.sg_tensor_map_cache_stats()
+    # three maps per call: looked up, encoded when new (an earlier test may have left a map of the same address and
+    # geometry behind), and found by the second call
+    assert (h1 - h0) + (m1 - m0) == 3 and m1 - m0 >= 1 and m2 == m1 and h2 - h1 == 3
+    torch.cuda.synchronize()
+    assert torch.equal(C, A.float() @ B.float())
+    # the same base pointers with another geometry: other keys, so other maps
+    A2, B2, C2 = A.view(-1)[:256 * 128].view(256, 128), B.view(-1)[:128 * 192].view(128, 192), C.view(-1)[:256 * 192].view(256, 192)
+    sg.sg_matmul(A2, B2, C2)
+    torch.cuda.synchronize()
+    assert torch.equal(C2, A2.float() @ B2.float())
+    # more distinct maps than the cache holds (2048): entries are replaced, results stay right
+    big = torch.randint(-2, 3, (128 + 900, 64), device="cuda").to(torch.bfloat16)
+    Bs = torch.randint(-2, 3, (64, 64), device="cuda").to(torch.bfloat16)
+    outs = torch.empty(900, 128 + 900, 64, device="cuda")
+    for i in range(900):
+        sg.sg_matmul(big[:128 + i], Bs, outs[i, :128 + i])
+    sg.sg_matmul(A, B, C)                    # its maps may have been evicted meanwhile
+    torch.cuda.synchronize()
+    want = big.float() @ Bs.float()
+    for i in (0, 1, 450, 899):
+        assert torch.equal(outs[i, :128 + i], want[:128 + i])
+    assert torch.equal(C, A.float() @ B.float())
+    h3, m3 = sg.sg_tensor_map_cache_stats()
+    assert m3 - m2 >= 1800                   # every one of those shapes needed its own input and output map
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_back_to_back_calls_that_depend_on_each_other(dtype):
+    """Tensor-core launches may start while the kernel ahead of them drains; they must still see its results (a call
+    that reads the previous call's output) and must not overwrite what it still reads (a call that writes the previous
+    call's input).  Small integers keep every result exact; no synchronisation between the calls."""
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    M, K = 1024, 256
+    A = torch.randint(-1, 2, (M, K), device="cuda").to(tdt)
+    Bm = torch.randint(-1, 2, (K, K), device="cuda").to(tdt)
+    P = torch.zeros(K, K, device="cuda")
+    P[torch.arange(K, device="cuda"), torch.randperm(K, device="cuda")] = 1.0          # a permutation: products stay in {-1, 0, 1}
+    P = P.to(tdt)
+    X = torch.empty(M, K, device="cuda")              # f32 outputs; re-read as inputs only on the f32 path
+    Y = torch.empty(M, K, device="cuda")
+    sg.sg_set_kernel_override(TENSOR)
+    if dtype == "f32":
+        sg.sg_matmul(A, Bm, X)                        # X = A.B           (|x| <= 256)
+        for _ in range(6):
+            sg.sg_matmul(X, P, Y)                     # reads X right behind the call that wrote it
+            sg.sg_matmul(Y, P, X)                     # writes X right behind the call that read it
+        torch.cuda.synchronize()
+        want = A.double() @ Bm.double()
+        for _ in range(12):
+            want = want @ P.double()
+        assert torch.equal(X.double(), want)
+    else:
+        # bf16 inputs cannot be an f32 output; alternate two products into the same output instead: the last one wins
+        B2 = torch.randint(-1, 2, (K, K), device="cuda").to(tdt)
+        for _ in range(6):
+            sg.sg_matmul(A, Bm, X)
+            sg.sg_matmul(A, B2, X)
+            sg.sg_matmul(A, Bm, X, sg.SG_ACCUMULATE)  # adds onto the call ahead of it
+        torch.cuda.synchronize()
+        assert torch.equal(X.double(), A.double() @ (B2.double() + Bm.double()))
     sg.sg_check()
