@@ -275,6 +275,8 @@ def op_specs(sg, seed, bw_rows=None):
         "matmul4096_f32": mm(4096, 4096, 4096, "f32", "matmul 4096^3 f32 (sweep corner)"),
         "matmul4096_bf16": mm(4096, 4096, 4096, "bf16", "matmul 4096^3 bf16 (sweep corner)"),
         "matmul1024_bf16": mm(1024, 1024, 1024, "bf16", "matmul 1024^3 bf16 (sweep point)"),
+        # a sweep shape of about the step's average size per f32 launch: the shape the DRAM-traffic capture is taken on
+        "matmul_2048x2048x1024_f32": mm(2048, 2048, 1024, "f32", "matmul 2048x2048x1024 f32 (sweep point)"),
         "matmul8192_bf16": mm(8192, 8192, 8192, "bf16", "matmul 8192^3 bf16 (config 5)"),
         "matmul_skinny_bf16": mm(16384, 64, 4096, "bf16", "matmul 16384x64x4096 bf16 (config 5, skinny)"),
         # conv1d config 3: N=32, W=1026, C=64, KW=3, F=128, f32

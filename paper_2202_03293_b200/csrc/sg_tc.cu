@@ -102,6 +102,42 @@ __device__ __forceinline__ void split4(const uint4 v, uint4 &h, uint4 &l) {
     }
 }
 
+// Packs two f32 values, rounded to the nearest bf16, into one word: `even` in the low half, `odd` in the high half.
+__device__ __forceinline__ uint32_t pack_bf16(float even, float odd) {
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(odd), "f"(even));
+    return d;
+}
+// The split used when the two correction products run as bf16 MMAs: x = hi + lo with hi = x rounded to tf32 (as above); the
+// main product hi*hi runs in tf32, the corrections lo*hi + hi*lo with all four factors rounded to bf16.  A correction term
+// is below 2^-11 of its product and bf16 keeps 8 bits of each factor, so the rounding moves a product by less than 2^-19 of
+// itself (what the dropped lo*lo term and the tensor core's f32 accumulation cost already), and the two bf16 products of a k-block are one
+// contraction over 64 values, [lo | hi] . [hi | lo], at twice the tf32 rate: two tensor-core units per term instead of three.
+// Words of magnitude >= 2^127, infinities and NaNs: hi and its bf16 copy are truncated, never rounded up to infinity.
+__device__ __forceinline__ void split4_mix(const uint4 v, uint4 &h, uint2 &h16, uint2 &l16) {
+    const float fx = __uint_as_float(v.x), fy = __uint_as_float(v.y), fz = __uint_as_float(v.z), fw = __uint_as_float(v.w);
+    const float big = fmaxf(fmaxf(fabsf(fx), fabsf(fy)), fmaxf(fabsf(fz), fabsf(fw)));
+    if (big < 1.7014118e38f) {
+        h.x = (v.x + 0x1000u) & 0xFFFFE000u; h.y = (v.y + 0x1000u) & 0xFFFFE000u;
+        h.z = (v.z + 0x1000u) & 0xFFFFE000u; h.w = (v.w + 0x1000u) & 0xFFFFE000u;
+        h16.x = pack_bf16(__uint_as_float(h.x), __uint_as_float(h.y));
+        h16.y = pack_bf16(__uint_as_float(h.z), __uint_as_float(h.w));
+        l16.x = pack_bf16(fx - __uint_as_float(h.x), fy - __uint_as_float(h.y));
+        l16.y = pack_bf16(fz - __uint_as_float(h.z), fw - __uint_as_float(h.w));
+    } else {
+        auto one = [](uint32_t x, uint32_t &hi, uint32_t &hi16, uint32_t &lo16) {
+            hi = x & 0xFFFFE000u;
+            hi16 = x >> 16;
+            const float d = __uint_as_float(x) - __uint_as_float(hi);
+            lo16 = (x & 0x7F800000u) == 0x7F800000u ? 0u : (pack_bf16(d, 0.f) & 0xFFFFu);     // (small: rounding cannot overflow)
+        };
+        uint32_t a[4], b[4];
+        one(v.x, h.x, a[0], b[0]); one(v.y, h.y, a[1], b[1]); one(v.z, h.z, a[2], b[2]); one(v.w, h.w, a[3], b[3]);
+        h16.x = a[0] | (a[1] << 16); h16.y = a[2] | (a[3] << 16);
+        l16.x = b[0] | (b[1] << 16); l16.y = b[2] | (b[3] << 16);
+    }
+}
+
 template <int BN, int CG, bool F32, int KPS = 1, bool TA = false>
 struct Cfg {
     // CG = 1: one CTA owns a 128 x BN tile.  CG = 2: a pair of CTAs (one cluster) owns a
@@ -179,8 +215,11 @@ __global__ void __launch_bounds__(Cfg<BN, CG, F32, KPS, (LAY & 4) != 0>::THREADS
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_flt,
                const __grid_constant__ CUtensorMap map_out, const TcParams p) {
     constexpr bool A_MN = (LAY & 1) != 0, B_KM = (LAY & 2) != 0, TA = (LAY & 4) != 0;
+    // MIX (f32, plain layout, split input in tensor memory): the correction products lo*hi + hi*lo run as bf16 MMAs
+    constexpr bool MIX = (LAY & 8) != 0;
     using C = Cfg<BN, CG, F32, KPS, TA>;
     static_assert(!TA || F32, "tensor-memory input operand: f32 path only");
+    static_assert(!MIX || LAY == 12, "bf16 corrections: plain layout with the split input in tensor memory");
     static_assert(LAY == 0 || KPS == 1, "transposed layouts: one k-block per stage");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -405,7 +444,30 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                         const int s = it & 1;
                         if (!wait_all(mbar_wait<CG == 2>(split_full_bar(s), (it >> 1) & 1, abort_flag))) { ok = false; break; }
                         tc_fence_after();
-                        if constexpr (TA) {
+                        if constexpr (MIX) {
+                            // slot: [filter hi, tf32, K-major | filter as bf16, K-major rows of 64 k: hi then lo].  Tensor
+                            // memory: input hi (32 columns of tf32) | input as bf16: lo (16 columns), hi (16 columns).
+                            // The corrections [lo | hi] . [hi | lo] are four bf16 k-steps of 16, the main term four tf32
+                            // k-steps of 8: 8 MMAs per k-block instead of 12.
+                            constexpr uint32_t idesc16 = make_idesc(BN, CG * BM, false, false, false);
+                            const uint32_t slot = split_addr + s * C::SPLIT_BYTES;
+                            const uint64_t bh = make_smem_desc(slot, 16, 1024);
+                            const uint64_t b16 = make_smem_desc(slot + C::B_STAGE_BYTES, 16, 1024);
+                            const uint32_t a_hi = tmem_base + (uint32_t)(C::ACC_BUFS * BN + s * 64), a16 = a_hi + 32;
+                            if (issuer) {
+#pragma unroll
+                                for (int k = 0; k < K_STEPS; ++k) {      // small terms first
+                                    const uint32_t acc = (kb > kb0 || k > 0) ? 1u : 0u;
+                                    if constexpr (CG == 1) umma_bf16_ts(d_tmem, a16 + k * 8, b16 + (uint64_t)(k * 2), idesc16, acc);
+                                    else umma_bf16_ts_cg2(d_tmem, a16 + k * 8, b16 + (uint64_t)(k * 2), idesc16, acc);
+                                }
+#pragma unroll
+                                for (int k = 0; k < K_STEPS; ++k) {
+                                    if constexpr (CG == 1) umma_tf32_ts(d_tmem, a_hi + k * 8, bh + (uint64_t)(k * 2), idesc, 1u);
+                                    else umma_tf32_ts_cg2(d_tmem, a_hi + k * 8, bh + (uint64_t)(k * 2), idesc, 1u);
+                                }
+                            }
+                        } else if constexpr (TA) {
                             // filter hi | lo in the slot (K-major); input hi | lo in tensor memory, 32 columns
                             // (k) each, lane = row: the MMA takes its A operand from there
                             const uint32_t slot = split_addr + s * C::SPLIT_BYTES;
@@ -570,11 +632,51 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     } else {
                         split_elementwise(raw, slot, slot + A_STAGE_BYTES, std::integral_constant<int, A_STAGE_BYTES>{});
                     }
-                    if constexpr (B_KM)
+                    if constexpr (MIX) {
+                        // filter sub-tiles [32 k][32 columns] -> K-major rows of 128 B per column: the tf32 hi tile, and a
+                        // bf16 tile whose row is [hi of the 32 k | lo of the 32 k]; both 128-byte swizzled.  Unit = 4 k of a
+                        // sub-tile: lane = column reads down its column and writes 16 + 8 + 8 bytes of its two rows.
+                        const float *braw = reinterpret_cast<const float *>(raw + A_STAGE_BYTES);
+                        constexpr int UNITS = 8 * C::B_COLS / 32;
+#pragma unroll
+                        for (int u = cw; u < UNITS; u += CONVERTER_THREADS / 32) {
+                            const int j = u >> 3, eighth = u & 7;
+                            const float *col = braw + j * (C::SUB_BYTES / 4) + eighth * 4 * 32 + lane;
+                            uint32_t x[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) x[k] = __float_as_uint(col[k * 32]);
+                            const int f = j * 32 + lane;
+                            const int rowoff = (f >> 3) * 1024 + (f & 7) * 128;
+                            uint4 h;
+                            uint2 h16, l16;
+                            split4_mix(make_uint4(x[0], x[1], x[2], x[3]), h, h16, l16);
+                            *reinterpret_cast<uint4 *>(b_slot + rowoff + ((eighth ^ (f & 7)) << 4)) = h;
+                            uint8_t *r16 = b_slot + C::B_STAGE_BYTES + rowoff + (eighth & 1) * 8;
+                            *reinterpret_cast<uint2 *>(r16 + (((eighth >> 1) ^ (f & 7)) << 4)) = h16;
+                            *reinterpret_cast<uint2 *>(r16 + (((4 + (eighth >> 1)) ^ (f & 7)) << 4)) = l16;
+                        }
+                    } else if constexpr (B_KM)
                         split_elementwise(raw + A_STAGE_BYTES, b_slot, b_slot + C::B_STAGE_BYTES, std::integral_constant<int, C::B_STAGE_BYTES>{});
                     else
                         split_transpose(raw + A_STAGE_BYTES, b_slot, b_slot + C::B_STAGE_BYTES, std::integral_constant<int, C::B_COLS>{});
-                    if constexpr (TA) {
+                    if constexpr (MIX) {
+                        const int quarter = warp & 3, kpart = cw >> 2;
+                        uint32_t hi[8], lo16[4], hi16[4];
+#pragma unroll
+                        for (int i = 0; i < 2; ++i) {
+                            uint4 h;
+                            uint2 a, b;
+                            split4_mix(a_raw[i], h, a, b);
+                            hi[4 * i] = h.x; hi[4 * i + 1] = h.y; hi[4 * i + 2] = h.z; hi[4 * i + 3] = h.w;
+                            hi16[2 * i] = a.x; hi16[2 * i + 1] = a.y;
+                            lo16[2 * i] = b.x; lo16[2 * i + 1] = b.y;
+                        }
+                        // this thread's 8 k: tf32 hi in columns 8*kpart.., bf16 pairs in columns 32 + 4*kpart.. (lo) and 48 + 4*kpart.. (hi)
+                        const uint32_t t_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(C::ACC_BUFS * BN + s * 64);
+                        tmem_st_32x8(t_base + kpart * 8, hi);
+                        tmem_st_32x4(t_base + 32 + kpart * 4, lo16);
+                        tmem_st_32x4(t_base + 48 + kpart * 4, hi16);
+                    } else if constexpr (TA) {
                         const int quarter = warp & 3, kpart = cw >> 2;
                         uint32_t hi[8], lo[8];
 #pragma unroll
@@ -731,6 +833,7 @@ struct Overrides {
     int ta = -1;     // SG_TC_TA (testing): 0 never, 1 always keep the split f32 input tile in tensor memory
     int pdl = -1;    // SG_TC_PDL (testing): 0 = launches never overlap the tail of the kernel ahead of them
     int conv_single = 0;   // SG_CONV_SINGLE=1 (testing): the stride-1 convolution kernel never uses CTA pairs
+    int mix = -1;    // SG_TC_MIX (testing): 0 = f32 correction products as tf32 MMAs (three tf32 products per term) instead of bf16
 };
 std::mutex g_mu;
 EncodeTiledFn g_encode_tiled = nullptr;
@@ -748,6 +851,7 @@ void read_env_locked() {
     g_ov.kps = env("SG_TC_KPS", 0); g_ov.ta = env("SG_TC_TA", -1); g_ov.sk = env("SG_TC_SK", -1);
     g_ov.pdl = env("SG_TC_PDL", -1);
     g_ov.conv_single = env("SG_CONV_SINGLE", 0);
+    g_ov.mix = env("SG_TC_MIX", -1);
     g_ov.env_read = true;
 }
 
@@ -1232,10 +1336,13 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     // 256-column tiles that costs the second accumulator buffer, which short reductions used to feel; since the
     // converters stopped being the bottleneck the sweep is no slower with it everywhere (5.72 to 5.79 ms per step
     // either way), so there is one rule.
-    const int lay_k = (f32 && ov.ta != 0) ? (lay | 4) : lay;
-    const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0) + lay_k * 3 * kNumVariants;
+    // In the plain layout the two correction products of the split run as bf16 MMAs (see split4_mix).
+    int lay_k = (f32 && ov.ta != 0) ? (lay | 4) : lay;
+    if (lay_k == 4 && ov.mix != 0) lay_k = 12;
+    const int slot = pick + (f32 ? kNumVariants : 0) + (kps == 2 ? 2 * kNumVariants : 0) + (lay_k == 12 ? 8 : lay_k) * 3 * kNumVariants;
 #define SG_LAUNCH(BN_, CG_)                                                                                \
-    (f32 ? (lay_k == 4 ? launch_variant<BN_, CG_, true, 1, 4>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)     \
+    (f32 ? (lay_k == 12 ? launch_variant<BN_, CG_, true, 1, 12>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)   \
+            : lay_k == 4 ? launch_variant<BN_, CG_, true, 1, 4>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)     \
             : lay_k == 6 ? launch_variant<BN_, CG_, true, 1, 6>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)   \
             : lay_k == 5 ? launch_variant<BN_, CG_, true, 1, 5>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)   \
             : lay_k == 7 ? launch_variant<BN_, CG_, true, 1, 7>(map_in, map_flt, map_out, tp, p.M, p.N, slot, ctx)   \
