@@ -15,10 +15,12 @@
 // tile's columns) is loaded once per CTA and stays in shared memory.
 //   bf16: each tap's MMAs read its strip through a matrix descriptor whose start address is
 //         shifted by kw*dw rows.
-//   f32:  the filter is split once into hi = tf32(x) and lo = tf32(x - hi) (and transposed to
-//         K-major, which kind::tf32 needs); sixteen converter warps split the strip rows of each
-//         tap the same way into tensor memory (the tap's shift is a row offset of their reads)
-//         and the MMA warp accumulates lo*hi + hi*lo + hi*hi with the A operand in tensor memory.
+//   f32:  x = hi + lo with hi = x rounded to tf32.  The filter is split once per CTA (and transposed
+//         to K-major, which kind::tf32 needs) into a tf32 tile of hi and a bf16 tile [hi | lo];
+//         sixteen converter warps split the strip rows of each tap the same way into tensor memory
+//         (the tap's shift is a row offset of their reads), and the MMA warp accumulates the
+//         corrections lo*hi + hi*lo as one bf16 contraction over [lo | hi] . [hi | lo] and the main
+//         term hi*hi in tf32, the A operand in tensor memory: 8 MMAs per 32 channels of a tap.
 //
 // Because tiles start at row beginnings, the epilogue is TMA only: TMEM -> registers -> a swizzled
 // staging copy of the whole tile, laid out [image row][32-column chunk][w][32 f32] -> ONE tensor
@@ -71,35 +73,13 @@ struct ConvParams {
 template <int BN, int CG, bool F32>
 struct ConvCfg {
     static constexpr int B_COLS = BN / CG;                           // filter columns resident in this CTA
-    static constexpr int BLOCK_BYTES = B_COLS * 128 * (F32 ? 2 : 1); // one (tap, channel block): [hi | lo] for f32
+    static constexpr int BLOCK_BYTES = B_COLS * 128 * (F32 ? 2 : 1); // one (tap, channel block); f32: [hi, tf32 | hi and lo, bf16]
     static constexpr int ACC_COLS = 2 * BN;
     static constexpr int USED_COLS = ACC_COLS + (F32 ? A_SLOTS * 64 : 0);
     static constexpr int TMEM_COLS = USED_COLS <= 128 ? 128 : USED_COLS <= 256 ? 256 : 512;
     static constexpr int THREADS = 64 + 128 + (F32 ? 32 * CONVERTER_WARPS : 0);
     static_assert(USED_COLS <= 512 && B_COLS % 64 == 0, "tile width");
 };
-
-// 3xTF32 split of four f32 words: hi = x rounded to the nearest tf32 value (on the bit pattern: add half an ulp, clear
-// the low 13 bits), lo = (x - hi) rounded the same way; x - hi is exact in f32, so x - hi - lo is below 2^-22 |x|.
-// Words of magnitude >= 2^127 (where rounding up could reach infinity), infinities and NaNs take a slow path:
-// hi truncated, lo = 0 unless finite.
-__device__ __forceinline__ void split4(const uint4 v, uint4 &h, uint4 &l) {
-    const float fx = __uint_as_float(v.x), fy = __uint_as_float(v.y), fz = __uint_as_float(v.z), fw = __uint_as_float(v.w);
-    const float big = fmaxf(fmaxf(fabsf(fx), fabsf(fy)), fmaxf(fabsf(fz), fabsf(fw)));
-    if (big < 1.7014118e38f) {
-        h.x = (v.x + 0x1000u) & 0xFFFFE000u; l.x = (__float_as_uint(fx - __uint_as_float(h.x)) + 0x1000u) & 0xFFFFE000u;
-        h.y = (v.y + 0x1000u) & 0xFFFFE000u; l.y = (__float_as_uint(fy - __uint_as_float(h.y)) + 0x1000u) & 0xFFFFE000u;
-        h.z = (v.z + 0x1000u) & 0xFFFFE000u; l.z = (__float_as_uint(fz - __uint_as_float(h.z)) + 0x1000u) & 0xFFFFE000u;
-        h.w = (v.w + 0x1000u) & 0xFFFFE000u; l.w = (__float_as_uint(fw - __uint_as_float(h.w)) + 0x1000u) & 0xFFFFE000u;
-    } else {
-        auto one = [](uint32_t x, uint32_t &hi, uint32_t &lo) {
-            hi = x & 0xFFFFE000u;
-            const float d = __uint_as_float(x) - __uint_as_float(hi);
-            lo = (x & 0x7F800000u) == 0x7F800000u ? 0u : __float_as_uint(d);
-        };
-        one(v.x, h.x, l.x); one(v.y, h.y, l.y); one(v.z, h.z, l.z); one(v.w, h.w, l.w);
-    }
-}
 
 __device__ __forceinline__ void tma_store_4d(const CUtensorMap *map, uint32_t src, int x, int y, int z, int w) {
     asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
@@ -314,26 +294,24 @@ conv_strip_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_const
                                 const int s = kbi & (A_SLOTS - 1);
                                 if (!wait_all(mbar_wait<CG == 2>(split_full_bar(s), (kbi / A_SLOTS) & 1, abort_flag))) { ok = false; break; }
                                 tc_fence_after();
-                                // filter block hi | lo (K-major, 8-column groups 1024 B apart); input hi | lo in tensor
-                                // memory, 32 columns (k) each, lane = position
+                                // filter block (K-major, 8-column groups 1024 B apart): hi in tf32 | [hi, lo] in bf16; input in
+                                // tensor memory, lane = position: hi in 32 columns of tf32 | [lo, hi] in 2 x 16 columns of bf16 pairs
+                                constexpr uint32_t idesc16 = make_idesc(BN, CG * BM, false, false, false);
                                 const uint32_t blk = flt_addr + (uint32_t)((cb * p.KH + kh) * p.KW + kw) * C::BLOCK_BYTES;
                                 const uint64_t bh = make_smem_desc(blk, 16, 1024);
-                                const uint64_t bl = make_smem_desc(blk + C::B_COLS * 128, 16, 1024);
-                                const uint32_t a_hi = tmem_base + (uint32_t)(C::ACC_COLS + s * 64), a_lo = a_hi + 32;
+                                const uint64_t b16 = make_smem_desc(blk + C::B_COLS * 128, 16, 1024);
+                                const uint32_t a_hi = tmem_base + (uint32_t)(C::ACC_COLS + s * 64), a16 = a_hi + 32;
                                 if (issuer) {
 #pragma unroll
-                                    for (int k = 0; k < 4; ++k) {
-                                        const uint64_t o = (uint64_t)(k * 2);
-                                        if constexpr (CG == 1) {
-                                            umma_tf32_ts(d_tmem, a_lo + k * 8, bh + o, idesc, acc);   // small terms first
-                                            umma_tf32_ts(d_tmem, a_hi + k * 8, bl + o, idesc, 1u);
-                                            umma_tf32_ts(d_tmem, a_hi + k * 8, bh + o, idesc, 1u);
-                                        } else {
-                                            umma_tf32_ts_cg2(d_tmem, a_lo + k * 8, bh + o, idesc, acc);
-                                            umma_tf32_ts_cg2(d_tmem, a_hi + k * 8, bl + o, idesc, 1u);
-                                            umma_tf32_ts_cg2(d_tmem, a_hi + k * 8, bh + o, idesc, 1u);
-                                        }
+                                    for (int k = 0; k < 4; ++k) {      // the corrections [lo | hi] . [hi | lo] first: small terms
+                                        if constexpr (CG == 1) umma_bf16_ts(d_tmem, a16 + k * 8, b16 + (uint64_t)(k * 2), idesc16, acc);
+                                        else umma_bf16_ts_cg2(d_tmem, a16 + k * 8, b16 + (uint64_t)(k * 2), idesc16, acc);
                                         acc = 1u;
+                                    }
+#pragma unroll
+                                    for (int k = 0; k < 4; ++k) {
+                                        if constexpr (CG == 1) umma_tf32_ts(d_tmem, a_hi + k * 8, bh + (uint64_t)(k * 2), idesc, 1u);
+                                        else umma_tf32_ts_cg2(d_tmem, a_hi + k * 8, bh + (uint64_t)(k * 2), idesc, 1u);
                                     }
                                 }
                                 commit_all(split_empty_bar(s));
@@ -399,12 +377,16 @@ conv_strip_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_const
 #pragma unroll
                 for (int k = 0; k < 4; ++k) x[k] = __float_as_uint(col[k * 32]);
                 const int f = j * 32 + lane;
-                const int off = (f >> 3) * 1024 + (f & 7) * 128 + ((eighth ^ (f & 7)) << 4);
-                uint4 h, l;
-                split4(make_uint4(x[0], x[1], x[2], x[3]), h, l);
+                const int rowoff = (f >> 3) * 1024 + (f & 7) * 128;
+                uint4 h;
+                uint2 h16, l16;
+                split4_mix(make_uint4(x[0], x[1], x[2], x[3]), h, h16, l16);
                 uint8_t *blk = smem_gen + (size_t)b * C::BLOCK_BYTES;
-                *reinterpret_cast<uint4 *>(blk + off) = h;
-                *reinterpret_cast<uint4 *>(blk + C::B_COLS * 128 + off) = l;
+                *reinterpret_cast<uint4 *>(blk + rowoff + ((eighth ^ (f & 7)) << 4)) = h;
+                // the bf16 tile's row of this column: [hi of the 32 k | lo of the 32 k], 8 bytes for these 4 k in each half
+                uint8_t *r16 = blk + C::B_COLS * 128 + rowoff + (eighth & 1) * 8;
+                *reinterpret_cast<uint2 *>(r16 + (((eighth >> 1) ^ (f & 7)) << 4)) = h16;
+                *reinterpret_cast<uint2 *>(r16 + (((4 + (eighth >> 1)) ^ (f & 7)) << 4)) = l16;
             };
             // ---- the strips: per (channel block, tap) this warp's 32 positions x 8 channels -> tensor memory
             int it = 0, kbi = 0;
@@ -429,20 +411,24 @@ conv_strip_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_const
 #pragma unroll
                             for (int i = 0; i < 2; ++i)
                                 a_raw[i] = *reinterpret_cast<const uint4 *>(rp + (((kpart * 2 + i) ^ (row & 7)) << 4));
-                            uint32_t hi[8], lo[8];
+                            uint32_t hi[8], lo16[4], hi16[4];
 #pragma unroll
                             for (int i = 0; i < 2; ++i) {
-                                uint4 h, l;
-                                split4(a_raw[i], h, l);
+                                uint4 h;
+                                uint2 a, b;
+                                split4_mix(a_raw[i], h, a, b);
                                 hi[4 * i] = h.x; hi[4 * i + 1] = h.y; hi[4 * i + 2] = h.z; hi[4 * i + 3] = h.w;
-                                lo[4 * i] = l.x; lo[4 * i + 1] = l.y; lo[4 * i + 2] = l.z; lo[4 * i + 3] = l.w;
+                                hi16[2 * i] = a.x; hi16[2 * i + 1] = a.y;
+                                lo16[2 * i] = b.x; lo16[2 * i + 1] = b.y;
                             }
                             // the MMAs that read this slot's tensor-memory columns four k-blocks ago are done
                             if (!mbar_wait<CG == 2>(split_empty_bar(s), ((kbi / A_SLOTS) & 1) ^ 1u, abort_flag)) { ok = false; break; }
                             tc_fence_after();
-                            const uint32_t t_hi = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(C::ACC_COLS + s * 64 + kpart * 8);
-                            tmem_st_32x8(t_hi, hi);
-                            tmem_st_32x8(t_hi + 32, lo);
+                            // this thread's 8 k: tf32 hi in columns 8*kpart.., bf16 pairs in columns 32 + 4*kpart.. (lo) and 48 + 4*kpart.. (hi)
+                            const uint32_t t_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(C::ACC_COLS + s * 64);
+                            tmem_st_32x8(t_base + kpart * 8, hi);
+                            tmem_st_32x4(t_base + 32 + kpart * 4, lo16);
+                            tmem_st_32x4(t_base + 48 + kpart * 4, hi16);
                             tmem_st_wait();
                             tc_fence_before();
                             __syncwarp();

@@ -77,67 +77,6 @@ struct TcParams {
                          // kernel: loads and stores both wait.  0: an ordinary launch.
 };
 
-// 3xTF32 split of four f32 words.  hi = x rounded to the nearest tf32 value (10 mantissa bits;
-// done on the bit pattern: add half an ulp, clear the low 13 bits); x - hi is exact in f32 and
-// lo is that difference rounded to tf32 the same way, so x - hi - lo is below 2^-22 |x|.  The
-// low bits of hi and lo are zero, so whatever rounding the tensor core applies to its inputs
-// leaves them unchanged.  Words of magnitude >= 2^127 (where rounding up
-// could reach infinity), infinities and NaNs take a slow path: hi truncated, lo = 0 unless
-// finite.
-__device__ __forceinline__ void split4(const uint4 v, uint4 &h, uint4 &l) {
-    const float fx = __uint_as_float(v.x), fy = __uint_as_float(v.y), fz = __uint_as_float(v.z), fw = __uint_as_float(v.w);
-    const float big = fmaxf(fmaxf(fabsf(fx), fabsf(fy)), fmaxf(fabsf(fz), fabsf(fw)));
-    if (big < 1.7014118e38f) {
-        h.x = (v.x + 0x1000u) & 0xFFFFE000u; l.x = (__float_as_uint(fx - __uint_as_float(h.x)) + 0x1000u) & 0xFFFFE000u;
-        h.y = (v.y + 0x1000u) & 0xFFFFE000u; l.y = (__float_as_uint(fy - __uint_as_float(h.y)) + 0x1000u) & 0xFFFFE000u;
-        h.z = (v.z + 0x1000u) & 0xFFFFE000u; l.z = (__float_as_uint(fz - __uint_as_float(h.z)) + 0x1000u) & 0xFFFFE000u;
-        h.w = (v.w + 0x1000u) & 0xFFFFE000u; l.w = (__float_as_uint(fw - __uint_as_float(h.w)) + 0x1000u) & 0xFFFFE000u;
-    } else {
-        auto one = [](uint32_t x, uint32_t &hi, uint32_t &lo) {
-            hi = x & 0xFFFFE000u;
-            const float d = __uint_as_float(x) - __uint_as_float(hi);
-            lo = (x & 0x7F800000u) == 0x7F800000u ? 0u : __float_as_uint(d);
-        };
-        one(v.x, h.x, l.x); one(v.y, h.y, l.y); one(v.z, h.z, l.z); one(v.w, h.w, l.w);
-    }
-}
-
-// Packs two f32 values, rounded to the nearest bf16, into one word: `even` in the low half, `odd` in the high half.
-__device__ __forceinline__ uint32_t pack_bf16(float even, float odd) {
-    uint32_t d;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(odd), "f"(even));
-    return d;
-}
-// The split used when the two correction products run as bf16 MMAs: x = hi + lo with hi = x rounded to tf32 (as above); the
-// main product hi*hi runs in tf32, the corrections lo*hi + hi*lo with all four factors rounded to bf16.  A correction term
-// is below 2^-11 of its product and bf16 keeps 8 bits of each factor, so the rounding moves a product by less than 2^-19 of
-// itself (what the dropped lo*lo term and the tensor core's f32 accumulation cost already), and the two bf16 products of a k-block are one
-// contraction over 64 values, [lo | hi] . [hi | lo], at twice the tf32 rate: two tensor-core units per term instead of three.
-// Words of magnitude >= 2^127, infinities and NaNs: hi and its bf16 copy are truncated, never rounded up to infinity.
-__device__ __forceinline__ void split4_mix(const uint4 v, uint4 &h, uint2 &h16, uint2 &l16) {
-    const float fx = __uint_as_float(v.x), fy = __uint_as_float(v.y), fz = __uint_as_float(v.z), fw = __uint_as_float(v.w);
-    const float big = fmaxf(fmaxf(fabsf(fx), fabsf(fy)), fmaxf(fabsf(fz), fabsf(fw)));
-    if (big < 1.7014118e38f) {
-        h.x = (v.x + 0x1000u) & 0xFFFFE000u; h.y = (v.y + 0x1000u) & 0xFFFFE000u;
-        h.z = (v.z + 0x1000u) & 0xFFFFE000u; h.w = (v.w + 0x1000u) & 0xFFFFE000u;
-        h16.x = pack_bf16(__uint_as_float(h.x), __uint_as_float(h.y));
-        h16.y = pack_bf16(__uint_as_float(h.z), __uint_as_float(h.w));
-        l16.x = pack_bf16(fx - __uint_as_float(h.x), fy - __uint_as_float(h.y));
-        l16.y = pack_bf16(fz - __uint_as_float(h.z), fw - __uint_as_float(h.w));
-    } else {
-        auto one = [](uint32_t x, uint32_t &hi, uint32_t &hi16, uint32_t &lo16) {
-            hi = x & 0xFFFFE000u;
-            hi16 = x >> 16;
-            const float d = __uint_as_float(x) - __uint_as_float(hi);
-            lo16 = (x & 0x7F800000u) == 0x7F800000u ? 0u : (pack_bf16(d, 0.f) & 0xFFFFu);     // (small: rounding cannot overflow)
-        };
-        uint32_t a[4], b[4];
-        one(v.x, h.x, a[0], b[0]); one(v.y, h.y, a[1], b[1]); one(v.z, h.z, a[2], b[2]); one(v.w, h.w, a[3], b[3]);
-        h16.x = a[0] | (a[1] << 16); h16.y = a[2] | (a[3] << 16);
-        l16.x = b[0] | (b[1] << 16); l16.y = b[2] | (b[3] << 16);
-    }
-}
-
 template <int BN, int CG, bool F32, int KPS = 1, bool TA = false>
 struct Cfg {
     // CG = 1: one CTA owns a 128 x BN tile.  CG = 2: a pair of CTAs (one cluster) owns a
@@ -156,6 +95,8 @@ struct Cfg {
     // bf16: one ring of stages, TMA -> MMA.  f32: the TMA ring holds raw tiles; a second ring of
     // two slots holds what the converter warps make of them, [input hi | input lo | filter hi |
     // filter lo], the filter transposed to K-major on the way (kind::tf32 takes no N-major operand).
+    // (two slots are enough: with three the kernel is no faster - a k-block is bound by shared-memory bandwidth: the raw tiles
+    // written by TMA and read by the converters, the split filter written, and the MMAs' filter reads)
     static constexpr int SPLIT_SLOTS = F32 ? 2 : 0;
     // TA (f32): the split input tile lives in tensor memory (the MMA reads its A operand there), which
     // takes its writes and its three reads per k-step off the shared-memory pipe; a slot then holds
@@ -167,7 +108,7 @@ struct Cfg {
     static constexpr int THREADS = 192 + (F32 ? CONVERTER_THREADS : 0) + 32;
     static constexpr int FLT_WARP = THREADS / 32 - 1;
     // two accumulator buffers (one when the split input's 2 slots x 64 columns would not fit beside two)
-    static constexpr int A_TMEM_COLS = TA ? 128 : 0;
+    static constexpr int A_TMEM_COLS = TA ? SPLIT_SLOTS * 64 : 0;
     static constexpr int ACC_BUFS = 2 * BN + A_TMEM_COLS > 512 ? 1 : 2;
     static constexpr int USED_COLS = ACC_BUFS * BN + A_TMEM_COLS;
     static constexpr int TMEM_COLS = USED_COLS <= 32 ? 32 : USED_COLS <= 64 ? 64 : USED_COLS <= 128 ? 128 : USED_COLS <= 256 ? 256 : 512;
@@ -231,15 +172,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
     uint8_t *staging_gen = smem_gen + C::STAGES * C::STAGE_BYTES + C::SPLIT_SLOTS * C::SPLIT_BYTES;
     const uint32_t bars_addr = staging_addr + STAGING_BYTES;
     uint8_t *bars_gen = staging_gen + STAGING_BYTES;
-    // barrier block: full[8] | empty[8] | split_full[2] | split_empty[2] | acc_full[2] | acc_empty[2] | tmem_ptr | abort
+    // barrier block: full[8] | empty[8] | split_full[4] | split_empty[4] | acc_full[2] | acc_empty[2] | tmem_ptr | abort
     auto full_bar = [&](int s) { return bars_addr + 8u * s; };
     auto empty_bar = [&](int s) { return bars_addr + 8u * (8 + s); };
     auto split_full_bar = [&](int s) { return bars_addr + 8u * (16 + s); };
-    auto split_empty_bar = [&](int s) { return bars_addr + 8u * (18 + s); };
-    auto acc_full_bar = [&](int b) { return bars_addr + 8u * (20 + b); };
-    auto acc_empty_bar = [&](int b) { return bars_addr + 8u * (22 + b); };
-    volatile uint32_t *tmem_ptr_slot = reinterpret_cast<volatile uint32_t *>(bars_gen + 8 * 24);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_gen + 8 * 24 + 4);
+    auto split_empty_bar = [&](int s) { return bars_addr + 8u * (20 + s); };
+    auto acc_full_bar = [&](int b) { return bars_addr + 8u * (24 + b); };
+    auto acc_empty_bar = [&](int b) { return bars_addr + 8u * (26 + b); };
+    volatile uint32_t *tmem_ptr_slot = reinterpret_cast<volatile uint32_t *>(bars_gen + 8 * 28);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_gen + 8 * 28 + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // A launch behind this one that asked for it may start now: its CTAs take an SM as soon as one of ours leaves it
@@ -441,8 +382,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = kb0; kb < kb1; kb += KPS, ++it) {
                     if constexpr (F32) {
-                        const int s = it & 1;
-                        if (!wait_all(mbar_wait<CG == 2>(split_full_bar(s), (it >> 1) & 1, abort_flag))) { ok = false; break; }
+                        const int s = it % C::SPLIT_SLOTS;
+                        if (!wait_all(mbar_wait<CG == 2>(split_full_bar(s), (it / C::SPLIT_SLOTS) & 1, abort_flag))) { ok = false; break; }
                         tc_fence_after();
                         if constexpr (MIX) {
                             // slot: [filter hi, tf32, K-major | filter as bf16, K-major rows of 64 k: hi then lo].  Tensor
@@ -546,18 +487,69 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
         if constexpr (F32) {
             const int cw = warp - 6;                       // converter warp
             const int ct = (int)threadIdx.x - 192;         // converter thread
+            // MIX: this thread's fixed share of a k-block.  Input: row (warp & 3) * 32 + lane (the TMEM lane quarter this warp
+            // may touch), k columns 8 * (cw >> 2) ..: two 16-byte chunks of the swizzled raw row.  Filter: unit cw = (sub-tile of
+            // 32 columns, quarter of its 32 k): lane = column f reads 8 k down its column and owns chunks of row f.
+            uint32_t mx_a_off[2] = {0, 0}, mx_hi_off[2] = {0, 0}, mx_b_src = 0, mx_h16_off = 0, mx_l16_off = 0, mx_tmem = 0;
+            bool mx_has_unit = false;
+            if constexpr (MIX) {
+                const int row = (warp & 3) * 32 + lane;
+                for (int i = 0; i < 2; ++i) mx_a_off[i] = (uint32_t)(row * 128 + ((((cw >> 2) * 2 + i) ^ (row & 7)) << 4));
+                const int uj = cw >> 2, uq = cw & 3, f = uj * 32 + lane;
+                mx_has_unit = cw < 4 * C::B_COLS / 32;
+                mx_b_src = (uint32_t)(A_STAGE_BYTES + uj * C::SUB_BYTES + (uq * 8 * 32 + lane) * 4);
+                const uint32_t rowoff = (uint32_t)((f >> 3) * 1024 + (f & 7) * 128);
+                mx_hi_off[0] = rowoff + (uint32_t)(((2 * uq) ^ (f & 7)) << 4);
+                mx_hi_off[1] = rowoff + (uint32_t)(((2 * uq + 1) ^ (f & 7)) << 4);
+                mx_h16_off = (uint32_t)C::B_STAGE_BYTES + rowoff + (uint32_t)((uq ^ (f & 7)) << 4);
+                mx_l16_off = (uint32_t)C::B_STAGE_BYTES + rowoff + (uint32_t)(((4 + uq) ^ (f & 7)) << 4);
+                mx_tmem = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(C::ACC_BUFS * BN);
+            }
             int it = 0;
             bool ok = true;
             Cursor cur{0, sk_u0};
             int tile, kb0, kb1, add;
             while (ok && next_item(cur, tile, kb0, kb1, add)) {
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                    const int r = it % C::STAGES, s = it & 1;
+                    const int r = it % C::STAGES, s = it % C::SPLIT_SLOTS;
                     if (!mbar_wait(full_bar(r), (it / C::STAGES) & 1, abort_flag)) { ok = false; break; }
-                    if (!mbar_wait<CG == 2>(split_empty_bar(s), ((it >> 1) & 1) ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait<CG == 2>(split_empty_bar(s), ((it / C::SPLIT_SLOTS) & 1) ^ 1u, abort_flag)) { ok = false; break; }
                     if constexpr (TA) tc_fence_after();     // the MMAs that read this slot's tensor-memory columns are done
                     const uint8_t *raw = smem_gen + r * C::STAGE_BYTES;
                     uint8_t *slot = smem_gen + C::STAGES * C::STAGE_BYTES + s * C::SPLIT_BYTES;
+                    if constexpr (MIX) {
+                        // Plain layout, corrections as bf16 MMAs.  Every address below is fixed per thread (set up ahead of
+                        // the loops); the loads go out first, input rows then filter columns.
+                        const uint4 a0 = *reinterpret_cast<const uint4 *>(raw + mx_a_off[0]);
+                        const uint4 a1 = *reinterpret_cast<const uint4 *>(raw + mx_a_off[1]);
+                        uint32_t x[8];
+                        if (mx_has_unit) {
+                            const float *col = reinterpret_cast<const float *>(raw + mx_b_src);
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) x[k] = __float_as_uint(col[k * 32]);
+                        }
+                        // input: this thread's 8 k of its row -> tf32 hi (8 columns), bf16 pairs lo and hi (4 columns each)
+                        {
+                            uint4 h0, h1, h16, l16;
+                            split8_mix(a0, a1, h0, h1, h16, l16);
+                            const uint32_t hi[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+                            const uint32_t lo4[4] = {l16.x, l16.y, l16.z, l16.w}, hi4[4] = {h16.x, h16.y, h16.z, h16.w};
+                            const uint32_t t_base = mx_tmem + (uint32_t)(s * 64);
+                            tmem_st_32x8(t_base + (cw >> 2) * 8, hi);
+                            tmem_st_32x4(t_base + 32 + (cw >> 2) * 4, lo4);
+                            tmem_st_32x4(t_base + 48 + (cw >> 2) * 4, hi4);
+                        }
+                        // filter: 8 k of this lane's column -> two chunks of its row of the tf32 hi tile, one chunk each of the
+                        // hi half and the lo half of its row of the bf16 tile (rows of 128 B, 128-byte swizzled)
+                        if (mx_has_unit) {
+                            uint4 h0, h1, h16, l16;
+                            split8_mix(make_uint4(x[0], x[1], x[2], x[3]), make_uint4(x[4], x[5], x[6], x[7]), h0, h1, h16, l16);
+                            *reinterpret_cast<uint4 *>(slot + mx_hi_off[0]) = h0;
+                            *reinterpret_cast<uint4 *>(slot + mx_hi_off[1]) = h1;
+                            *reinterpret_cast<uint4 *>(slot + mx_h16_off) = h16;
+                            *reinterpret_cast<uint4 *>(slot + mx_l16_off) = l16;
+                        }
+                    } else {
                     // An operand tile that arrives K-major (rows of 32 k, 128-byte swizzled by the TMA) is
                     // split elementwise: the swizzled placement of the elements is kept.
                     auto split_elementwise = [&](const uint8_t *src_tile, uint8_t *hi_tile, uint8_t *lo_tile, auto bytes_tag) {
@@ -632,51 +624,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                     } else {
                         split_elementwise(raw, slot, slot + A_STAGE_BYTES, std::integral_constant<int, A_STAGE_BYTES>{});
                     }
-                    if constexpr (MIX) {
-                        // filter sub-tiles [32 k][32 columns] -> K-major rows of 128 B per column: the tf32 hi tile, and a
-                        // bf16 tile whose row is [hi of the 32 k | lo of the 32 k]; both 128-byte swizzled.  Unit = 4 k of a
-                        // sub-tile: lane = column reads down its column and writes 16 + 8 + 8 bytes of its two rows.
-                        const float *braw = reinterpret_cast<const float *>(raw + A_STAGE_BYTES);
-                        constexpr int UNITS = 8 * C::B_COLS / 32;
-#pragma unroll
-                        for (int u = cw; u < UNITS; u += CONVERTER_THREADS / 32) {
-                            const int j = u >> 3, eighth = u & 7;
-                            const float *col = braw + j * (C::SUB_BYTES / 4) + eighth * 4 * 32 + lane;
-                            uint32_t x[4];
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) x[k] = __float_as_uint(col[k * 32]);
-                            const int f = j * 32 + lane;
-                            const int rowoff = (f >> 3) * 1024 + (f & 7) * 128;
-                            uint4 h;
-                            uint2 h16, l16;
-                            split4_mix(make_uint4(x[0], x[1], x[2], x[3]), h, h16, l16);
-                            *reinterpret_cast<uint4 *>(b_slot + rowoff + ((eighth ^ (f & 7)) << 4)) = h;
-                            uint8_t *r16 = b_slot + C::B_STAGE_BYTES + rowoff + (eighth & 1) * 8;
-                            *reinterpret_cast<uint2 *>(r16 + (((eighth >> 1) ^ (f & 7)) << 4)) = h16;
-                            *reinterpret_cast<uint2 *>(r16 + (((4 + (eighth >> 1)) ^ (f & 7)) << 4)) = l16;
-                        }
-                    } else if constexpr (B_KM)
+                    if constexpr (B_KM)
                         split_elementwise(raw + A_STAGE_BYTES, b_slot, b_slot + C::B_STAGE_BYTES, std::integral_constant<int, C::B_STAGE_BYTES>{});
                     else
                         split_transpose(raw + A_STAGE_BYTES, b_slot, b_slot + C::B_STAGE_BYTES, std::integral_constant<int, C::B_COLS>{});
-                    if constexpr (MIX) {
-                        const int quarter = warp & 3, kpart = cw >> 2;
-                        uint32_t hi[8], lo16[4], hi16[4];
-#pragma unroll
-                        for (int i = 0; i < 2; ++i) {
-                            uint4 h;
-                            uint2 a, b;
-                            split4_mix(a_raw[i], h, a, b);
-                            hi[4 * i] = h.x; hi[4 * i + 1] = h.y; hi[4 * i + 2] = h.z; hi[4 * i + 3] = h.w;
-                            hi16[2 * i] = a.x; hi16[2 * i + 1] = a.y;
-                            lo16[2 * i] = b.x; lo16[2 * i + 1] = b.y;
-                        }
-                        // this thread's 8 k: tf32 hi in columns 8*kpart.., bf16 pairs in columns 32 + 4*kpart.. (lo) and 48 + 4*kpart.. (hi)
-                        const uint32_t t_base = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(C::ACC_BUFS * BN + s * 64);
-                        tmem_st_32x8(t_base + kpart * 8, hi);
-                        tmem_st_32x4(t_base + 32 + kpart * 4, lo16);
-                        tmem_st_32x4(t_base + 48 + kpart * 4, hi16);
-                    } else if constexpr (TA) {
+                    if constexpr (TA) {
                         const int quarter = warp & 3, kpart = cw >> 2;
                         uint32_t hi[8], lo[8];
 #pragma unroll
@@ -690,6 +642,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                         tmem_st_32x8(t_hi, hi);
                         tmem_st_32x8(t_hi + 32, lo);
                     }
+                    }   // (!MIX)
                     fence_async_smem();     // generic-proxy writes -> visible to the tensor core's reads
                     if constexpr (TA) {
                         tmem_st_wait();

@@ -323,6 +323,78 @@ __device__ __forceinline__ void umma_commit_cg2(uint32_t cluster_bar) {
 }
 
 
+// ---------------------------------------------------------------- f32 inputs on the tensor cores: the hi/lo split
+// 3xTF32 split of four f32 words.  hi = x rounded to the nearest tf32 value (10 mantissa bits;
+// done on the bit pattern: add half an ulp, clear the low 13 bits); x - hi is exact in f32 and
+// lo is that difference rounded to tf32 the same way, so x - hi - lo is below 2^-22 |x|.  The
+// low bits of hi and lo are zero, so whatever rounding the tensor core applies to its inputs
+// leaves them unchanged.  Words of magnitude >= 2^127 (where rounding up
+// could reach infinity), infinities and NaNs take a slow path: hi truncated, lo = 0 unless
+// finite.
+__device__ __forceinline__ void split4(const uint4 v, uint4 &h, uint4 &l) {
+    const float fx = __uint_as_float(v.x), fy = __uint_as_float(v.y), fz = __uint_as_float(v.z), fw = __uint_as_float(v.w);
+    const float big = fmaxf(fmaxf(fabsf(fx), fabsf(fy)), fmaxf(fabsf(fz), fabsf(fw)));
+    if (big < 1.7014118e38f) {
+        h.x = (v.x + 0x1000u) & 0xFFFFE000u; l.x = (__float_as_uint(fx - __uint_as_float(h.x)) + 0x1000u) & 0xFFFFE000u;
+        h.y = (v.y + 0x1000u) & 0xFFFFE000u; l.y = (__float_as_uint(fy - __uint_as_float(h.y)) + 0x1000u) & 0xFFFFE000u;
+        h.z = (v.z + 0x1000u) & 0xFFFFE000u; l.z = (__float_as_uint(fz - __uint_as_float(h.z)) + 0x1000u) & 0xFFFFE000u;
+        h.w = (v.w + 0x1000u) & 0xFFFFE000u; l.w = (__float_as_uint(fw - __uint_as_float(h.w)) + 0x1000u) & 0xFFFFE000u;
+    } else {
+        auto one = [](uint32_t x, uint32_t &hi, uint32_t &lo) {
+            hi = x & 0xFFFFE000u;
+            const float d = __uint_as_float(x) - __uint_as_float(hi);
+            lo = (x & 0x7F800000u) == 0x7F800000u ? 0u : __float_as_uint(d);
+        };
+        one(v.x, h.x, l.x); one(v.y, h.y, l.y); one(v.z, h.z, l.z); one(v.w, h.w, l.w);
+    }
+}
+
+// Packs two f32 values, rounded to the nearest bf16, into one word: `even` in the low half, `odd` in the high half.
+__device__ __forceinline__ uint32_t pack_bf16(float even, float odd) {
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(odd), "f"(even));
+    return d;
+}
+// The split used when the two correction products run as bf16 MMAs: x = hi + lo with hi = x rounded to tf32 (as above); the
+// main product hi*hi runs in tf32, the corrections lo*hi + hi*lo with all four factors rounded to bf16.  A correction term
+// is below 2^-11 of its product and bf16 keeps 8 bits of each factor, so the rounding moves a product by less than 2^-19 of
+// itself (what the dropped lo*lo term and the tensor core's f32 accumulation cost already), and the two bf16 products of a k-block are one
+// contraction over 64 values, [lo | hi] . [hi | lo], at twice the tf32 rate: two tensor-core units per term instead of three.
+// Words of magnitude >= 2^127, infinities and NaNs: hi and its bf16 copy are truncated, never rounded up to infinity.
+__device__ __forceinline__ void split4_mix(const uint4 v, uint4 &h, uint2 &h16, uint2 &l16) {
+    const float fx = __uint_as_float(v.x), fy = __uint_as_float(v.y), fz = __uint_as_float(v.z), fw = __uint_as_float(v.w);
+    const float big = fmaxf(fmaxf(fabsf(fx), fabsf(fy)), fmaxf(fabsf(fz), fabsf(fw)));
+    if (big < 1.7014118e38f) {
+        h.x = (v.x + 0x1000u) & 0xFFFFE000u; h.y = (v.y + 0x1000u) & 0xFFFFE000u;
+        h.z = (v.z + 0x1000u) & 0xFFFFE000u; h.w = (v.w + 0x1000u) & 0xFFFFE000u;
+        h16.x = pack_bf16(__uint_as_float(h.x), __uint_as_float(h.y));
+        h16.y = pack_bf16(__uint_as_float(h.z), __uint_as_float(h.w));
+        l16.x = pack_bf16(fx - __uint_as_float(h.x), fy - __uint_as_float(h.y));
+        l16.y = pack_bf16(fz - __uint_as_float(h.z), fw - __uint_as_float(h.w));
+    } else {
+        auto one = [](uint32_t x, uint32_t &hi, uint32_t &hi16, uint32_t &lo16) {
+            hi = x & 0xFFFFE000u;
+            hi16 = x >> 16;
+            const float d = __uint_as_float(x) - __uint_as_float(hi);
+            lo16 = (x & 0x7F800000u) == 0x7F800000u ? 0u : (pack_bf16(d, 0.f) & 0xFFFFu);     // (small: rounding cannot overflow)
+        };
+        uint32_t a[4], b[4];
+        one(v.x, h.x, a[0], b[0]); one(v.y, h.y, a[1], b[1]); one(v.z, h.z, a[2], b[2]); one(v.w, h.w, a[3], b[3]);
+        h16.x = a[0] | (a[1] << 16); h16.y = a[2] | (a[3] << 16);
+        l16.x = b[0] | (b[1] << 16); l16.y = b[2] | (b[3] << 16);
+    }
+}
+
+
+// The same for eight values (two chunks of four): hi of each chunk, and the eight bf16 values of hi and of lo packed in k order.
+__device__ __forceinline__ void split8_mix(const uint4 v0, const uint4 v1, uint4 &h0, uint4 &h1, uint4 &h16, uint4 &l16) {
+    uint2 a, b, c, d;
+    split4_mix(v0, h0, a, b);
+    split4_mix(v1, h1, c, d);
+    h16 = make_uint4(a.x, a.y, c.x, c.y);
+    l16 = make_uint4(b.x, b.y, d.x, d.y);
+}
+
 // Reads and clears this translation unit's status word; the caller has synchronised the stream.
 inline sg_status read_status_word(cudaStream_t stream) {
     unsigned int word = 0, zero = 0;
