@@ -97,18 +97,6 @@ __device__ __forceinline__ void tma_reduce_add_5d(const CUtensorMap *map, uint32
     asm volatile("cp.reduce.async.bulk.tensor.5d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
                  ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v) : "memory");
 }
-// The four epilogue warps agree on one answer (all of them reach this barrier whatever they found).
-__device__ __forceinline__ bool epilogue_all(bool mine) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.and.pred p, 1, 128, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out) : "r"((uint32_t)mine) : "memory");
-    return out != 0;
-}
-
 // CG = 1: one CTA computes a tile of 128 positions x BN columns.  CG = 2: a CTA pair (one cluster) computes two
 // neighbouring tiles x BN columns with tcgen05.mma.cta_group::2: each CTA loads the strips of its own tile and keeps
 // its own BN/2 columns of the filter, which halves the resident filter and leaves room for a deeper ring of strips.

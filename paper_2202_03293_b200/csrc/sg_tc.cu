@@ -22,14 +22,13 @@
 //                          filter is stored [k][f] with f contiguous, so it is consumed as
 //                          an MN-major operand instead of being transposed.
 //
-// f32 inputs run on the same pipeline as three tf32 products per k-step ("3xTF32"): the TMA
-// writes the raw f32 tiles into its ring, sixteen converter warps split every element x into two
-// values hi = x rounded to tf32 and lo = x - hi and write them to a second ring of two slots
-// (transposing the filter tile to K-major on the way, which kind::tf32 needs; the input tile's
-// hi and lo go to tensor memory when it is stored [m][k]), and the MMA
-// thread accumulates lo*hi + hi*lo + hi*hi in f32: the dropped terms are below 2^-21 |a*b|, so
-// f32 accuracy is kept.  Raw tiles are 128 rows x 32 f32 (input) and 32 k-rows x 32 f32
-// sub-tiles (filter), again 128 bytes per row.
+// f32 inputs run on the same pipeline with every element split as x = hi + lo, hi = x rounded to tf32: the TMA
+// writes the raw f32 tiles into its ring, sixteen converter warps split them and write a second ring of two slots
+// (transposing the filter tile to K-major on the way, which kind::tf32 needs; the split input tile goes to tensor
+// memory), and the MMA thread accumulates lo*hi + hi*lo + hi*hi in f32: the dropped term is below 2^-21 |a*b|, so
+// f32 accuracy is kept.  In the plain layout hi*hi runs in tf32 and the two corrections as one bf16 contraction over
+// [lo | hi] . [hi | lo] (8 MMAs per k-block); the transposed layouts run three tf32 products (12).  Raw tiles are
+// 128 rows x 32 f32 (input) and 32 k-rows x 32 f32 sub-tiles (filter), again 128 bytes per row.
 //
 // Every wait in this file is bounded: a wait that expires sets an abort flag in shared
 // memory and a bit in the device status word, every role then leaves its loop, the CTA
@@ -679,9 +678,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
             tile_coords(tile, p.num_m_tiles, p.num_n_tiles, mt, nt);
             const int m0 = (mt * CG + (int)cta_rank) * BM, n0 = nt * BN;
             const int buf = tl % C::ACC_BUFS;
-            // (the barrier's phase stays complete until these warps hand the buffer back, so the four
-            // warps take the same way here and meet at every epi_sync below)
-            if (!mbar_wait(acc_full_bar(buf), (tl / C::ACC_BUFS) & 1, abort_flag)) { ok = false; break; }
+            // (the four warps take the same way here and meet at every epi_sync below)
+            if (!epilogue_all(mbar_wait(acc_full_bar(buf), (tl / C::ACC_BUFS) & 1, abort_flag))) { ok = false; break; }
             tc_fence_after();
 #pragma unroll 1
             for (int j = 0; j < BN / 32; ++j, ++chunk_count) {

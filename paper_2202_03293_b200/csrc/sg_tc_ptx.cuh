@@ -291,6 +291,19 @@ __device__ __forceinline__ void tma_tile_3d(uint32_t dst, const CUtensorMap *map
         asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
 }
+// The four epilogue warps (128 threads, named barrier 1) agree on one answer: all of them reach this barrier whatever
+// they found, so a bounded wait that one warp gave up on and another passed cannot leave them at different barriers.
+__device__ __forceinline__ bool epilogue_all(bool mine) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.and.pred p, 1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out) : "r"((uint32_t)mine) : "memory");
+    return out != 0;
+}
+
 // True in exactly one lane of the (converged) warp, the same lane on every call.
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred;
