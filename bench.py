@@ -454,8 +454,9 @@ def sweep_table(sg, peaks, bufs, torch):
         for (m, n, k) in SHAPES:
             a, b, c = bufs[dtype, m, n, k]
             flops = 2.0 * m * n * k
-            reps = int(max(3, min(40, 2e-3 / max(flops / 3e14, 8e-6))))
-            ms = time_launches(lambda i: sg.sg_matmul(a, b, c), reps, 2)
+            # device time by graph replay of a few back-to-back calls (the host's call overhead stays outside)
+            ncalls = int(max(2, min(16, 1e-3 / max(flops / 3e14, 8e-6))))
+            ms = statistics.median(time_graph([lambda: sg.sg_matmul(a, b, c)] * ncalls, 5))
             t_c, t_b = flops / peak, ((m * k + k * n) * es + m * n * 4) / (peaks["hbm_gbs"] * 1e9)
             rows.append({"dtype": dtype, "M": m, "N": n, "K": k, "us": round(ms * 1e3, 2),
                          "gflops": round(flops / (ms * 1e-3) / 1e9, 1), "bound": "hbm" if t_b > t_c else "tensor",

@@ -88,6 +88,30 @@ def matmul(A, B, C_in=None, threads=0):
     return C, S
 
 
+def matmul_bias_act(A, B, bias=None, act="none", threads=0):
+    """C[m,n] = act(sum_k A[m,k]*B[k,n] + bias[n]); act "none" or "relu".  Returns (C, S) with S = sum|a*b| + |bias|."""
+    A, B = _f32(A), _f32(B)
+    M, K = A.shape
+    K2, N = B.shape
+    assert K == K2
+    code = {"none": 0, "relu": 1}[act]
+    C = np.zeros((M, N), np.float64)
+    S = np.zeros((M, N), np.float64)
+    sa, sb = _estrides(A), _estrides(B)
+    if bias is not None:
+        bias = _f32(bias)
+        assert bias.shape == (N,)
+        bp, bs = _ptr(bias), _estrides(bias)[0]
+    else:
+        bp, bs = ctypes.c_void_p(0), 0
+    rc = lib().sg_ref_matmul_bias_act(_i64(M), _i64(N), _i64(K), _ptr(A), _i64(sa[0]), _i64(sa[1]),
+                                      _ptr(B), _i64(sb[0]), _i64(sb[1]), bp, _i64(bs), ctypes.c_int(code),
+                                      _ptr(C), _i64(N), _i64(1), _ptr(S), ctypes.c_int(threads))
+    if rc:
+        raise ValueError("sg_ref_matmul_bias_act rejected its arguments")
+    return C, S
+
+
 def matmul_points(A, B, pm, pn, threads=0):
     A, B = _f32(A), _f32(B)
     K = A.shape[1]

@@ -92,6 +92,44 @@ int sg_ref_matmul(int64_t M, int64_t N, int64_t K,
     return 0;
 }
 
+/*
+ * Matmul with a fused pointwise consumer (Section 2.1: tensor operations are fused at the tiled level; Section 3.3,
+ * items 1 and 2 of the vectorization cases: a pointwise op has identity indexing maps, a lower-dimensional operand
+ * is broadcast).  The consumer is the generic op with maps (m,n)->(m,n) for the product, (m,n)->(n) for the bias
+ * and (m,n)->(m,n) for the result, and body  r = act(p + b):
+ *     C[m,n] = act( sum_k A[m,k]*B[k,n] + bias[n] ),   act = identity (0) or max(., 0) (1).
+ * Evaluated the unfused way: the whole sum first, in f64, then the consumer on it.  bias may be NULL (no bias).
+ * S (optional) = sum_k |a*b| + |bias[n]|: the scale of the comparison bound.
+ */
+int sg_ref_matmul_bias_act(int64_t M, int64_t N, int64_t K,
+                           const float *A, int64_t a_sm, int64_t a_sk,
+                           const float *B, int64_t b_sk, int64_t b_sn,
+                           const float *bias, int64_t bias_sn, int act,
+                           double *C, int64_t c_sm, int64_t c_sn,
+                           double *S, int threads)
+{
+    if (M < 0 || N < 0 || K < 0 || (act != 0 && act != 1)) return 1;
+    int nt = use_threads(threads);
+    (void)nt;
+#pragma omp parallel for num_threads(nt) schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        for (int64_t n = 0; n < N; ++n) {
+            double acc = 0.0, sab = 0.0;
+            for (int64_t k = 0; k < K; ++k) {
+                double p = (double)A[m * a_sm + k * a_sk] * (double)B[k * b_sk + n * b_sn];
+                acc += p;
+                sab += fabs(p);
+            }
+            double b = bias ? (double)bias[n * bias_sn] : 0.0;
+            double r = acc + b;
+            if (act == 1 && r < 0.0) r = 0.0;
+            C[m * c_sm + n * c_sn] = r;
+            if (S) S[m * N + n] = sab + fabs(b);
+        }
+    }
+    return 0;
+}
+
 /* Selected elements only: (pm[i], pn[i]) -> out[i], sabs[i]. No accumulate input. */
 int sg_ref_matmul_points(int64_t K,
                          const float *A, int64_t a_sm, int64_t a_sk,

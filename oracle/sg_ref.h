@@ -33,6 +33,14 @@ int sg_ref_matmul(int64_t M, int64_t N, int64_t K,
                   const float *B, int64_t b_sk, int64_t b_sn,
                   double *C, int64_t c_sm, int64_t c_sn,
                   double *S, int mode, int threads);
+/* matmul with a fused pointwise consumer (Sections 2.1, 3.3): C[m,n] = act(sum_k A[m,k]*B[k,n] + bias[n]); act 0 identity,
+ * 1 max(., 0); bias may be NULL; overwrite only; S = sum |a*b| + |bias| */
+int sg_ref_matmul_bias_act(int64_t M, int64_t N, int64_t K,
+                           const float *A, int64_t a_sm, int64_t a_sk,
+                           const float *B, int64_t b_sk, int64_t b_sn,
+                           const float *bias, int64_t bias_sn, int act,
+                           double *C, int64_t c_sm, int64_t c_sn,
+                           double *S, int threads);
 /* listed elements (pm[i], pn[i]) of the same product -> out[i], sabs[i]; overwrite only */
 int sg_ref_matmul_points(int64_t K,
                          const float *A, int64_t a_sm, int64_t a_sk,
