@@ -255,6 +255,14 @@ def op_specs(sg, seed, bw_rows=None):
         return (f"{'ColRed2D' if kind == 'colred2d' else 'RowRed2D'} {R}x{C} {dtype}", float(R * C), R * C * es + n_out * 4, dtype,
                 lambda s: (src(s), torch.empty(n_out, device="cuda")), lambda a, o: fn(a, o))
 
+    def mm_fused(Mx, Nx, Kx, dtype, label):
+        # matmul with the pointwise consumer relu(. + bias[n]) folded into its write-back (Sections 2.1, 3.3)
+        es = 2 if dtype == "bf16" else 4
+        return (label, 2.0 * Mx * Nx * Kx, (Mx * Kx + Kx * Nx) * es + Nx * 4 + Mx * Nx * 4, dtype,
+                lambda s: (gpu_operand((Mx, Kx), seed, 10 + s, "uniform", dtype), gpu_operand((Kx, Nx), seed, 40 + s, "uniform", dtype),
+                           gpu_operand((Nx,), seed, 60, "normal", "f32"), torch.empty(Mx, Nx, device="cuda")),
+                lambda a, b, bias, c: sg.sg_matmul_bias_act(a, b, bias, c, sg.SG_ACT_RELU))
+
     paper_shape = (250, 960)      # the one size the paper names for these kernels (caption of its L3 bandwidth figure)
     return {
         "copy2d_f32": bw("copy2d", "f32"), "copy2d_bf16": bw("copy2d", "bf16"),
@@ -277,6 +285,8 @@ def op_specs(sg, seed, bw_rows=None):
         "matmul1024_bf16": mm(1024, 1024, 1024, "bf16", "matmul 1024^3 bf16 (sweep point)"),
         # a sweep shape of about the step's average size per f32 launch: the shape the DRAM-traffic capture is taken on
         "matmul_2048x2048x1024_f32": mm(2048, 2048, 1024, "f32", "matmul 2048x2048x1024 f32 (sweep point)"),
+        "matmul_bias_relu_bf16": mm_fused(4096, 4096, 1024, "bf16", "matmul 4096x4096x1024 bf16 + bias + relu, fused write-back"),
+        "matmul4096x4096x1024_bf16": mm(4096, 4096, 1024, "bf16", "matmul 4096x4096x1024 bf16 (the same product, unfused)"),
         "matmul8192_bf16": mm(8192, 8192, 8192, "bf16", "matmul 8192^3 bf16 (config 5)"),
         "matmul_skinny_bf16": mm(16384, 64, 4096, "bf16", "matmul 16384x64x4096 bf16 (config 5, skinny)"),
         # conv1d config 3: N=32, W=1026, C=64, KW=3, F=128, f32

@@ -73,6 +73,9 @@ typedef enum { SG_F32 = 0, SG_BF16 = 1 } sg_dtype;
 
 enum { SG_OVERWRITE = 0, SG_ACCUMULATE = 1 };
 
+/* Pointwise consumers that sg_matmul_bias_act can fold into the write-back. */
+enum { SG_ACT_NONE = 0, SG_ACT_RELU = 1 };
+
 /* Kernel families, for sg_set_kernel_override(). */
 enum {
     SG_KERNEL_AUTO = 0,
@@ -101,6 +104,28 @@ sg_status sg_matmul(int64_t M, int64_t N, int64_t K,
                     const void *B, int64_t b_stride_k, int64_t b_stride_n,
                     float *C, int64_t c_stride_m, int64_t c_stride_n,
                     sg_dtype in_dtype, int mode, sg_stream_t stream);
+
+/*
+ * Matrix multiplication with a fused pointwise consumer (the paper fuses tensor operations at the
+ * tiled level, Section 2.1; a pointwise op has identity indexing maps and a lower-dimensional
+ * operand is broadcast, Section 3.3 items 1 and 2):
+ *     C[m,n] = act( sum_k A[m,k] * B[k,n] + bias[n] )
+ * i.e. sg_matmul followed by the generic op with maps (m,n)->(m,n), (m,n)->(n), (m,n)->(m,n) and body
+ * r = act(p + b), evaluated in the contraction's write-back so that the product never goes to memory.
+ *   bias: N f32 values (device), element n at bias[n*bias_stride]; may be NULL (no bias)
+ *   act : SG_ACT_NONE (identity) or SG_ACT_RELU (max(., 0)); other values SG_ERR_UNSUPPORTED
+ * C is overwritten (there is no accumulating form: the consumer is not linear).  An empty reduction
+ * (K = 0) writes act(bias[n]).  A, B, C, in_dtype, stream as for sg_matmul; the sum is accumulated in
+ * f32, bias added and act applied in f32.  With a unit bias stride and a 16-byte aligned bias the call
+ * takes the tensor-core path where sg_matmul would (one work item per tile: a split reduction or a
+ * stream-K tail cannot apply a non-linear consumer to partial sums); otherwise the CUDA-core kernel.
+ */
+sg_status sg_matmul_bias_act(int64_t M, int64_t N, int64_t K,
+                             const void *A, int64_t a_stride_m, int64_t a_stride_k,
+                             const void *B, int64_t b_stride_k, int64_t b_stride_n,
+                             const float *bias, int64_t bias_stride, int act,
+                             float *C, int64_t c_stride_m, int64_t c_stride_n,
+                             sg_dtype in_dtype, sg_stream_t stream);
 
 /*
  * 1-D convolution, input layout NWC, filter layout WCF, output NWF

@@ -26,7 +26,7 @@ EXPORTS = [
     "sg_depthwise_conv2d_nhwc_hwc", "sg_copy2d", "sg_transpose2d", "sg_colred2d", "sg_rowred2d", "sg_check", "sg_status_string",
     "sg_version", "sg_last_kernel", "sg_launch_count", "sg_set_kernel_override", "sg_set_tile_override",
     "sg_last_tile_choice", "sg_last_stream_k", "sg_shutdown", "sg_last_kernel_name", "sg_selftest_wait_timeout",
-    "sg_tensor_map_cache_stats",
+    "sg_tensor_map_cache_stats", "sg_matmul_bias_act",
 ]
 
 
@@ -48,6 +48,8 @@ def lib() -> ctypes.CDLL:
         p64 = ctypes.POINTER(ctypes.c_int64)
         L.sg_matmul.argtypes = [i64, i64, i64, vp, i64, i64, vp, i64, i64, vp, i64, i64, ci, ci, vp]
         L.sg_matmul.restype = ci
+        L.sg_matmul_bias_act.argtypes = [i64, i64, i64, vp, i64, i64, vp, i64, i64, vp, i64, ci, vp, i64, i64, ci, vp]
+        L.sg_matmul_bias_act.restype = ci
         L.sg_conv1d_nwc_wcf.argtypes = [i64] * 8 + [vp, p64, vp, p64, vp, p64, ci, ci, vp]
         L.sg_conv1d_nwc_wcf.restype = ci
         L.sg_conv2d_nhwc_hwcf.argtypes = [i64] * 13 + [vp, p64, vp, p64, vp, p64, ci, ci, vp]
@@ -130,6 +132,25 @@ def sg_matmul(A: torch.Tensor, B: torch.Tensor, C: torch.Tensor, mode: int = SG_
                          _ptr(C), C.stride(0), C.stride(1), _dtype_code(A), mode, _stream(stream))
     if rc != SG_OK:
         raise SgError(rc, "sg_matmul")
+    return C
+
+
+SG_ACT_NONE, SG_ACT_RELU = 0, 1
+
+
+def sg_matmul_bias_act(A: torch.Tensor, B: torch.Tensor, bias, C: torch.Tensor, act: int = SG_ACT_NONE, stream=None) -> torch.Tensor:
+    """C[m,n] = act(sum_k A[m,k]*B[k,n] + bias[n]); bias an f32 vector of N values or None; C is overwritten."""
+    M, K = A.shape
+    K2, N = B.shape
+    if K != K2 or tuple(C.shape) != (M, N) or C.dtype != torch.float32 or A.dtype != B.dtype:
+        raise ValueError("shape or dtype mismatch")
+    if bias is not None and (tuple(bias.shape) != (N,) or bias.dtype != torch.float32):
+        raise ValueError("bias must be an f32 vector of N values")
+    rc = lib().sg_matmul_bias_act(M, N, K, _ptr(A), A.stride(0), A.stride(1), _ptr(B), B.stride(0), B.stride(1),
+                                  _ptr(bias) if bias is not None else None, bias.stride(0) if bias is not None else 0, int(act),
+                                  _ptr(C), C.stride(0), C.stride(1), _dtype_code(A), _stream(stream))
+    if rc != SG_OK:
+        raise SgError(rc, "sg_matmul_bias_act")
     return C
 
 

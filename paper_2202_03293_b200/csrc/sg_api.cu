@@ -19,6 +19,12 @@ constexpr int64_t kTileSlack = 1 << 20;   // head room for extents rounded up to
 
 sg_status run(const Problem &p, const void *In, const void *Flt, float *O, cudaStream_t stream) {
     if (p.M == 0 || p.N == 0) return SG_OK;                       // nothing to write
+    if (p.K == 0 && (p.bias != nullptr || p.act != SG_ACT_NONE)) {
+        // empty reduction under a fused consumer: act(bias), written by the CUDA-core kernel's write-back
+        if (launch_ffma(p, In, Flt, O, stream) != cudaSuccess) return SG_ERR_CUDA;
+        t_last_kernel = SG_KERNEL_FFMA;
+        return SG_OK;
+    }
     if (p.K == 0) {                                               // empty reduction: the sum is 0
         if (p.accumulate) return SG_OK;
         return launch_zero_fill(p, O, stream) == cudaSuccess ? SG_OK : SG_ERR_CUDA;
@@ -84,6 +90,35 @@ sg_status sg_matmul(int64_t M, int64_t N, int64_t K, const void *A, int64_t a_st
     p.k_kh = 0; p.k_kw = 0; p.k_c = b_stride_k; p.k_f = b_stride_n;
     p.o_n = 0; p.o_h = 0; p.o_w = c_stride_m; p.o_f = c_stride_n;
     p.in_bf16 = in_dtype == SG_BF16; p.accumulate = mode == SG_ACCUMULATE; p.spatial_rank = 0;
+    return run(p, A, B, C, static_cast<cudaStream_t>(stream));
+}
+
+sg_status sg_matmul_bias_act(int64_t M, int64_t N, int64_t K, const void *A, int64_t a_stride_m, int64_t a_stride_k,
+                             const void *B, int64_t b_stride_k, int64_t b_stride_n, const float *bias, int64_t bias_stride,
+                             int act, float *C, int64_t c_stride_m, int64_t c_stride_n, sg_dtype in_dtype, sg_stream_t stream) {
+    if (M < 0 || N < 0 || K < 0) return SG_ERR_INVALID_ARG;
+    sg_status st = check_common(A, B, C, in_dtype, SG_OVERWRITE);
+    if (st != SG_OK) return st;
+    if (act != SG_ACT_NONE && act != SG_ACT_RELU) return SG_ERR_UNSUPPORTED;
+    if (bias && reinterpret_cast<uintptr_t>(bias) % 4) return SG_ERR_ALIGNMENT;
+    if (!fits(M) || !fits(N) || !fits(K)) return SG_ERR_UNSUPPORTED;
+    const bool has_out = M > 0 && N > 0;
+    if (has_out && !C) return SG_ERR_INVALID_ARG;
+    if (has_out && K > 0 && (!A || !B)) return SG_ERR_INVALID_ARG;
+    if (a_stride_m < 0 || a_stride_k < 0 || b_stride_k < 0 || b_stride_n < 0 || c_stride_m < 0 || c_stride_n < 0 || bias_stride < 0)
+        return SG_ERR_INVALID_ARG;
+    if ((M > 1 && c_stride_m == 0) || (N > 1 && c_stride_n == 0)) return SG_ERR_INVALID_ARG;
+    Problem p{};
+    p.M = (int)M; p.N = (int)N; p.K = (int)K;
+    p.batch = 1; p.Ho = 1; p.Wo = (int)M;
+    p.KH = 1; p.KW = 1; p.C = (int)K;
+    p.Hin = 1; p.Win = (int)M;
+    p.sh = p.sw = p.dh = p.dw = 1;
+    p.i_n = 0; p.i_h = 0; p.i_w = a_stride_m; p.i_c = a_stride_k;
+    p.k_kh = 0; p.k_kw = 0; p.k_c = b_stride_k; p.k_f = b_stride_n;
+    p.o_n = 0; p.o_h = 0; p.o_w = c_stride_m; p.o_f = c_stride_n;
+    p.in_bf16 = in_dtype == SG_BF16; p.accumulate = 0; p.spatial_rank = 0;
+    p.bias = bias; p.bias_f = bias_stride; p.act = act;
     return run(p, A, B, C, static_cast<cudaStream_t>(stream));
 }
 

@@ -175,6 +175,21 @@ ffma_kernel(Problem p, const T *__restrict__ In, const T *__restrict__ Flt, floa
         __syncthreads();
     }
 
+    // ---- fused pointwise consumer (Sections 2.1, 3.3): r = act(acc + bias[f]), the bias broadcast along the rows ----
+    if (p.bias != nullptr || p.act != SG_ACT_NONE) {
+#pragma unroll
+        for (int jh = 0; jh < 2; ++jh)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int n = n0 + jh * 64 + tx * 4 + j;
+                const float b = (p.bias != nullptr && n < p.N) ? p.bias[(int64_t)n * p.bias_f] : 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float v = acc[i][jh * 4 + j] + b;
+                    acc[i][jh * 4 + j] = (p.act == SG_ACT_RELU && v < 0.f) ? 0.f : v;
+                }
+            }
+    }
     // ---- write-back: O = acc  or  O = O_in + acc ----
 #pragma unroll
     for (int i = 0; i < 8; ++i) {

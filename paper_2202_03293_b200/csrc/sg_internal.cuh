@@ -29,6 +29,10 @@ struct Problem {
     int in_bf16;             // 1: inputs are bf16, 0: f32
     int accumulate;          // 1: O = O_in + result
     int spatial_rank;        // 0 matmul, 1 conv1d, 2 conv2d
+    // fused pointwise consumer of the write-back (overwrite mode only): O = act(acc + bias[f])
+    const float *bias;       // f32 vector over f (device), or null
+    int64_t bias_f;          // its element stride
+    int act;                 // SG_ACT_NONE or SG_ACT_RELU
 };
 
 // Launchers (each returns the cudaError_t of its launch).

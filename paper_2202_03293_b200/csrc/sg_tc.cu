@@ -70,6 +70,8 @@ struct TcParams {
     int b_blocked;       // 1: the filter map is blocked by sub-tile columns: one TMA load fetches the whole filter tile
     int sk_first_tile;   // stream-K tail: tiles from this one on are not dealt out whole; their k-blocks, taken as one
     int sk_units;        //   sequence, are cut into equal runs of `sk_units` k-blocks, one run per CTA (or pair); 0 = no tail
+    const float *bias;   // fused pointwise consumer of the write-back: O = act(acc + bias[column]); null = no bias
+    int act;             // SG_ACT_NONE or SG_ACT_RELU (only with one work item per tile and in overwrite mode)
     int wait_prior;      // the launch may start before the kernel ahead of it in the stream has finished (programmatic
                          // dependent launch).  1: that kernel is this library's clearing kernel, which touches only the
                          // output: the stores wait for it (griddepcontrol.wait), the loads need not.  2: it is any
@@ -686,6 +688,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant
                 uint32_t r[32];
                 tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + j * 32), r);
                 tmem_ld_wait();
+                if (p.bias != nullptr || p.act != SG_ACT_NONE) {
+                    // fused pointwise consumer (Sections 2.1, 3.3): r = act(acc + bias[column]); the bias loads are
+                    // warp-uniform 16-byte loads (every lane holds the same 32 columns of its own row)
+                    const int x = n0 + j * 32;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (p.bias != nullptr && x + 4 * c < p.N) b = __ldg(reinterpret_cast<const float4 *>(p.bias + x) + c);
+                        const float bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            float v = __uint_as_float(r[4 * c + e]) + bv[e];
+                            r[4 * c + e] = __float_as_uint((p.act == SG_ACT_RELU && v < 0.f) ? 0.f : v);
+                        }
+                    }
+                }
                 const int sb = chunk_count & 1;
                 // staging tile sb was last read by the store of two chunks ago, whose issuer waited for
                 // that read before the previous chunk's epi_sync
@@ -1065,6 +1083,11 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     const int64_t pitch_limit = (int64_t)1 << 40;
     if (a_pitch * es >= pitch_limit || b_pitch * es >= pitch_limit || p.o_w * 4 >= pitch_limit) return SG_ERR_UNSUPPORTED;
 
+    // a fused consumer: unit-stride, 16-byte aligned bias (the epilogue reads it in float4); overwrite mode only
+    const bool fused = p.bias != nullptr || p.act != SG_ACT_NONE;
+    if (fused && (p.accumulate || p.spatial_rank != 0)) return SG_ERR_UNSUPPORTED;
+    if (p.bias != nullptr && (p.bias_f != 1 || reinterpret_cast<uintptr_t>(p.bias) % 16)) return SG_ERR_UNSUPPORTED;
+
     LaunchCtx ctx{nullptr, 0, stream};
     Overrides ov;
     ctx.dev = device_state(&ctx.device, &ov);
@@ -1079,6 +1102,8 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
     tp.num_kb = p.KH * p.KW * tp.kb_per_tap;
     tp.Ho = p.Ho; tp.Wo = p.Wo; tp.sh = p.sh; tp.sw = p.sw; tp.dh = p.dh; tp.dw = p.dw;
     tp.accumulate = p.accumulate;
+    tp.bias = p.bias; tp.act = p.act;
+    if (fused) { ov.split = 1; ov.sk = 0; }      // the consumer is not linear: whole reductions only
 
     // ---- input operand ----
     if (p.spatial_rank == 0) {
@@ -1148,6 +1173,7 @@ sg_status launch_tensor(const Problem &p, const void *In, const void *Flt, float
         // (a forced pair count that no variant can honour on this shape is dropped in a second pass)
         for (int pass = 0; pass < 2 && pick < 0; ++pass)
         for (int i = 0; i < kNumVariants; ++i) {
+            // (forced == 1 for a fused consumer: one work item per tile)
             const Variant &v = kVariants[i];
             if (pass == 0 && ov.cg > 0 && v.cg != ov.cg && !(v.cg == 1 && p.M <= BM)) continue;
             if (f32 && v.bn == 256 && v.cg == 1) continue;       // not built (shared-memory budget)
